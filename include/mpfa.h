@@ -1,0 +1,200 @@
+/*
+ * mpfa.h - C ABI of the QK4PV8 mixed-precision attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the two stages of the paper's Algorithm 1:
+ *   stage 1 (lines 1-5, Sections 4.2-4.3): sequence centering of Q and K, NVFP4
+ *     quantization of the centered tensors (E2M1 values, one E4M3 scale per 16
+ *     head-dimension elements, Eq. 1), FP8 E4M3 quantization of V, and the
+ *     compensation vector Delta_S (Eq. 9);
+ *   stage 2 (lines 6-20, Sections 4.1, 5.1-5.3): the attention main loop that consumes
+ *     only those quantized tensors - a rank-one BF16 MMA seeding the score accumulator
+ *     with Delta_S (Eq. 11), the block-scaled FP4 MMA, online softmax (Eq. 3-6) with P
+ *     quantized to E4M3 at the fixed scale 448, the FP8 PV MMA - for causal GQA
+ *     prefill and for split-KV decode over a paged KV cache.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its name starts with h_.  The caller owns
+ *     all buffers.  No call allocates, frees or synchronises: work is only enqueued on
+ *     `stream`.
+ *   - head_dim is 128.  H_q must be a multiple of H_kv (GQA); q head hq uses kv head
+ *     hq / (H_q / H_kv).
+ *   - Inputs Q, K, V are BF16, token-major: [B, N, H, 128].  Outputs are BF16
+ *     [B, N_q, H_q, 128] (prefill) or [B, H_q, 128] (decode).
+ *   - Every function returns an mpfa_status (0 = success, negative = error).  Argument,
+ *     shape and alignment errors are detected on the host before anything is launched.
+ *     Errors found on the device (a bounded wait that gave up, a page index out of range)
+ *     are OR-ed into *device_status, which the caller reads after synchronising.
+ *   - Results are deterministic: the same inputs give bit-identical outputs.
+ *
+ * Physical layouts (all offsets in bytes, N_pad = N rounded up to a multiple of 128)
+ *   NVFP4 tensor ("tile layout", mpfa_fp4_tensor):
+ *     codes  [B, H, N_pad, 64]   two E2M1 codes per byte, even channel in bits 3:0;
+ *                                rows N..N_pad-1 are zero.
+ *     sf     [B, H, N_pad/128, 2, 512]   unsigned E4M3 block scales.  Token t, 16-channel
+ *                                block g (0..7) lives in tile t/128, half g/4, at byte
+ *                                (r%32)*16 + (r/32)*4 + (g%4) with r = t%128 - the
+ *                                32-lane x 16-byte image the tensor core's scale-factor
+ *                                copy expects.  mpfa_sf_offset() is this map.
+ *   Delta_S  BF16 [B, H_q, N_kv_pad], in units of (true logit) / (q_gscale * k_gscale).
+ *   V        E4M3 [B, H_kv, N_kv_pad, 128], pad rows zero.
+ *   Paged KV cache (mpfa_paged_kv): 64-token pages; within a page and kv head the bytes are
+ *     ordered for the decode kernel's register fragments, see mpfa_paged_kv below.
+ */
+#ifndef MPFA_H_
+#define MPFA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int mpfa_status;
+enum {
+  MPFA_OK = 0,
+  MPFA_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, inconsistent struct fields */
+  MPFA_ERR_UNSUPPORTED = -2, /* H_q % H_kv != 0, page_size != 64, GQA group > 8 (decode), ... */
+  MPFA_ERR_ALIGNMENT = -3,   /* a buffer is not aligned as documented */
+  MPFA_ERR_WORKSPACE = -4,   /* workspace_bytes smaller than the matching *_workspace_bytes() */
+  MPFA_ERR_ARCH = -5,        /* the current device is not compute capability 10.x */
+  MPFA_ERR_CUDA = -6,        /* a CUDA call failed; see mpfa_last_cuda_error() */
+  MPFA_ERR_TIMEOUT = -7      /* reserved for device_status: a bounded device wait gave up */
+};
+
+/* bits OR-ed into *device_status by the kernels */
+enum {
+  MPFA_DEV_TIMEOUT = 1,  /* a bounded mbarrier wait expired; the output is invalid */
+  MPFA_DEV_BAD_PAGE = 2  /* a page-table entry was outside [0, num_pages); that page was skipped */
+};
+
+/* flags of mpfa_quantize_qk / mpfa_quantize_kv_paged */
+enum {
+  MPFA_SMOOTH = 1,       /* center with the sequence means and emit Delta_S (Section 4.2-4.3).
+                            Without it: the paper's "direct" variant, means = 0, no Delta_S. */
+  MPFA_STATS_FROZEN = 2  /* read means and tensor scales from `stats` instead of computing them
+                            (decode-time tokens are centered against the frozen prefill
+                            statistics, Section 6). */
+};
+
+/* Per-request statistics, caller-owned.  Written by the quantizers unless
+ * MPFA_STATS_FROZEN, read by them when it is set, and read by the attention calls
+ * (tensor scales only). */
+typedef struct {
+  float *q_mean;   /* [B, H_q, 128]  Eq. 7 */
+  float *k_mean;   /* [B, H_kv, 128] Eq. 7 */
+  float *q_gscale; /* [B] per-tensor scale d_Q = max|Q - mean| / 2688 (1.0 if the tensor is all zero) */
+  float *k_gscale; /* [B] d_K */
+} mpfa_stats;
+
+/* One NVFP4 tensor in the tile layout described at the top. codes and sf must be
+ * 1024-byte aligned.  Sizes: mpfa_fp4_codes_bytes / mpfa_fp4_sf_bytes. */
+typedef struct {
+  uint8_t *codes;
+  uint8_t *sf;
+  int32_t B, H, N;
+} mpfa_fp4_tensor;
+
+/* Paged KV cache for decode: num_pages physical pages of 64 tokens, shared by all
+ * requests through a page table.  Inside a (page, kv head) slab the bytes are ordered so
+ * that every 16-byte load of the decode kernel is one thread's tensor-core fragment.
+ * With token t (0..63) of the page:
+ *   k_codes [P, H_kv, 4096]  byte j (0..7) of 16-channel block g (0..7) of token t at
+ *             (t/8)*512 + ((t%8)*4 + j/2)*16 + g*2 + (j%2)
+ *   k_sf    [P, H_kv, 512]   block g of token t at t*8 + g
+ *   v_fp8   [P, H_kv, 8192]  channel c (0..127) of token t, with u = t%32, at
+ *             (t/32)*4096 + (c/16)*512 + ((c%8)*4 + (u%8)/2)*16 + ((c/8)%2)*8 + (u/16)*4 + ((u/8)%2)*2 + (u%2)
+ *   delta_s [P, H_q, 64]     BF16, token t at index t (NULL when compensation is off)
+ * mpfa_paged_k_offset / mpfa_paged_v_offset are these maps.  All pools 256-byte aligned. */
+typedef struct {
+  uint8_t *k_codes;
+  uint8_t *k_sf;
+  uint8_t *v_fp8;
+  void *delta_s_bf16;
+  int32_t num_pages;
+  int32_t page_size; /* must be 64 */
+} mpfa_paged_kv;
+
+/* ---- stage 1: Algorithm 1 lines 1-5 -------------------------------------------------- */
+
+/* Means (Eq. 7), centering, per-tensor scales, NVFP4 quantization (Eq. 1) of Q and K,
+ * and Delta_S (Eq. 9; needs both tensors' statistics, written when k_bf16 != NULL).
+ *   q_bf16 [B, N_q, H_q, 128] or NULL (quantize K only; needs MPFA_STATS_FROZEN for the Q side
+ *          if MPFA_SMOOTH, because Delta_S uses the query mean);
+ *   k_bf16 [B, N_kv, H_kv, 128] or NULL (quantize Q only);
+ *   q_out / k_out: tile-layout tensors with B, H, N filled in by the caller;
+ *   delta_s_bf16 [B, H_q, N_kv_pad]: required iff MPFA_SMOOTH and k_bf16 != NULL;
+ *   workspace: mpfa_quantize_workspace_bytes() bytes, 256-byte aligned; contents are
+ *          scratch (column sums and maxima), overwritten by every call.
+ * All arithmetic is specified bit by bit (FP64 column sums, one rounding to FP32, IEEE
+ * divisions); outputs are reproducible to the bit. */
+mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, int B, int N_q, int N_kv, int H_q,
+                             int H_kv, int flags, mpfa_stats *h_stats, mpfa_fp4_tensor *h_q_out,
+                             mpfa_fp4_tensor *h_k_out, void *delta_s_bf16, void *workspace,
+                             size_t workspace_bytes, void *stream);
+
+/* Algorithm 1 line 4: V is not centered; code = E4M3(v / v_scale), round to nearest even,
+ * saturating at +-448.  v_bf16 [B, N_kv, H_kv, 128] -> v_fp8 [B, H_kv, N_kv_pad, 128]
+ * (1024-byte aligned).  v_scale = 1.0f is the plain cast. */
+mpfa_status mpfa_quantize_v(const void *v_bf16, int B, int N_kv, int H_kv, float v_scale, uint8_t *v_fp8,
+                            void *stream);
+
+/* The same arithmetic for ONE request, written through its page-table row into the paged
+ * cache (Section 6: low-bit K/V cache writes fused with quantization and compensation
+ * generation).  k_bf16, v_bf16 [N_tokens, H_kv, 128] are the tokens at positions
+ * [first_token, first_token + N_tokens) of the request; page_table_row[i] is the physical
+ * page of tokens [64 i, 64 i + 64).  h_stats points at this request's statistics
+ * (B = 1 slices).  Without MPFA_STATS_FROZEN (allowed only when first_token == 0) k_mean and
+ * k_gscale are computed from these tokens; q_mean and q_gscale are always read.
+ * Slots of the last page beyond the written tokens are zero-filled. */
+mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_bf16, int N_tokens, int first_token,
+                                   int H_q, int H_kv, int flags, mpfa_stats *h_stats, float v_scale,
+                                   const mpfa_paged_kv *h_kv, const int32_t *page_table_row,
+                                   void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- stage 2: Algorithm 1 lines 6-20 -------------------------------------------------- */
+
+/* QK4PV8 prefill.  q: [B, H_q, N_q] tile-layout tensor, k: [B, H_kv, N_kv], v_fp8 and
+ * delta_s_bf16 as written by stage 1 (delta_s_bf16 == NULL: no compensation MMA).
+ * KV blocks of 128 keys are visited from the last visible block down to block 0
+ * (Section 4.1); causal != 0 masks key j for query i when j > i + N_kv - N_q.
+ * softmax_scale is folded into the exponent together with the tensor scales
+ * (Section 5.1): lambda = softmax_scale * log2(e) * q_gscale[b] * k_gscale[b].
+ * out_bf16 [B, N_q, H_q, 128]; out_f32 (optional, may be NULL) receives the same values
+ * before the final BF16 rounding.  device_status: one int32, caller-zeroed. */
+mpfa_status mpfa_prefill(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tensor *h_k, const uint8_t *v_fp8,
+                         const void *delta_s_bf16, const mpfa_stats *h_stats, float v_scale, int causal,
+                         float softmax_scale, void *out_bf16, float *out_f32, int32_t *device_status,
+                         void *stream);
+
+/* QK4PV8 decode (Section 5.3): one query token per request (q: tile-layout tensor with
+ * N = 1, centered with the frozen means), its first seq_lens[b] keys found through
+ * page_table [B, max_pages_per_req].  Each (request, kv head, 1024-token partition) keeps a
+ * local (m, l, O) state for its GQA group in `workspace`; a second kernel merges the
+ * partitions by log-sum-exp.  The number of partitions is fixed by max_seq_len, so the call
+ * sequence does not depend on seq_lens.  out_bf16 [B, H_q, 128]; out_f32 optional. */
+mpfa_status mpfa_decode(const mpfa_fp4_tensor *h_q, const mpfa_paged_kv *h_kv, const int32_t *page_table,
+                        int max_pages_per_req, const int32_t *seq_lens, const mpfa_stats *h_stats,
+                        float v_scale, float softmax_scale, void *out_bf16, float *out_f32, void *workspace,
+                        size_t workspace_bytes, int32_t *device_status, void *stream);
+
+/* ---- sizes, layout maps, diagnostics (host only, no CUDA calls) ----------------------- */
+size_t mpfa_quantize_workspace_bytes(int B, int H_q, int H_kv);
+size_t mpfa_decode_workspace_bytes(int B, int H_q, int H_kv, int max_pages_per_req);
+size_t mpfa_fp4_codes_bytes(int B, int H, int N);
+size_t mpfa_fp4_sf_bytes(int B, int H, int N);
+size_t mpfa_delta_s_bytes(int B, int H_q, int N_kv);
+size_t mpfa_v_fp8_bytes(int B, int H_kv, int N_kv);
+/* byte offset of the scale of (b, h, token, block) inside mpfa_fp4_tensor.sf */
+size_t mpfa_sf_offset(int H, int N, int b, int h, int token, int block);
+/* byte offsets inside one (page, kv head) slab of the paged cache */
+size_t mpfa_paged_k_offset(int token, int block, int byte_in_block);
+size_t mpfa_paged_v_offset(int token, int channel);
+const char *mpfa_status_string(mpfa_status s);
+int mpfa_last_cuda_error(void);
+int mpfa_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MPFA_H_ */

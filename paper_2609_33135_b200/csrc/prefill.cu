@@ -1,0 +1,517 @@
+// QK4PV8 prefill (Algorithm 1 lines 6-20) for sm_100a.
+//
+// One CTA owns one 128-row query tile of one q head and walks its KV blocks (128 keys)
+// from the last visible block down to block 0 (Section 4.1).  Roles:
+//   warp 0      TMA producer: K codes (tensor map, 64B swizzle), K scale factors and
+//               Delta_S (bulk copies) and V (tensor map, 128B swizzle) into a 3-stage ring;
+//   warp 1      MMA issuer: per block a rank-one BF16 MMA seeds S with 1 x Delta_S
+//               (Eq. 11), two block-scaled FP4 MMAs (K = 64 each) accumulate Q K^T into
+//               the same TMEM columns, and four FP8 MMAs (A = P_hat from TMEM, B = V from
+//               shared memory, MN-major) accumulate P V into O;
+//   warps 4-7   softmax: one thread per row; mask, running max, 2^(lam S - lam m), row sum
+//               from the unquantized P, P -> E4M3 at the fixed scale 448 written back over
+//               the first 32 columns of the score buffer (Algorithm 1 lines 11-14);
+//   warps 8-11  correction + epilogue: O *= alpha whenever a row's maximum moved
+//               (Eq. 6), final O / (448 l) * v_scale -> BF16.
+// Tensor memory (512 columns): S0 [0,128) S1 [128,256) O [256,384), scale factors of Q
+// [384,392) and of the two in-flight K blocks [392,400) [400,408).  The score buffer is
+// double-buffered over KV blocks so Q K^T of block t+1 overlaps the softmax of block t and
+// P V of block t overlaps the softmax of block t+1.
+//
+// Every mbarrier wait is bounded; on expiry the CTA raises MPFA_DEV_TIMEOUT in
+// *device_status, all roles leave their loops, outstanding TMA copies are drained and
+// tensor memory is released.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp8.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace mpfa {
+namespace {
+
+constexpr int KSTAGES = 3;
+constexpr int VSTAGES = 3;
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // 2 s: far beyond any legitimate wait
+constexpr int NTHREADS = 384;
+
+constexpr uint32_t OFF_Q = 0;
+constexpr uint32_t OFF_K = OFF_Q + 8192;
+constexpr uint32_t OFF_V = OFF_K + KSTAGES * 8192;
+constexpr uint32_t OFF_DELTA = OFF_V + VSTAGES * 16384;
+constexpr uint32_t OFF_ONES = OFF_DELTA + KSTAGES * 4096;
+constexpr uint32_t OFF_SFQ = OFF_ONES + 4096;
+constexpr uint32_t OFF_SFK = OFF_SFQ + 1024;
+constexpr uint32_t OFF_ALPHA = OFF_SFK + KSTAGES * 1024;
+constexpr uint32_t OFF_L = OFF_ALPHA + 2 * 128 * 4;
+constexpr uint32_t OFF_BAR = OFF_L + 128 * 4;
+enum {
+  BAR_Q_FULL = 0,
+  BAR_K_FULL = 1,
+  BAR_K_EMPTY = BAR_K_FULL + KSTAGES,
+  BAR_V_FULL = BAR_K_EMPTY + KSTAGES,
+  BAR_V_EMPTY = BAR_V_FULL + VSTAGES,
+  BAR_S_FULL = BAR_V_EMPTY + VSTAGES,
+  BAR_P_FULL = BAR_S_FULL + 2,
+  BAR_A_FULL = BAR_P_FULL + 2,
+  BAR_O_FULL = BAR_A_FULL + 2,
+  BAR_O_READY = BAR_O_FULL + 1,
+  BAR_L_FULL = BAR_O_READY + 1,
+  NUM_BARS = BAR_L_FULL + 1
+};
+constexpr uint32_t OFF_MISC = OFF_BAR + NUM_BARS * 8;   // tmem base, abort flag
+constexpr uint32_t SMEM_BYTES = OFF_MISC + 16 + 1024;   // + slack for the 1024-byte alignment
+
+constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_O = 256, TM_SFQ = 384, TM_SFK0 = 392, TM_SFK1 = 400;
+constexpr uint32_t TMEM_COLS = 512;
+
+struct PrefillParams {
+  const uint8_t *q_sf;
+  const uint8_t *k_sf;
+  const __nv_bfloat16 *delta;  // may be null
+  const float *q_gscale;
+  const float *k_gscale;
+  __nv_bfloat16 *out;
+  float *out_f32;  // may be null
+  int32_t *status;
+  int B, N_q, N_kv, H_q, H_kv, nq_tiles, nk_tiles;
+  int causal;
+  float softmax_scale, v_scale;
+};
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct Ctx {
+  uint32_t bars;      // shared address of barrier 0
+  volatile int *abort_flag;
+  int32_t *status;
+  __device__ __forceinline__ uint32_t bar(int i) const { return bars + 8u * (uint32_t)i; }
+  // Wait bounded in wall-clock time (try_wait itself may suspend the thread for a
+  // system-dependent interval, so an iteration count alone does not bound the wait).
+  // Also gives up as soon as another role has failed.
+  __device__ __forceinline__ bool wait(int i, uint32_t parity) const {
+    const uint32_t a = bar(i);
+    if (mbar_try_wait(a, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    for (;;) {
+      if (mbar_try_wait(a, parity)) return true;
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) break;
+    }
+    *abort_flag = 1;
+    atomicOr(status, MPFA_DEV_TIMEOUT);
+    return false;
+  }
+};
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+               const __grid_constant__ CUtensorMap tm_v, const PrefillParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // ---- work item: kv head outermost so co-resident CTAs share K/V through L2; within a
+  // head the longest (latest) query tiles first, the GQA group innermost.
+  const int G = p.H_q / p.H_kv;
+  int w = blockIdx.x;
+  const int g = w % G;
+  w /= G;
+  const int qt = p.nq_tiles - 1 - (w % p.nq_tiles);
+  w /= p.nq_tiles;
+  const int hk = w % p.H_kv;
+  const int b = w / p.H_kv;
+  const int hq = hk * G + g;
+
+  const int off = p.N_kv - p.N_q;   // causal masks are bottom-right aligned
+  const int row0 = qt * TILE;
+  const int last_row = min(p.N_q - 1, row0 + TILE - 1);
+  const int last_key = p.causal ? min(p.N_kv - 1, last_row + off) : p.N_kv - 1;
+  const int T = last_key < 0 ? 0 : last_key / TILE + 1;   // KV blocks to visit
+
+  Ctx cx;
+  cx.bars = sbase + OFF_BAR;
+  cx.abort_flag = reinterpret_cast<volatile int *>(smem + OFF_MISC + 4);
+  cx.status = p.status;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + OFF_MISC);
+
+  // ---- one-time setup
+  if (tid == 0) {
+    *cx.abort_flag = 0;
+    mbar_init(cx.bar(BAR_Q_FULL), 1);
+    for (int i = 0; i < KSTAGES; ++i) { mbar_init(cx.bar(BAR_K_FULL + i), 1); mbar_init(cx.bar(BAR_K_EMPTY + i), 1); }
+    for (int i = 0; i < VSTAGES; ++i) { mbar_init(cx.bar(BAR_V_FULL + i), 1); mbar_init(cx.bar(BAR_V_EMPTY + i), 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(cx.bar(BAR_S_FULL + i), 1);
+      mbar_init(cx.bar(BAR_P_FULL + i), 128);
+      mbar_init(cx.bar(BAR_A_FULL + i), 128);
+    }
+    mbar_init(cx.bar(BAR_O_FULL), 1);
+    mbar_init(cx.bar(BAR_O_READY), 128);
+    mbar_init(cx.bar(BAR_L_FULL), 128);
+    mbar_init_fence();
+    prefetch_tmap(&tm_q);
+    prefetch_tmap(&tm_k);
+    prefetch_tmap(&tm_v);
+  }
+  // rank-one operands: MN-major, 128B swizzle, K = 16.  Row k = 0 of each 64-element half
+  // holds the data (ones / Delta_S), every other row stays zero for the CTA's lifetime.
+  for (int i = tid; i < (KSTAGES * 4096 + 4096) / 16; i += NTHREADS)
+    reinterpret_cast<uint4 *>(smem + OFF_DELTA)[i] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+  if (tid < 128) reinterpret_cast<uint16_t *>(smem + OFF_ONES)[(tid >> 6) * 1024 + (tid & 63)] = 0x3F80;  // 1.0
+  fence_proxy_async_smem();
+  if (warp == 2) {
+    tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tm = *tmem_slot;
+
+  const bool has_delta = p.delta != nullptr;
+  const size_t q_row = ((size_t)b * p.H_q + hq) * (size_t)(p.nq_tiles * TILE) + row0;
+  const size_t k_row = ((size_t)b * p.H_kv + hk) * (size_t)(p.nk_tiles * TILE);
+
+  if (warp == 0) {
+    // =========================== TMA producer ===========================
+    if (lane == 0 && T > 0) {
+      int armed = 0;
+      mbar_expect_tx(cx.bar(BAR_Q_FULL), 8192 + 1024);
+      tma_load_2d(sbase + OFF_Q, &tm_q, 0, (int)q_row, cx.bar(BAR_Q_FULL));
+      bulk_load(sbase + OFF_SFQ, p.q_sf + (((size_t)b * p.H_q + hq) * p.nq_tiles + qt) * 1024, 1024,
+                cx.bar(BAR_Q_FULL));
+      bool ok = true;
+      for (int t = 0; t < T && ok; ++t) {
+        const int jb = T - 1 - t;
+        const int ks = t % KSTAGES, vs = t % VSTAGES;
+        if (t >= KSTAGES) ok = cx.wait(BAR_K_EMPTY + ks, (uint32_t)(t / KSTAGES - 1) & 1u);
+        if (!ok) break;
+        mbar_expect_tx(cx.bar(BAR_K_FULL + ks), 8192 + 1024 + (has_delta ? 256 : 0));
+        tma_load_2d(sbase + OFF_K + ks * 8192, &tm_k, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_K_FULL + ks));
+        bulk_load(sbase + OFF_SFK + ks * 1024, p.k_sf + (((size_t)b * p.H_kv + hk) * p.nk_tiles + jb) * 1024, 1024,
+                  cx.bar(BAR_K_FULL + ks));
+        if (has_delta) {
+          const __nv_bfloat16 *d = p.delta + ((size_t)b * p.H_q + hq) * (size_t)(p.nk_tiles * TILE) + (size_t)jb * TILE;
+          bulk_load(sbase + OFF_DELTA + ks * 4096, d, 128, cx.bar(BAR_K_FULL + ks));
+          bulk_load(sbase + OFF_DELTA + ks * 4096 + 2048, d + 64, 128, cx.bar(BAR_K_FULL + ks));
+        }
+        if (t >= VSTAGES) ok = cx.wait(BAR_V_EMPTY + vs, (uint32_t)(t / VSTAGES - 1) & 1u);
+        if (!ok) { armed = -(t + 1); break; }   // K of block t armed, V not
+        mbar_expect_tx(cx.bar(BAR_V_FULL + vs), 16384);
+        tma_load_2d(sbase + OFF_V + vs * 16384, &tm_v, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
+        armed = t + 1;
+      }
+      if (*cx.abort_flag) {
+        // Drain: copies still in flight must land before the CTA's shared memory is released.
+        const int nk = armed < 0 ? -armed : armed, nv = armed < 0 ? -armed - 1 : armed;
+        for (int t = max(0, nk - KSTAGES); t < nk; ++t)
+          mbar_wait_ns(cx.bar(BAR_K_FULL + t % KSTAGES), (uint32_t)(t / KSTAGES) & 1u, WAIT_LIMIT_NS);
+        for (int t = max(0, nv - VSTAGES); t < nv; ++t)
+          mbar_wait_ns(cx.bar(BAR_V_FULL + t % VSTAGES), (uint32_t)(t / VSTAGES) & 1u, WAIT_LIMIT_NS);
+        mbar_wait_ns(cx.bar(BAR_Q_FULL), 0, WAIT_LIMIT_NS);
+      }
+    }
+  } else if (warp == 1) {
+    // =========================== MMA issuer ===========================
+    if (lane == 0 && T > 0) {
+      const uint32_t id_fp4 = idesc_nvfp4(128, 128);
+      const uint32_t id_bf16 = idesc_bf16(128, 128, 1, 1);
+      const uint32_t id_fp8 = idesc_e4m3(128, 128, 0, 1);
+      const uint64_t d_ones = smem_desc(sbase + OFF_ONES, 2048, 1024, SWZ_128B);
+      bool ok = cx.wait(BAR_Q_FULL, 0);
+      if (ok) {
+        tc_fence_after();
+        for (int kc = 0; kc < 2; ++kc)
+          tmem_cp_32x128b_warpx4(tm + TM_SFQ + 4 * kc, smem_desc(sbase + OFF_SFQ + 512 * kc, 0, 128, SWZ_NONE));
+      }
+      auto issue_qk = [&](int t) -> bool {
+        const int ks = t % KSTAGES, sb = t & 1;
+        if (!cx.wait(BAR_K_FULL + ks, (uint32_t)(t / KSTAGES) & 1u)) return false;
+        tc_fence_after();
+        const uint32_t tS = tm + (sb ? TM_S1 : TM_S0);
+        const uint32_t tSFK = tm + (sb ? TM_SFK1 : TM_SFK0);
+        for (int kc = 0; kc < 2; ++kc)
+          tmem_cp_32x128b_warpx4(tSFK + 4 * kc, smem_desc(sbase + OFF_SFK + ks * 1024 + 512 * kc, 0, 128, SWZ_NONE));
+        uint32_t acc = 0;
+        if (has_delta) {
+          mma_bf16_ss(tS, d_ones, smem_desc(sbase + OFF_DELTA + ks * 4096, 2048, 1024, SWZ_128B), id_bf16, 0);
+          acc = 1;
+        }
+        for (int kc = 0; kc < 2; ++kc) {
+          mma_nvfp4_ss(tS, smem_desc(sbase + OFF_Q + 32 * kc, 16, 512, SWZ_64B),
+                       smem_desc(sbase + OFF_K + ks * 8192 + 32 * kc, 16, 512, SWZ_64B), id_fp4,
+                       tm + TM_SFQ + 4 * kc, tSFK + 4 * kc, acc);
+          acc = 1;
+        }
+        mma_commit(cx.bar(BAR_K_EMPTY + ks));
+        mma_commit(cx.bar(BAR_S_FULL + sb));
+        return true;
+      };
+      if (ok) ok = issue_qk(0);
+      for (int t = 0; t < T && ok; ++t) {
+        if (t + 1 < T) ok = issue_qk(t + 1);
+        if (!ok) break;
+        const int sb = t & 1, vs = t % VSTAGES;
+        ok = cx.wait(BAR_P_FULL + sb, (uint32_t)(t >> 1) & 1u) && cx.wait(BAR_O_READY, (uint32_t)t & 1u) &&
+             cx.wait(BAR_V_FULL + vs, (uint32_t)(t / VSTAGES) & 1u);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tP = tm + (sb ? TM_S1 : TM_S0);
+        for (int k4 = 0; k4 < 4; ++k4)
+          mma_e4m3_ts(tm + TM_O, tP + 8 * k4, smem_desc(sbase + OFF_V + vs * 16384 + 4096 * k4, 16, 1024, SWZ_128B),
+                      id_fp8, (t > 0 || k4 > 0) ? 1u : 0u);
+        mma_commit(cx.bar(BAR_V_EMPTY + vs));
+        mma_commit(cx.bar(BAR_O_FULL));
+      }
+    }
+  } else if (warp >= 4 && warp < 8) {
+    // =========================== softmax ===========================
+    const int row = (warp - 4) * 32 + lane;
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const int r_abs = row0 + row;
+    const int limit = p.causal ? min(p.N_kv - 1, r_abs + off) : p.N_kv - 1;   // last visible key
+    const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[b]), p.k_gscale[b]);
+    float m = -INFINITY, l = 0.0f;
+    float *s_alpha = reinterpret_cast<float *>(smem + OFF_ALPHA);
+    bool ok = true;
+    for (int t = 0; t < T; ++t) {
+      const int sb = t & 1;
+      const int key0 = (T - 1 - t) * TILE;
+      ok = __all_sync(0xffffffffu, cx.wait(BAR_S_FULL + sb, (uint32_t)(t >> 1) & 1u));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t tS = tm + (sb ? TM_S1 : TM_S0) + lane_off;
+      const bool need_mask = key0 + TILE - 1 > limit;
+      // pass 1: row maximum (Eq. 3)
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c0 = 0; c0 < TILE; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tS + c0, r);
+        tmem_ld_wait();
+        if (need_mask) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (key0 + c0 + i > limit) r[i] = 0xFF800000u;   // -inf
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+      }
+      const float m_new = fmaxf(m, mx);
+      const float alpha = (m_new == m) ? 1.0f : ex2_approx(__fmul_rn(m - m_new, lam));
+      s_alpha[sb * 128 + row] = alpha;
+      mbar_arrive(cx.bar(BAR_A_FULL + sb));
+      const float neg_mlam = (m_new == -INFINITY) ? 0.0f : -__fmul_rn(m_new, lam);
+      // pass 2: P = 2^(lam S - lam m) (Eq. 4), row sum of the unquantized P (Eq. 5),
+      // P_hat = E4M3(448 P) written over the first 32 columns of this score buffer.
+      float sum0 = 0.0f, sum1 = 0.0f, sum2 = 0.0f, sum3 = 0.0f;
+#pragma unroll
+      for (int c0 = 0; c0 < TILE; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tS + c0, r);
+        tmem_ld_wait();
+        if (need_mask) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (key0 + c0 + i > limit) r[i] = 0xFF800000u;
+        }
+        uint32_t packed[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float p0 = ex2_approx(__fmaf_rn(__uint_as_float(r[4 * i]), lam, neg_mlam));
+          const float p1 = ex2_approx(__fmaf_rn(__uint_as_float(r[4 * i + 1]), lam, neg_mlam));
+          const float p2 = ex2_approx(__fmaf_rn(__uint_as_float(r[4 * i + 2]), lam, neg_mlam));
+          const float p3 = ex2_approx(__fmaf_rn(__uint_as_float(r[4 * i + 3]), lam, neg_mlam));
+          sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+          const uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(p0, 448.0f), __fmul_rn(p1, 448.0f)),
+                                                                 __NV_SATFINITE, __NV_E4M3);
+          const uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(p2, 448.0f), __fmul_rn(p3, 448.0f)),
+                                                                 __NV_SATFINITE, __NV_E4M3);
+          packed[i] = (lo & 0xFFFFu) | (hi << 16);
+        }
+        tmem_st8(tS + (c0 >> 2), packed);
+      }
+      l = __fadd_rn(__fmul_rn(alpha, l), (sum0 + sum1) + (sum2 + sum3));
+      m = m_new;
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(cx.bar(BAR_P_FULL + sb));
+    }
+    reinterpret_cast<float *>(smem + OFF_L)[row] = l;
+    mbar_arrive(cx.bar(BAR_L_FULL));
+  } else if (warp >= 8) {
+    // =========================== correction + epilogue ===========================
+    const int row = (warp - 8) * 32 + lane;
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const int r_abs = row0 + row;
+    const float *s_alpha = reinterpret_cast<const float *>(smem + OFF_ALPHA);
+    const uint32_t tO = tm + TM_O + lane_off;
+    bool ok = true;
+    for (int t = 0; t < T; ++t) {
+      const int sb = t & 1;
+      ok = __all_sync(0xffffffffu, cx.wait(BAR_A_FULL + sb, (uint32_t)(t >> 1) & 1u));
+      if (!ok) break;
+      const float alpha = s_alpha[sb * 128 + row];
+      if (t > 0) {
+        ok = __all_sync(0xffffffffu, cx.wait(BAR_O_FULL, (uint32_t)(t - 1) & 1u));
+        if (!ok) break;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, alpha != 1.0f)) {   // identical result when every alpha is exactly 1
+#pragma unroll
+          for (int c0 = 0; c0 < HEAD_DIM; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(tO + c0, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__fmul_rn(__uint_as_float(r[i]), alpha));
+            tmem_st32(tO + c0, r);
+          }
+          tmem_st_wait();
+        }
+        tc_fence_before();
+      }
+      mbar_arrive(cx.bar(BAR_O_READY));
+    }
+    // final normalisation (Algorithm 1 line 17): O / (448 l) * v_scale -> BF16
+    float l = 0.0f;
+    if (T > 0 && ok) {
+      ok = cx.wait(BAR_O_FULL, (uint32_t)(T - 1) & 1u) && cx.wait(BAR_L_FULL, 0);
+      tc_fence_after();
+      if (ok) l = reinterpret_cast<const float *>(smem + OFF_L)[row];
+    }
+    // tcgen05.ld is warp-collective: every lane loads, only the stores are predicated.
+    const bool warp_ok = __all_sync(0xffffffffu, ok);
+    const bool store = r_abs < p.N_q && (warp_ok || T == 0);
+    const size_t o_off = (((size_t)b * p.N_q + (store ? r_abs : 0)) * p.H_q + hq) * HEAD_DIM;
+    const float denom = __fmul_rn(448.0f, l);
+#pragma unroll
+    for (int c0 = 0; c0 < HEAD_DIM; c0 += 32) {
+      uint32_t r[32];
+      if (T > 0 && warp_ok) {
+        tmem_ld32(tO + c0, r);
+        tmem_ld_wait();
+      }
+#pragma unroll
+      for (int i = 0; i < 32; ++i)
+        r[i] = (l > 0.0f) ? __float_as_uint(__fmul_rn(__fdiv_rn(__uint_as_float(r[i]), denom), p.v_scale)) : 0u;
+      if (store) {
+        if (p.out_f32) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4)
+            *reinterpret_cast<uint4 *>(p.out_f32 + o_off + c0 + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+        }
+#pragma unroll
+        for (int i = 0; i < 32; i += 8) {
+          uint32_t h[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[i + 2 * j]), __uint_as_float(r[i + 2 * j + 1]));
+            h[j] = *reinterpret_cast<uint32_t *>(&v);
+          }
+          *reinterpret_cast<uint4 *>(p.out + o_off + c0 + i) = make_uint4(h[0], h[1], h[2], h[3]);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) tmem_dealloc(tm, TMEM_COLS);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver entry point is looked up through the runtime so the library does not link libcuda.
+mpfa_status get_encoder(EncodeTiledFn *fn) {
+  static EncodeTiledFn cached = nullptr;
+  if (!cached) {
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    MPFA_CUDA_OK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q));
+    if (q != cudaDriverEntryPointSuccess || !ptr) return cuda_fail(cudaErrorNotSupported);
+    cached = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  *fn = cached;
+  return MPFA_OK;
+}
+
+// 2D byte tensor [rows][row_bytes], box = 128 rows x row_bytes, hardware swizzle = row_bytes.
+mpfa_status make_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, uint64_t rows, uint32_t row_bytes) {
+  cuuint64_t dims[2] = {row_bytes, rows};
+  cuuint64_t strides[1] = {row_bytes};
+  cuuint32_t box[2] = {row_bytes, 128};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda_error = (int)r;
+    return MPFA_ERR_CUDA;
+  }
+  return MPFA_OK;
+}
+
+}  // namespace
+}  // namespace mpfa
+
+using namespace mpfa;
+
+extern "C" mpfa_status mpfa_prefill(const mpfa_fp4_tensor *q, const mpfa_fp4_tensor *k, const uint8_t *v_fp8,
+                                    const void *delta_s_bf16, const mpfa_stats *st, float v_scale, int causal,
+                                    float softmax_scale, void *out_bf16, float *out_f32, int32_t *device_status,
+                                    void *stream) {
+  if (!q || !k || !v_fp8 || !st || !out_bf16 || !device_status) return MPFA_ERR_INVALID_ARG;
+  if (!q->codes || !q->sf || !k->codes || !k->sf || !st->q_gscale || !st->k_gscale) return MPFA_ERR_INVALID_ARG;
+  if (q->B <= 0 || q->B != k->B || q->H <= 0 || k->H <= 0 || q->N <= 0 || k->N <= 0) return MPFA_ERR_INVALID_ARG;
+  if (!(softmax_scale > 0.0f) || !(v_scale > 0.0f)) return MPFA_ERR_INVALID_ARG;
+  if (q->H % k->H != 0 || q->H / k->H > 8) return MPFA_ERR_UNSUPPORTED;
+  if (!aligned(q->codes, 1024) || !aligned(k->codes, 1024) || !aligned(q->sf, 1024) || !aligned(k->sf, 1024) ||
+      !aligned(v_fp8, 1024) || !aligned(delta_s_bf16, 256) || !aligned(out_bf16, 16) || !aligned(out_f32, 16))
+    return MPFA_ERR_ALIGNMENT;
+  const int nq_tiles = pad128(q->N) / TILE, nk_tiles = pad128(k->N) / TILE;
+  const uint64_t q_rows = (uint64_t)q->B * q->H * nq_tiles * TILE, k_rows = (uint64_t)k->B * k->H * nk_tiles * TILE;
+  if (q_rows >= (1ull << 31) || k_rows >= (1ull << 31)) return MPFA_ERR_UNSUPPORTED;
+  const uint64_t n_cta = (uint64_t)q->B * q->H * nq_tiles;
+  if (n_cta >= (1ull << 31)) return MPFA_ERR_UNSUPPORTED;
+  mpfa_status rc = check_arch();
+  if (rc != MPFA_OK) return rc;
+  EncodeTiledFn enc;
+  rc = get_encoder(&enc);
+  if (rc != MPFA_OK) return rc;
+  CUtensorMap tq, tk, tv;
+  if ((rc = make_map(enc, &tq, q->codes, q_rows, 64)) != MPFA_OK) return rc;
+  if ((rc = make_map(enc, &tk, k->codes, k_rows, 64)) != MPFA_OK) return rc;
+  if ((rc = make_map(enc, &tv, v_fp8, k_rows, 128)) != MPFA_OK) return rc;
+  PrefillParams p;
+  p.q_sf = q->sf;
+  p.k_sf = k->sf;
+  p.delta = static_cast<const __nv_bfloat16 *>(delta_s_bf16);
+  p.q_gscale = st->q_gscale;
+  p.k_gscale = st->k_gscale;
+  p.out = static_cast<__nv_bfloat16 *>(out_bf16);
+  p.out_f32 = out_f32;
+  p.status = device_status;
+  p.B = q->B;
+  p.N_q = q->N;
+  p.N_kv = k->N;
+  p.H_q = q->H;
+  p.H_kv = k->H;
+  p.nq_tiles = nq_tiles;
+  p.nk_tiles = nk_tiles;
+  p.causal = causal ? 1 : 0;
+  p.softmax_scale = softmax_scale;
+  p.v_scale = v_scale;
+  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+  prefill_kernel<<<(unsigned)n_cta, NTHREADS, SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p);
+  MPFA_LAUNCH_OK();
+  return MPFA_OK;
+}

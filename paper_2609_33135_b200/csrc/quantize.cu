@@ -1,0 +1,503 @@
+// Stage 1 of the QK4PV8 path (Algorithm 1 lines 1-5): sequence means (Eq. 7), centering,
+// per-tensor scales, NVFP4 quantization (Eq. 1) of Q and K into the tile layout consumed
+// by the prefill kernel (or the fragment-ordered paged layout consumed by decode), the
+// compensation vector Delta_S (Eq. 9) and the FP8 quantization of V.
+//
+// Everything here is bandwidth work: 16-byte global loads, 8/16-byte stores, tiles staged in
+// shared memory where the destination order differs from the source order.  Every
+// floating-point step uses an explicitly rounded intrinsic so the results are defined to
+// the bit (no FMA contraction, IEEE division).
+#include <cuda_bf16.h>
+#include <cuda_fp4.h>
+#include <cuda_fp8.h>
+
+#include "common.cuh"
+
+namespace mpfa {
+
+thread_local int g_last_cuda_error = 0;
+
+mpfa_status check_arch() {
+  int dev = 0, major = 0;
+  MPFA_CUDA_OK(cudaGetDevice(&dev));
+  MPFA_CUDA_OK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  return major == 10 ? MPFA_OK : MPFA_ERR_ARCH;
+}
+
+namespace {
+
+constexpr int COLS_PER_BLOCK = 2048;  // 256 threads x 8 columns
+constexpr int TOK_PER_BLOCK = 128;
+
+__device__ __forceinline__ void unpack8(const uint4 &u, float (&f)[8]) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
+// Column sums in FP64.  For BF16 inputs whose nonzero magnitudes are >= 2^-14 every
+// partial sum of up to 2^17 tokens is exactly representable, so the atomic accumulation
+// order cannot change the result.
+__global__ void __launch_bounds__(256) colsum_kernel(const __nv_bfloat16 *__restrict__ x, int N, int cols,
+                                                     double *__restrict__ sums) {
+  const int b = blockIdx.z;
+  const int col = blockIdx.y * COLS_PER_BLOCK + threadIdx.x * 8;
+  if (col >= cols) return;
+  const int t0 = blockIdx.x * TOK_PER_BLOCK;
+  const int t1 = min(N, t0 + TOK_PER_BLOCK);
+  double acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  const __nv_bfloat16 *p = x + ((size_t)b * N + t0) * cols + col;
+  for (int t = t0; t < t1; ++t, p += cols) {
+    float f[8];
+    unpack8(*reinterpret_cast<const uint4 *>(p), f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] += (double)f[i];
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) atomicAdd(&sums[(size_t)b * cols + col + i], acc[i]);
+}
+
+__global__ void finalize_mean_kernel(const double *__restrict__ sums, int n, int N, float *__restrict__ mean) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) mean[i] = __double2float_rn(__ddiv_rn(sums[i], (double)N));
+}
+
+// max |x - mean| per batch element; non-negative floats order like their bit patterns.
+__global__ void __launch_bounds__(256) amax_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ mean,
+                                                   int N, int cols, unsigned int *__restrict__ amax) {
+  const int b = blockIdx.z;
+  const int col = blockIdx.y * COLS_PER_BLOCK + threadIdx.x * 8;
+  float m = 0.0f;
+  if (col < cols) {
+    float mu[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) mu[i] = mean[(size_t)b * cols + col + i];
+    const int t0 = blockIdx.x * TOK_PER_BLOCK;
+    const int t1 = min(N, t0 + TOK_PER_BLOCK);
+    const __nv_bfloat16 *p = x + ((size_t)b * N + t0) * cols + col;
+    for (int t = t0; t < t1; ++t, p += cols) {
+      float f[8];
+      unpack8(*reinterpret_cast<const uint4 *>(p), f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(__fsub_rn(f[i], mu[i])));
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  __shared__ float wmax[8];
+  if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int i = 1; i < 8; ++i) m = fmaxf(m, wmax[i]);
+    atomicMax(&amax[b], __float_as_uint(m));
+  }
+}
+
+__global__ void finalize_scale_kernel(const unsigned int *__restrict__ amax, int B, float *__restrict__ gscale) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < B) {
+    float a = __uint_as_float(amax[i]);
+    gscale[i] = a > 0.0f ? __fdiv_rn(a, 2688.0f) : 1.0f;
+  }
+}
+
+// One NVFP4 block (Eq. 1): 16 centered values -> E4M3 scale code + 8 bytes of E2M1 codes.
+__device__ __forceinline__ void quantize_block16(const float (&xc)[16], float d, uint8_t &scale_code, uint2 &codes) {
+  float a = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) a = fmaxf(a, fabsf(xc[i]));
+  const float e = __fmul_rn(6.0f, d);
+  const float r = __fdiv_rn(a, e);
+  scale_code = (uint8_t)__nv_cvt_float_to_fp8(r, __NV_SATFINITE, __NV_E4M3);
+  const float sdec = __half2float(__half(__nv_cvt_fp8_to_halfraw(scale_code, __NV_E4M3)));
+  const float s = __fmul_rn(sdec, d);
+  float inv = __fdiv_rn(1.0f, s);
+  if (!(s > 0.0f) || isinf(inv)) inv = 0.0f;
+  uint32_t w[2] = {0u, 0u};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float2 v = make_float2(__fmul_rn(xc[2 * i], inv), __fmul_rn(xc[2 * i + 1], inv));
+    uint32_t byte = (uint32_t)__nv_cvt_float2_to_fp4x2(v, __NV_E2M1, cudaRoundNearest);
+    w[i >> 2] |= (byte & 0xFFu) << (8 * (i & 3));
+  }
+  codes = make_uint2(w[0], w[1]);
+}
+
+__device__ __forceinline__ void load_center16(const __nv_bfloat16 *row, const float *mu, float (&xc)[16]) {
+  float f[8];
+  unpack8(reinterpret_cast<const uint4 *>(row)[0], f);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) xc[i] = __fsub_rn(f[i], mu[i]);
+  unpack8(reinterpret_cast<const uint4 *>(row)[1], f);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) xc[8 + i] = __fsub_rn(f[i], mu[8 + i]);
+}
+
+// grid (N_pad/128, H, B); one 128-token tile of one head per block.
+__global__ void __launch_bounds__(256) quantize_fp4_tile_kernel(const __nv_bfloat16 *__restrict__ x,
+                                                                const float *__restrict__ mean,
+                                                                const float *__restrict__ gscale, int N, int H,
+                                                                uint8_t *__restrict__ codes, uint8_t *__restrict__ sf) {
+  __shared__ float mu[HEAD_DIM];
+  __shared__ __align__(16) uint8_t sf_tile[1024];
+  const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int n_pad = gridDim.x * TILE;
+  if (threadIdx.x < HEAD_DIM) mu[threadIdx.x] = mean[((size_t)b * H + h) * HEAD_DIM + threadIdx.x];
+  __syncthreads();
+  const float d = gscale[b];
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int id = it * 256 + threadIdx.x;
+    const int r = id >> 3, g = id & 7;
+    const int t = tile * TILE + r;
+    uint2 c = make_uint2(0u, 0u);
+    uint8_t sc = 0;
+    if (t < N) {
+      float xc[16];
+      load_center16(x + (((size_t)b * N + t) * H + h) * HEAD_DIM + g * 16, mu + g * 16, xc);
+      quantize_block16(xc, d, sc, c);
+    }
+    *reinterpret_cast<uint2 *>(codes + (((size_t)b * H + h) * n_pad + t) * 64 + g * 8) = c;
+    sf_tile[(g >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (g & 3)] = sc;
+  }
+  __syncthreads();
+  uint32_t *dst = reinterpret_cast<uint32_t *>(sf + (((size_t)b * H + h) * gridDim.x + tile) * 1024);
+  dst[threadIdx.x] = reinterpret_cast<const uint32_t *>(sf_tile)[threadIdx.x];
+}
+
+// Eq. 9, one thread per key token: Delta_S[hq][t] = qmean[hq] . (k[t] - kmean), FP64
+// accumulation with channels ascending, expressed in units of gscale_q * gscale_k and
+// rounded once to BF16.  grid (N_pad/128, H_kv, B).  dst_stride / dst_base let the same
+// kernel write the dense [B, H_q, N_pad] vector or one page of the paged side cache.
+template <bool PAGED>
+__global__ void __launch_bounds__(128) delta_s_kernel(const __nv_bfloat16 *__restrict__ k,
+                                                      const float *__restrict__ q_mean,
+                                                      const float *__restrict__ k_mean,
+                                                      const float *__restrict__ q_gscale,
+                                                      const float *__restrict__ k_gscale, int N, int H_q, int H_kv,
+                                                      __nv_bfloat16 *__restrict__ delta,
+                                                      const int32_t *__restrict__ page_row, int num_pages) {
+  constexpr int MAXG = 8;
+  __shared__ float kmu[HEAD_DIM];
+  __shared__ float qmu[MAXG][HEAD_DIM];
+  const int tile = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+  const int G = H_q / H_kv;
+  const int n_pad = gridDim.x * TILE;
+  kmu[threadIdx.x] = k_mean[((size_t)b * H_kv + hk) * HEAD_DIM + threadIdx.x];
+  for (int g = 0; g < G; ++g) qmu[g][threadIdx.x] = q_mean[((size_t)b * H_q + hk * G + g) * HEAD_DIM + threadIdx.x];
+  __syncthreads();
+  const int t = tile * TILE + threadIdx.x;
+  double acc[MAXG];
+#pragma unroll
+  for (int g = 0; g < MAXG; ++g) acc[g] = 0.0;
+  if (t < N) {
+    const __nv_bfloat16 *row = k + (((size_t)b * N + t) * H_kv + hk) * HEAD_DIM;
+    for (int c0 = 0; c0 < HEAD_DIM; c0 += 8) {
+      float f[8];
+      unpack8(*reinterpret_cast<const uint4 *>(row + c0), f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const double kc = (double)__fsub_rn(f[i], kmu[c0 + i]);
+#pragma unroll
+        for (int g = 0; g < MAXG; ++g)
+          if (g < G) acc[g] = fma((double)qmu[g][c0 + i], kc, acc[g]);
+      }
+    }
+  }
+  const double denom = (double)q_gscale[b] * (double)k_gscale[b];
+#pragma unroll
+  for (int g = 0; g < MAXG; ++g) {
+    if (g < G) {
+      const float v = (t < N) ? __double2float_rn(__ddiv_rn(acc[g], denom)) : 0.0f;
+      if (PAGED) {
+        if ((t >> 6) < (N + PAGE - 1) / PAGE) {   // slots past N inside the last page are zero-filled
+          const int page = page_row[t >> 6];
+          if (page >= 0 && page < num_pages)
+            delta[((size_t)page * H_q + hk * G + g) * PAGE + (t & 63)] = __float2bfloat16_rn(v);
+        }
+      } else {
+        delta[((size_t)b * H_q + hk * G + g) * n_pad + t] = __float2bfloat16_rn(v);
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ uint4 quantize_v16(const __nv_bfloat16 *row, float inv) {
+  float f[16];
+  {
+    float t8[8];
+    unpack8(reinterpret_cast<const uint4 *>(row)[0], t8);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f[i] = t8[i];
+    unpack8(reinterpret_cast<const uint4 *>(row)[1], t8);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f[8 + i] = t8[i];
+  }
+  uint32_t w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(
+        make_float2(__fmul_rn(f[4 * i], inv), __fmul_rn(f[4 * i + 1], inv)), __NV_SATFINITE, __NV_E4M3);
+    uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(
+        make_float2(__fmul_rn(f[4 * i + 2], inv), __fmul_rn(f[4 * i + 3], inv)), __NV_SATFINITE, __NV_E4M3);
+    w[i] = (lo & 0xFFFFu) | (hi << 16);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// grid (N_pad/128, H, B): V tile -> [B, H, N_pad, 128] E4M3.
+__global__ void __launch_bounds__(256) quantize_v_tile_kernel(const __nv_bfloat16 *__restrict__ v, int N, int H,
+                                                              float inv_scale, uint8_t *__restrict__ out) {
+  const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int n_pad = gridDim.x * TILE;
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int id = it * 256 + threadIdx.x;
+    const int r = id >> 3, seg = id & 7;
+    const int t = tile * TILE + r;
+    uint4 c = make_uint4(0u, 0u, 0u, 0u);
+    if (t < N) c = quantize_v16(v + (((size_t)b * N + t) * H + h) * HEAD_DIM + seg * 16, inv_scale);
+    *reinterpret_cast<uint4 *>(out + (((size_t)b * H + h) * n_pad + t) * HEAD_DIM + seg * 16) = c;
+  }
+}
+
+// Paged cache write for one request: grid (pages, H_kv).  K and V of one (page, head) are
+// quantized into shared memory in the decode kernel's fragment order and copied out with
+// 16-byte stores.
+__global__ void __launch_bounds__(256) quantize_kv_page_kernel(const __nv_bfloat16 *__restrict__ k,
+                                                               const __nv_bfloat16 *__restrict__ v,
+                                                               const float *__restrict__ k_mean,
+                                                               const float *__restrict__ k_gscale, int N, int H_kv,
+                                                               float inv_vscale, const int32_t *__restrict__ page_row,
+                                                               int first_page, int num_pages,
+                                                               uint8_t *__restrict__ k_codes, uint8_t *__restrict__ k_sf,
+                                                               uint8_t *__restrict__ v_fp8) {
+  __shared__ float mu[HEAD_DIM];
+  __shared__ __align__(16) uint8_t sk[4096];
+  __shared__ __align__(16) uint8_t ssf[512];
+  __shared__ __align__(16) uint8_t sv[8192];
+  const int lp = blockIdx.x, h = blockIdx.y;
+  const int page = page_row[first_page + lp];
+  if (page < 0 || page >= num_pages) return;  // the host validates the shape; a bad id is skipped
+  if (threadIdx.x < HEAD_DIM) mu[threadIdx.x] = k_mean[(size_t)h * HEAD_DIM + threadIdx.x];
+  __syncthreads();
+  const float d = k_gscale[0];
+#pragma unroll
+  for (int it = 0; it < 2; ++it) {
+    const int id = it * 256 + threadIdx.x;
+    const int t = id >> 3, g = id & 7;   // token in page, 16-channel block / segment
+    const int tok = lp * PAGE + t;
+    uint2 c = make_uint2(0u, 0u);
+    uint8_t sc = 0;
+    uint4 vc = make_uint4(0u, 0u, 0u, 0u);
+    if (tok < N) {
+      float xc[16];
+      load_center16(k + ((size_t)tok * H_kv + h) * HEAD_DIM + g * 16, mu + g * 16, xc);
+      quantize_block16(xc, d, sc, c);
+      vc = quantize_v16(v + ((size_t)tok * H_kv + h) * HEAD_DIM + g * 16, inv_vscale);
+    }
+    // K: byte j of block g of token t at (t/8)*512 + ((t%8)*4 + j/2)*16 + g*2 + (j%2)
+    const uint32_t cw[2] = {c.x, c.y};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint16_t two = (uint16_t)(cw[q >> 1] >> (16 * (q & 1)));
+      *reinterpret_cast<uint16_t *>(sk + (t >> 3) * 512 + ((t & 7) * 4 + q) * 16 + g * 2) = two;
+    }
+    ssf[t * 8 + g] = sc;
+    // V: channel c of token t (u = t%32) at
+    // (t/32)*4096 + (c/16)*512 + ((c%8)*4 + (u%8)/2)*16 + ((c/8)%2)*8 + (u/16)*4 + ((u/8)%2)*2 + (u%2)
+    const uint32_t vw[4] = {vc.x, vc.y, vc.z, vc.w};
+    const int u = t & 31;
+    const int tbase = (t >> 5) * 4096 + g * 512 + ((u & 7) >> 1) * 16 + (u >> 4) * 4 + ((u >> 3) & 1) * 2 + (u & 1);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int ch = i;  // channel inside the 16-channel segment g
+      sv[tbase + (ch & 7) * 64 + (ch >> 3) * 8] = (uint8_t)(vw[i >> 2] >> (8 * (i & 3)));
+    }
+  }
+  __syncthreads();
+  const size_t slab = (size_t)page * H_kv + h;
+  reinterpret_cast<uint4 *>(k_codes + slab * 4096)[threadIdx.x] = reinterpret_cast<const uint4 *>(sk)[threadIdx.x];
+  if (threadIdx.x < 32) reinterpret_cast<uint4 *>(k_sf + slab * 512)[threadIdx.x] = reinterpret_cast<const uint4 *>(ssf)[threadIdx.x];
+  reinterpret_cast<uint4 *>(v_fp8 + slab * 8192)[threadIdx.x] = reinterpret_cast<const uint4 *>(sv)[threadIdx.x];
+  reinterpret_cast<uint4 *>(v_fp8 + slab * 8192)[threadIdx.x + 256] = reinterpret_cast<const uint4 *>(sv)[threadIdx.x + 256];
+}
+
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+struct StatsWorkspace {
+  double *sums_q, *sums_k;
+  unsigned int *amax_q, *amax_k;
+  size_t bytes;
+};
+
+StatsWorkspace carve(void *ws, int B, int H_q, int H_kv) {
+  StatsWorkspace w;
+  size_t o = 0;
+  uint8_t *base = static_cast<uint8_t *>(ws);
+  w.sums_q = reinterpret_cast<double *>(base + o);
+  o += align256((size_t)B * H_q * HEAD_DIM * sizeof(double));
+  w.sums_k = reinterpret_cast<double *>(base + o);
+  o += align256((size_t)B * H_kv * HEAD_DIM * sizeof(double));
+  w.amax_q = reinterpret_cast<unsigned int *>(base + o);
+  o += align256((size_t)B * sizeof(unsigned int));
+  w.amax_k = reinterpret_cast<unsigned int *>(base + o);
+  o += align256((size_t)B * sizeof(unsigned int));
+  w.bytes = o;
+  return w;
+}
+
+// Means and per-tensor scale of one tensor [B, N, H, 128].
+mpfa_status tensor_stats(const __nv_bfloat16 *x, int B, int N, int H, bool smooth, double *sums, unsigned int *amax,
+                         float *mean, float *gscale, cudaStream_t st) {
+  const int cols = H * HEAD_DIM;
+  dim3 grid((N + TOK_PER_BLOCK - 1) / TOK_PER_BLOCK, (cols + COLS_PER_BLOCK - 1) / COLS_PER_BLOCK, B);
+  if (smooth) {
+    colsum_kernel<<<grid, 256, 0, st>>>(x, N, cols, sums);
+    MPFA_LAUNCH_OK();
+    finalize_mean_kernel<<<(B * cols + 255) / 256, 256, 0, st>>>(sums, B * cols, N, mean);
+    MPFA_LAUNCH_OK();
+  } else {
+    MPFA_CUDA_OK(cudaMemsetAsync(mean, 0, (size_t)B * cols * sizeof(float), st));
+  }
+  amax_kernel<<<grid, 256, 0, st>>>(x, mean, N, cols, amax);
+  MPFA_LAUNCH_OK();
+  finalize_scale_kernel<<<(B + 127) / 128, 128, 0, st>>>(amax, B, gscale);
+  MPFA_LAUNCH_OK();
+  return MPFA_OK;
+}
+
+}  // namespace
+}  // namespace mpfa
+
+using namespace mpfa;
+
+extern "C" size_t mpfa_quantize_workspace_bytes(int B, int H_q, int H_kv) {
+  if (B <= 0 || H_q <= 0 || H_kv <= 0) return 0;
+  return carve(nullptr, B, H_q, H_kv).bytes;
+}
+
+extern "C" mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, int B, int N_q, int N_kv, int H_q,
+                                        int H_kv, int flags, mpfa_stats *st, mpfa_fp4_tensor *q_out,
+                                        mpfa_fp4_tensor *k_out, void *delta_s_bf16, void *workspace,
+                                        size_t workspace_bytes, void *stream) {
+  const bool smooth = flags & MPFA_SMOOTH, frozen = flags & MPFA_STATS_FROZEN;
+  if (!st || (!q_bf16 && !k_bf16) || B <= 0 || H_q <= 0 || H_kv <= 0) return MPFA_ERR_INVALID_ARG;
+  if ((q_bf16 && (N_q <= 0 || !q_out)) || (k_bf16 && (N_kv <= 0 || !k_out))) return MPFA_ERR_INVALID_ARG;
+  if (!st->q_mean || !st->k_mean || !st->q_gscale || !st->k_gscale) return MPFA_ERR_INVALID_ARG;
+  if (H_q % H_kv != 0 || H_q / H_kv > 8) return MPFA_ERR_UNSUPPORTED;
+  if (N_q > (1 << 24) || N_kv > (1 << 24)) return MPFA_ERR_UNSUPPORTED;
+  if (smooth && k_bf16 && !delta_s_bf16) return MPFA_ERR_INVALID_ARG;
+  if (smooth && !q_bf16 && !frozen) return MPFA_ERR_INVALID_ARG;  // Delta_S needs the query mean
+  if (q_bf16 && (q_out->B != B || q_out->H != H_q || q_out->N != N_q || !q_out->codes || !q_out->sf))
+    return MPFA_ERR_INVALID_ARG;
+  if (k_bf16 && (k_out->B != B || k_out->H != H_kv || k_out->N != N_kv || !k_out->codes || !k_out->sf))
+    return MPFA_ERR_INVALID_ARG;
+  if (!aligned(q_bf16, 16) || !aligned(k_bf16, 16) || !aligned(delta_s_bf16, 256)) return MPFA_ERR_ALIGNMENT;
+  if (q_bf16 && (!aligned(q_out->codes, 1024) || !aligned(q_out->sf, 1024))) return MPFA_ERR_ALIGNMENT;
+  if (k_bf16 && (!aligned(k_out->codes, 1024) || !aligned(k_out->sf, 1024))) return MPFA_ERR_ALIGNMENT;
+  StatsWorkspace w{};
+  if (!frozen) {
+    if (!workspace) return MPFA_ERR_INVALID_ARG;
+    if (!aligned(workspace, 256)) return MPFA_ERR_ALIGNMENT;
+    w = carve(workspace, B, H_q, H_kv);
+    if (workspace_bytes < w.bytes) return MPFA_ERR_WORKSPACE;
+  }
+  mpfa_status rc = check_arch();
+  if (rc != MPFA_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(q_bf16);
+  const __nv_bfloat16 *k = static_cast<const __nv_bfloat16 *>(k_bf16);
+  if (!frozen) {
+    MPFA_CUDA_OK(cudaMemsetAsync(workspace, 0, w.bytes, s));
+    if (q) {
+      rc = tensor_stats(q, B, N_q, H_q, smooth, w.sums_q, w.amax_q, st->q_mean, st->q_gscale, s);
+      if (rc != MPFA_OK) return rc;
+    }
+    if (k) {
+      rc = tensor_stats(k, B, N_kv, H_kv, smooth, w.sums_k, w.amax_k, st->k_mean, st->k_gscale, s);
+      if (rc != MPFA_OK) return rc;
+    }
+  }
+  if (q) {
+    dim3 grid(pad128(N_q) / TILE, H_q, B);
+    quantize_fp4_tile_kernel<<<grid, 256, 0, s>>>(q, st->q_mean, st->q_gscale, N_q, H_q, q_out->codes, q_out->sf);
+    MPFA_LAUNCH_OK();
+  }
+  if (k) {
+    dim3 grid(pad128(N_kv) / TILE, H_kv, B);
+    quantize_fp4_tile_kernel<<<grid, 256, 0, s>>>(k, st->k_mean, st->k_gscale, N_kv, H_kv, k_out->codes, k_out->sf);
+    MPFA_LAUNCH_OK();
+    if (smooth) {
+      delta_s_kernel<false><<<grid, 128, 0, s>>>(k, st->q_mean, st->k_mean, st->q_gscale, st->k_gscale, N_kv, H_q,
+                                                 H_kv, static_cast<__nv_bfloat16 *>(delta_s_bf16), nullptr, 0);
+      MPFA_LAUNCH_OK();
+    }
+  }
+  return MPFA_OK;
+}
+
+extern "C" mpfa_status mpfa_quantize_v(const void *v_bf16, int B, int N_kv, int H_kv, float v_scale, uint8_t *v_fp8,
+                                       void *stream) {
+  if (!v_bf16 || !v_fp8 || B <= 0 || N_kv <= 0 || H_kv <= 0 || !(v_scale > 0.0f)) return MPFA_ERR_INVALID_ARG;
+  if (!aligned(v_bf16, 16) || !aligned(v_fp8, 1024)) return MPFA_ERR_ALIGNMENT;
+  mpfa_status rc = check_arch();
+  if (rc != MPFA_OK) return rc;
+  dim3 grid(pad128(N_kv) / TILE, H_kv, B);
+  quantize_v_tile_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16 *>(v_bf16), N_kv, H_kv, 1.0f / v_scale, v_fp8);
+  MPFA_LAUNCH_OK();
+  return MPFA_OK;
+}
+
+extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_bf16, int N_tokens, int first_token,
+                                              int H_q, int H_kv, int flags, mpfa_stats *st, float v_scale,
+                                              const mpfa_paged_kv *kv, const int32_t *page_table_row,
+                                              void *workspace, size_t workspace_bytes, void *stream) {
+  const bool smooth = flags & MPFA_SMOOTH, frozen = flags & MPFA_STATS_FROZEN;
+  if (!k_bf16 || !v_bf16 || !st || !kv || !page_table_row || N_tokens <= 0 || first_token < 0 || H_q <= 0 ||
+      H_kv <= 0 || !(v_scale > 0.0f))
+    return MPFA_ERR_INVALID_ARG;
+  if (!st->q_mean || !st->k_mean || !st->q_gscale || !st->k_gscale) return MPFA_ERR_INVALID_ARG;
+  if (!kv->k_codes || !kv->k_sf || !kv->v_fp8 || kv->num_pages <= 0) return MPFA_ERR_INVALID_ARG;
+  if (smooth && !kv->delta_s_bf16) return MPFA_ERR_INVALID_ARG;
+  if (kv->page_size != PAGE || H_q % H_kv != 0 || H_q / H_kv > 8) return MPFA_ERR_UNSUPPORTED;
+  if (first_token % PAGE != 0) return MPFA_ERR_UNSUPPORTED;  // appends inside a partly filled page: not built yet
+  if (!frozen && first_token != 0) return MPFA_ERR_INVALID_ARG;
+  if (!aligned(k_bf16, 16) || !aligned(v_bf16, 16) || !aligned(kv->k_codes, 256) || !aligned(kv->k_sf, 256) ||
+      !aligned(kv->v_fp8, 256) || !aligned(kv->delta_s_bf16, 256))
+    return MPFA_ERR_ALIGNMENT;
+  StatsWorkspace w{};
+  if (!frozen) {
+    if (!workspace) return MPFA_ERR_INVALID_ARG;
+    if (!aligned(workspace, 256)) return MPFA_ERR_ALIGNMENT;
+    w = carve(workspace, 1, H_q, H_kv);
+    if (workspace_bytes < w.bytes) return MPFA_ERR_WORKSPACE;
+  }
+  mpfa_status rc = check_arch();
+  if (rc != MPFA_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const __nv_bfloat16 *k = static_cast<const __nv_bfloat16 *>(k_bf16);
+  const __nv_bfloat16 *v = static_cast<const __nv_bfloat16 *>(v_bf16);
+  if (!frozen) {
+    MPFA_CUDA_OK(cudaMemsetAsync(workspace, 0, w.bytes, s));
+    rc = tensor_stats(k, 1, N_tokens, H_kv, smooth, w.sums_k, w.amax_k, st->k_mean, st->k_gscale, s);
+    if (rc != MPFA_OK) return rc;
+  }
+  const int n_pages = (N_tokens + PAGE - 1) / PAGE;
+  quantize_kv_page_kernel<<<dim3(n_pages, H_kv), 256, 0, s>>>(k, v, st->k_mean, st->k_gscale, N_tokens, H_kv,
+                                                              1.0f / v_scale, page_table_row, first_token / PAGE,
+                                                              kv->num_pages, kv->k_codes, kv->k_sf, kv->v_fp8);
+  MPFA_LAUNCH_OK();
+  if (smooth) {
+    delta_s_kernel<true><<<dim3(pad128(N_tokens) / TILE, H_kv, 1), 128, 0, s>>>(
+        k, st->q_mean, st->k_mean, st->q_gscale, st->k_gscale, N_tokens, H_q, H_kv,
+        static_cast<__nv_bfloat16 *>(kv->delta_s_bf16), page_table_row + first_token / PAGE, kv->num_pages);
+    MPFA_LAUNCH_OK();
+  }
+  return MPFA_OK;
+}

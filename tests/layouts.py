@@ -1,0 +1,48 @@
+"""Index maps between the library's physical layouts and plain row-major arrays, written
+from the layout description in include/mpfa.h (test helper; numpy only)."""
+import numpy as np
+
+
+def pad128(n):
+    return (n + 127) // 128 * 128
+
+
+def codes_to_logical(codes: np.ndarray, B, H, N) -> np.ndarray:
+    """tile-layout codes (flat uint8) -> [B,H,N,64]; also returns the pad rows for a zero check."""
+    a = codes.reshape(B, H, pad128(N), 64)
+    return a[:, :, :N, :], a[:, :, N:, :]
+
+
+def sf_to_logical(sf: np.ndarray, B, H, N) -> np.ndarray:
+    """tile-layout scale factors (flat uint8) -> [B,H,N_pad,8]."""
+    tiles = pad128(N) // 128
+    a = sf.reshape(B, H, tiles, 2, 512)
+    r = np.arange(128)
+    g = np.arange(8)
+    off = (r[:, None] % 32) * 16 + (r[:, None] // 32) * 4 + (g[None, :] % 4)     # [128, 8]
+    half = np.broadcast_to(g[None, :] // 4, (128, 8))
+    out = a[:, :, :, half, off]                                                   # [B,H,tiles,128,8]
+    return out.reshape(B, H, tiles * 128, 8)
+
+
+def paged_k_offset(t, g, j):
+    return (t // 8) * 512 + ((t % 8) * 4 + j // 2) * 16 + g * 2 + (j % 2)
+
+
+def paged_v_offset(t, c):
+    u = t % 32
+    return ((t // 32) * 4096 + (c // 16) * 512 + ((c % 8) * 4 + (u % 8) // 2) * 16 + ((c // 8) % 2) * 8 +
+            (u // 16) * 4 + ((u // 8) % 2) * 2 + (u % 2))
+
+
+def paged_k_to_logical(slab: np.ndarray) -> np.ndarray:
+    """[..., 4096] page slab -> [..., 64 tokens, 64 bytes]."""
+    t, g, j = np.meshgrid(np.arange(64), np.arange(8), np.arange(8), indexing="ij")
+    off = paged_k_offset(t, g, j).reshape(64, 64)
+    return slab[..., off]
+
+
+def paged_v_to_logical(slab: np.ndarray) -> np.ndarray:
+    """[..., 8192] page slab -> [..., 64 tokens, 128 channels]."""
+    t, c = np.meshgrid(np.arange(64), np.arange(128), indexing="ij")
+    return slab[..., paged_v_offset(t, c)]

@@ -1,0 +1,103 @@
+"""GPU parity: stage-1 kernels against the oracle, bit for bit (codes, block scales, tensor
+scales, means, compensation vector, V codes), through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mpfa_oracle as orc
+from paper_2609_33135_b200 import workloads as wl
+
+from layouts import codes_to_logical, pad128, sf_to_logical
+
+pytestmark = pytest.mark.gpu
+
+
+def _cases():
+    return {
+        "cfg1": lambda: wl.config1_tiny(),
+        "cfg1b": lambda: wl.config1b_tiny_qbias(),
+        "ragged_gqa": lambda: wl.prefill_workload("ragged", 41, 2, 333, 4, 2, True, N_q=300, q_bias=True),
+        "gqa5_2k": lambda: wl.prefill_workload("gqa5", 42, 1, 2048 + 77, 10, 2, True, q_bias=True),
+    }
+
+
+def run_stage1_gpu(w, smooth=True, v_scale=1.0):
+    from paper_2609_33135_b200 import binding
+    return binding.stage1(w.q.cuda(), w.k.cuda(), w.v.cuda(), smooth=smooth, v_scale=v_scale)
+
+
+def check_stage1(w, s1, z, smooth=True):
+    B, Nq, Hq, Nkv, Hkv = w.B, w.N_q, w.H_q, w.N_kv, w.H_kv
+    torch.cuda.synchronize()
+    assert np.array_equal(s1.stats.q_mean.cpu().numpy(), z.q_mean)
+    assert np.array_equal(s1.stats.k_mean.cpu().numpy(), z.k_mean)
+    assert np.array_equal(s1.stats.q_gscale.cpu().numpy(), z.dq)
+    assert np.array_equal(s1.stats.k_gscale.cpu().numpy(), z.dk)
+    for t, codes, sf, H, N in ((s1.q, z.q_codes, z.q_sf, Hq, Nq), (s1.k, z.k_codes, z.k_sf, Hkv, Nkv)):
+        got, padrows = codes_to_logical(t.codes.cpu().numpy(), B, H, N)
+        assert np.array_equal(got, codes)
+        assert not padrows.any()
+        gsf = sf_to_logical(t.sf.cpu().numpy(), B, H, N)
+        assert np.array_equal(gsf[:, :, :N], sf)
+        assert not gsf[:, :, N:].any()
+    gv = s1.v_fp8.cpu().numpy().reshape(B, Hkv, pad128(Nkv), 128)
+    assert np.array_equal(gv[:, :, :Nkv], z.v_codes)
+    assert not gv[:, :, Nkv:].any()
+    if smooth:
+        gd = s1.delta.view(torch.uint16).cpu().numpy()
+        assert np.array_equal(gd[:, :, :Nkv], z.delta)
+        assert not gd[:, :, Nkv:].any()
+    else:
+        assert s1.delta is None
+
+
+@pytest.mark.parametrize("name", list(_cases()))
+def test_stage1_bit_exact(name):
+    w = _cases()[name]()
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+    check_stage1(w, run_stage1_gpu(w), z)
+
+
+def test_stage1_direct_variant_and_v_scale():
+    w = _cases()["ragged_gqa"]()
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v), smooth=False, v_scale=0.5)
+    s1 = run_stage1_gpu(w, smooth=False, v_scale=0.5)
+    check_stage1(w, s1, z, smooth=False)
+    assert not s1.stats.q_mean.any() and not s1.stats.k_mean.any()
+
+
+def test_frozen_statistics_single_token_query():
+    """Decode-time query: one token centered and scaled with the frozen prefill statistics."""
+    from paper_2609_33135_b200 import binding
+    w = _cases()["ragged_gqa"]()
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+    s1 = run_stage1_gpu(w)
+    qn = w.q[:, 17:18].contiguous()
+    zq = orc.stage1(orc.bf16_bits(qn), orc.bf16_bits(w.k), orc.bf16_bits(w.v), frozen=z)
+    q4 = binding.Fp4Tensor.empty(w.B, w.H_q, 1)
+    binding.mpfa_quantize_qk(qn.cuda(), None, binding.MPFA_SMOOTH | binding.MPFA_STATS_FROZEN, s1.stats, q4, None,
+                             None, None)
+    torch.cuda.synchronize()
+    got, pad = codes_to_logical(q4.codes.cpu().numpy(), w.B, w.H_q, 1)
+    assert np.array_equal(got, zq.q_codes) and not pad.any()
+    assert np.array_equal(sf_to_logical(q4.sf.cpu().numpy(), w.B, w.H_q, 1)[:, :, :1], zq.q_sf)
+
+
+def test_deterministic_and_argument_errors():
+    from paper_2609_33135_b200 import binding
+    w = _cases()["cfg1b"]()
+    a = run_stage1_gpu(w)
+    b = run_stage1_gpu(w)
+    torch.cuda.synchronize()
+    assert torch.equal(a.q.codes, b.q.codes) and torch.equal(a.k.sf, b.k.sf) and torch.equal(a.delta, b.delta)
+    q = w.q.cuda()
+    st = binding.Stats.empty(1, 1, 1)
+    q4 = binding.Fp4Tensor.empty(1, 1, 256)
+    ws = binding.quantize_workspace(1, 1, 1)
+    with pytest.raises(binding.MpfaError, match="workspace"):
+        binding.mpfa_quantize_qk(q, None, 0, st, q4, None, None, ws[:256])
+    with pytest.raises(binding.MpfaError, match="misaligned"):
+        bad = binding.Fp4Tensor(q4.codes[16:], q4.sf, 1, 1, 255)
+        binding.mpfa_quantize_qk(q[:, :255].contiguous(), None, 0, st, bad, None, None, ws)
+    with pytest.raises(binding.MpfaError, match="invalid"):
+        binding.mpfa_quantize_qk(q, None, 0, st, binding.Fp4Tensor(q4.codes, q4.sf, 1, 1, 128), None, None, ws)
