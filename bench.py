@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the QK4PV8 hot path on B200.
+
+A step is one pass of the whole path over one batch of the Llama-3.1-8B-shaped causal
+prefill workload (batch 1, 32 q heads / 8 kv heads, head_dim 128, 16384 tokens): stage 1
+(means, scales, NVFP4 quantization of Q and K, Delta_S, FP8 V) followed by the prefill
+attention kernel.  `value` is attention TFLOPS (4 N^2 d H_q / 2 per step) over the whole
+step with inputs resident in HBM; `e2e` is the same with pinned-host inputs copied in and
+the BF16 output copied back inside the timed region.  The paged decode workload is timed
+separately in the same run and reported under "decode" in GB/s of KV-cache bytes.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same workload on its own
+batch element: the path shards by (batch, head) with no data-path collective, so scaling is
+weak and `value` is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "QK4PV8 prefill TFLOPS @16K-128K; decode KV GB/s vs HBM peak"
+KERNELS_PER_STEP = 13  # colsum, mean, amax, scale (x2 tensors), fp4 quantize x2, Delta_S, V quantize, prefill
+# Nominal dense tensor rates relative to BF16: FP4 4x, FP8 2x.  Per (query, key) pair the path does
+# 2d FP4 FLOP and 2d FP8 FLOP, so F attention FLOPs take (F/2)/(4P) + (F/2)/(2P) = 3F/(8P): the
+# mixed-precision bound in attention FLOP/s is 8/3 of the BF16 peak P.
+MIXED_OVER_BF16 = 8.0 / 3.0
+KV_BYTES_PER_TOKEN_HEAD = 64 + 8 + 128 + 2 * 4  # K codes, K scales, V, Delta_S for a 4-head GQA group
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16": p["bf16_tflops"], "bf16_sustained": p["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        for ts, line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            mx = float(parts[2])
+            if t0 - 0.05 <= ts <= t1 + 0.15:
+                sm.append(float(parts[1]))
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        if not sm:
+            sm = [float(l.split(",")[1]) for _, l in self.lines[-3:] if len(l.split(",")) >= 9]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_setup(n):
+    if n <= 1:
+        return 0, 1, 0
+    import torch.distributed as dist
+    rank, world, local = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"]), int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(x: float, world) -> float:
+    if world <= 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ------------------------------------------------------------------------------------------
+def cpu_oracle_sample(w, steps: int, rows_per_head: int):
+    """The oracle, as it stands, on a bounded sample of the prefill workload: stage 1 on the full
+    tensors once, then `rows_per_head` evenly spaced query rows of every head against all their keys."""
+    from oracle import mpfa_oracle as orc
+    import numpy as np
+    q, k, v = orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v)
+    stride = max(1, w.N_q // rows_per_head)
+    idx = np.arange(stride - 1, w.N_q, stride, dtype=np.int32)
+    rows = np.stack([np.zeros(len(idx) * w.H_q, np.int32), np.repeat(np.arange(w.H_q, dtype=np.int32), len(idx)),
+                     np.tile(idx, w.H_q)], axis=1)
+    pairs = float((idx.astype(np.int64) + 1 + (w.N_kv - w.N_q)).clip(0, w.N_kv).sum() * w.H_q)
+    times = []
+    z = None
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        z = orc.stage1(q, k, v)
+        orc.prefill_rows(z, rows, w.softmax_scale, w.causal)
+        times.append(time.perf_counter() - t0)
+    return pairs * 4 * 128, times, f"stage 1 on the full tensors + {len(rows)} (head, query row) pairs " \
+                                  f"(every {stride}th row of each head) against all their keys"
+
+
+def run_reference(args, rank):
+    """Reference arm: the CPU oracle on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    from paper_2609_33135_b200 import workloads as wl
+    w = wl.config2_llama()
+    cores = os.cpu_count() or 1
+    flops, times, sample = cpu_oracle_sample(w, args.warmup + args.steps, rows_per_head=256)
+    times = times[args.warmup:]
+    ms = 1e3 * sum(times) / len(times)
+    val = flops / (ms * 1e-3) / 1e12
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "nvfp4/fp8 emulated in f32", "data": "synthetic",
+        "config": {"workload": w.name, "B": 1, "H_q": 32, "H_kv": 8, "head_dim": 128, "N": w.N_q, "causal": True},
+        "cpu_baseline": {"value": val, "unit": "TFLOPS", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ------------------------------------------------------------------------------------------
+def bench_decode(binding, wl, steps, warmup, peaks, small):
+    """Paged decode (config 5): KV GB/s = sum_r L_r * H_kv * 208 B / time."""
+    if not hasattr(binding, "build_decode_cache"):
+        return None
+    B = 32
+    lo, hi = (2048, 8192) if small else (16384, 131072)
+    w = wl.config5_decode(B, lo, hi)
+    state = binding.build_decode_cache(w, synthetic_fill=True)
+    run = lambda: binding.decode_step(state)
+    for _ in range(warmup):
+        run()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        a.record()
+        run()
+        b.record()
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in evs]
+    bytes_ = float(w.total_tokens) * w.H_kv * KV_BYTES_PER_TOKEN_HEAD
+    mean = sum(ms) / len(ms)
+    gbs = bytes_ / (mean * 1e-3) / 1e9
+    return {"workload": w.name, "value": gbs, "unit": "GB/s", "ms_mean": mean, "ms_min": min(ms),
+            "kv_bytes": bytes_, "tokens": w.total_tokens, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+            "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
+            "status": int(state["status"].item())}
+
+
+def run_ours(args, rank, world, local):
+    from paper_2609_33135_b200 import binding, workloads as wl
+    binding.lib()  # fail loudly if the CUDA library is missing
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the QK4PV8 path has no CPU fallback")
+    peaks = load_peaks()
+    dev = torch.device("cuda", local)
+    N = args.seq_len
+    w = wl.config2_llama(N)
+    hq, hk, hv = w.q.pin_memory(), w.k.pin_memory(), w.v.pin_memory()
+    q, k, v = hq.to(dev), hk.to(dev), hv.to(dev)
+    s1 = binding.stage1(q, k, v)           # allocates outputs once; steps reuse them
+    ws = binding.quantize_workspace(w.B, w.H_q, w.H_kv, dev)
+    out = torch.empty(w.B, w.N_q, w.H_q, 128, dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    host_out = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def step(kernel_events=None):
+        binding.stage1(q, k, v, workspace=ws, out=s1)
+        if kernel_events is not None:
+            kernel_events[0].record()
+        binding.prefill(s1, w.causal, w.softmax_scale, out=out, status=status)
+        if kernel_events is not None:
+            kernel_events[1].record()
+
+    def step_e2e():
+        q.copy_(hq, non_blocking=True)
+        k.copy_(hk, non_blocking=True)
+        v.copy_(hv, non_blocking=True)
+        step()
+        host_out.copy_(out, non_blocking=True)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+
+    # ---- timed region: K steps, device-timed, barrier + synchronize on both sides
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    kev = [(ev(), ev()) for _ in range(args.steps)]
+    barrier(world)
+    e0, e1 = ev(), ev()
+    t_wall0 = time.time()
+    e0.record()
+    for i in range(args.steps):
+        step(kev[i])
+    e1.record()
+    barrier(world)
+    t_wall1 = time.time()
+    total_ms = max_over_ranks(e0.elapsed_time(e1), world)
+    clocks = sampler.stop(t_wall0, t_wall1)
+    ms_step = total_ms / args.steps
+    kernel_ms = sum(a.elapsed_time(b) for a, b in kev) / args.steps
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+
+    # ---- end to end: pinned host inputs in, BF16 output back, every step
+    for _ in range(2):
+        step_e2e()
+    barrier(world)
+    e0, e1 = ev(), ev()
+    e0.record()
+    for _ in range(args.steps):
+        step_e2e()
+    e1.record()
+    barrier(world)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world) / args.steps
+    _ = float(host_out[0, 0, 0, 0])  # the host reads the result
+
+    flops = w.flops
+    value = world * flops / (ms_step * 1e-3) / 1e12
+    long_run = total_ms > 2000.0
+    bf16_peak = peaks["bf16_sustained"] if long_run else peaks["bf16"]
+    peak = bf16_peak * MIXED_OVER_BF16
+    achieved = flops / (kernel_ms * 1e-3) / 1e12
+    result = {
+        "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "nvfp4 (QK^T) + fp8 e4m3 (PV), f32 accumulate", "data": "synthetic",
+        "config": {"workload": w.name, "B_per_gpu": 1, "H_q": w.H_q, "H_kv": w.H_kv, "head_dim": 128, "N": N,
+                   "causal": True, "parallelism": f"dp{world} (independent batch elements, no collective)",
+                   "l2": "inputs_exceed_l2 (Q+K+V 201 MB, output 134 MB per step vs 126 MB L2)",
+                   "step": "quantize_qk + quantize_v + prefill"},
+        "clocks": clocks,
+        "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOPS", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": (q.numel() + k.numel() + v.numel()) * 2, "d2h_bytes_per_step": out.numel() * 2},
+        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "roofline": {"kernel": "prefill_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
+                     "unit": "TFLOP/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(N),
+                     "kernel_ms": kernel_ms,
+                     "peak_note": f"{peaks['source']} bf16 {'sustained' if long_run else 'burst'} {bf16_peak} TF/s x 8/3 "
+                                  "(nominal fp4 4x / fp8 2x of bf16; equal FP4 and FP8 FLOPs per pair)",
+                     "exp_ceiling_tflops_at_sampled_clock":
+                         (148 * 16 * clocks["sm_mhz"] * 1e6 * 512 / 1e12) if clocks.get("sm_mhz") else None},
+        "prefill_kernel_only": {"value": achieved, "unit": "TFLOPS", "ms": kernel_ms,
+                                "note": "attention kernel alone, quantization excluded (as the paper times it)"},
+        "quantize_ms": ms_step - kernel_ms,
+    }
+    if rank == 0:
+        if not args.no_decode:
+            try:
+                result["decode"] = bench_decode(binding, wl, max(3, args.steps // 2), 3, peaks, args.small_decode)
+            except Exception as e:  # decode is a secondary line; never lose the main one
+                result["decode"] = {"error": repr(e)}
+        if world == 1 and not args.no_cpu:
+            cores = os.cpu_count() or 1
+            fl, times, sample = cpu_oracle_sample(w, 1, rows_per_head=args.cpu_rows_per_head)
+            result["cpu_baseline"] = {"value": fl / times[0] / 1e12, "unit": "TFLOPS", "cores": cores,
+                                      "kind": "oracle", "sample": sample, "seconds": times[0]}
+        print(json.dumps(result))
+
+
+# DRAM bytes per prefill launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum);
+# filled in from profiles/ once captured, keyed by sequence length.
+NCU_TRAFFIC_BYTES = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--seq-len", type=int, default=16384)
+    ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--small-decode", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-rows-per-head", type=int, default=2048)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args, int(os.environ.get("RANK", 0)))
+        return
+    rank, world, local = dist_setup(args.gpus)
+    try:
+        run_ours(args, rank, world, local)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
