@@ -113,6 +113,7 @@ typedef struct {
   void *delta_s_bf16;
   int32_t num_pages;
   int32_t page_size; /* must be 64 */
+  int32_t H_q, H_kv; /* head counts the pools were sized for */
 } mpfa_paged_kv;
 
 /* ---- stage 1: Algorithm 1 lines 1-5 -------------------------------------------------- */

@@ -40,7 +40,8 @@ class _Fp4(ctypes.Structure):
 
 class _PagedKV(ctypes.Structure):
     _fields_ = [("k_codes", ctypes.c_void_p), ("k_sf", ctypes.c_void_p), ("v_fp8", ctypes.c_void_p),
-                ("delta_s_bf16", ctypes.c_void_p), ("num_pages", ctypes.c_int32), ("page_size", ctypes.c_int32)]
+                ("delta_s_bf16", ctypes.c_void_p), ("num_pages", ctypes.c_int32), ("page_size", ctypes.c_int32),
+                ("H_q", ctypes.c_int32), ("H_kv", ctypes.c_int32)]
 
 
 _lib = None
@@ -181,7 +182,8 @@ class PagedKV:
 
     def c(self) -> _PagedKV:
         return _PagedKV(self.k_codes.data_ptr(), self.k_sf.data_ptr(), self.v_fp8.data_ptr(),
-                        None if self.delta is None else self.delta.data_ptr(), self.num_pages, PAGE)
+                        None if self.delta is None else self.delta.data_ptr(), self.num_pages, PAGE,
+                        self.H_q, self.H_kv)
 
 
 def quantize_workspace(B: int, H_q: int, H_kv: int, device="cuda") -> torch.Tensor:

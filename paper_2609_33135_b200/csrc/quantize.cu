@@ -466,6 +466,7 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
   if (!kv->k_codes || !kv->k_sf || !kv->v_fp8 || kv->num_pages <= 0) return MPFA_ERR_INVALID_ARG;
   if (smooth && !kv->delta_s_bf16) return MPFA_ERR_INVALID_ARG;
   if (kv->page_size != PAGE || H_q % H_kv != 0 || H_q / H_kv > 8) return MPFA_ERR_UNSUPPORTED;
+  if (kv->H_q != H_q || kv->H_kv != H_kv) return MPFA_ERR_INVALID_ARG;
   if (first_token % PAGE != 0) return MPFA_ERR_UNSUPPORTED;  // appends inside a partly filled page: not built yet
   if (!frozen && first_token != 0) return MPFA_ERR_INVALID_ARG;
   if (!aligned(k_bf16, 16) || !aligned(v_bf16, 16) || !aligned(kv->k_codes, 256) || !aligned(kv->k_sf, 256) ||

@@ -168,14 +168,25 @@ class DecodeWorkload:
     seed: int
     n_outlier: int
 
-    def kv_for_request(self, b: int):
-        """K, V [1, L_b, H_kv, 128] (BF16, CPU) of request b, drawn on demand."""
+    def kv_for_request(self, b: int, device: str = "cpu"):
+        """K, V [1, L_b, H_kv, 128] (BF16) of request b, drawn on demand.  On "cpu" the draw
+        uses the CPU generator; on a CUDA device it uses that device's generator with the same
+        seed (a different but equally reproducible stream), which keeps the 128K-token
+        benchmark cache off the host."""
         L = int(self.seq_lens[b])
         s = self.seed * 64 + b
-        k = _randn_chunked((L, self.H_kv, HEAD_DIM), _gen(s, "k")).view(1, L, self.H_kv, HEAD_DIM)
         bias, factor = k_structure(self.seed, self.H_kv, self.n_outlier)
+        if device == "cpu":
+            k = _randn_chunked((L, self.H_kv, HEAD_DIM), _gen(s, "k")).view(1, L, self.H_kv, HEAD_DIM)
+            v = _randn_chunked((L, self.H_kv, HEAD_DIM), _gen(s, "v")).view(1, L, self.H_kv, HEAD_DIM)
+        else:
+            g = torch.Generator(device=device)
+            g.manual_seed(s * 16 + _SUB["k"])
+            k = torch.randn(1, L, self.H_kv, HEAD_DIM, generator=g, device=device)
+            g.manual_seed(s * 16 + _SUB["v"])
+            v = torch.randn(1, L, self.H_kv, HEAD_DIM, generator=g, device=device)
+            bias, factor = bias.to(device), factor.to(device)
         k = k * factor + bias
-        v = _randn_chunked((L, self.H_kv, HEAD_DIM), _gen(s, "v")).view(1, L, self.H_kv, HEAD_DIM)
         return _finish(k), _finish(v)
 
     @property
@@ -185,8 +196,12 @@ class DecodeWorkload:
 
 def decode_workload(name: str, seed: int, B: int, H_q: int, H_kv: int, len_lo: int, len_hi: int,
                     n_stat_tokens: int = 1024, shuffle_pages: bool = True,
-                    extra_pages: int = 3) -> DecodeWorkload:
-    seq_lens = torch.randint(len_lo, len_hi + 1, (B,), generator=_gen(seed, "seq_lens"), dtype=torch.int64)
+                    extra_pages: int = 3, seq_lens=None) -> DecodeWorkload:
+    if seq_lens is None:
+        seq_lens = torch.randint(len_lo, len_hi + 1, (B,), generator=_gen(seed, "seq_lens"), dtype=torch.int64)
+    else:
+        seq_lens = torch.as_tensor(seq_lens, dtype=torch.int64)
+        assert seq_lens.shape == (B,)
     pages_per_req = (seq_lens + PAGE_SIZE - 1) // PAGE_SIZE
     total = int(pages_per_req.sum())
     num_pages = total + extra_pages

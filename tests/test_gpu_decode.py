@@ -1,0 +1,112 @@
+"""GPU parity: paged cache write (bit-exact) and split-KV decode (tolerance) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mpfa_oracle as orc
+from paper_2609_33135_b200 import workloads as wl
+
+from layouts import paged_k_to_logical, paged_v_to_logical
+from test_gpu_prefill import MAX_ABS, MEAN_ABS, bf16_neighbours_ok
+
+pytestmark = pytest.mark.gpu
+
+
+def oracle_decode(w, smooth=True, v_scale=1.0):
+    """Per request: stage 1 with the frozen query statistics, then the partitioned main loop."""
+    outs32, outs16, caches = [], [], []
+    for b in range(w.B):
+        k, v = w.kv_for_request(b)
+        qs = w.q_sample[b:b + 1].contiguous()
+        z = orc.stage1(orc.bf16_bits(qs), orc.bf16_bits(k), orc.bf16_bits(v), smooth=smooth, v_scale=v_scale)
+        zq = orc.stage1(orc.bf16_bits(w.q_new[b:b + 1].contiguous()), orc.bf16_bits(k), orc.bf16_bits(v),
+                        smooth=smooth, v_scale=v_scale, frozen=z)
+        o32, o16 = orc.decode(zq.q_codes[:, :, 0], zq.q_sf[:, :, 0], z.k_codes, z.k_sf, z.v_codes, z.delta, z.dq,
+                              z.dk, v_scale, w.softmax_scale, np.array([int(w.seq_lens[b])], np.int32))
+        outs32.append(o32[0])
+        outs16.append(o16[0])
+        caches.append(z)
+    return np.stack(outs32), np.stack(outs16), caches
+
+
+def check_cache(state, w, caches, smooth=True):
+    kc = state.kv.k_codes.cpu().numpy()
+    ks = state.kv.k_sf.cpu().numpy()
+    vv = state.kv.v_fp8.cpu().numpy()
+    dl = state.kv.delta.view(torch.uint16).cpu().numpy() if smooth else None
+    for b in range(w.B):
+        z, L = caches[b], int(w.seq_lens[b])
+        for i in range((L + 63) // 64):
+            page = int(w.page_table[b, i])
+            n = min(64, L - 64 * i)
+            lk = paged_k_to_logical(kc[page])          # [H_kv, 64, 64]
+            lv = paged_v_to_logical(vv[page])          # [H_kv, 64, 128]
+            assert np.array_equal(lk[:, :n], z.k_codes[0, :, 64 * i:64 * i + n])
+            assert np.array_equal(ks[page].reshape(w.H_kv, 64, 8)[:, :n], z.k_sf[0, :, 64 * i:64 * i + n])
+            assert np.array_equal(lv[:, :n], z.v_codes[0, :, 64 * i:64 * i + n])
+            assert not lk[:, n:].any() and not lv[:, n:].any()
+            if smooth:
+                assert np.array_equal(dl[page][:, :n], z.delta[0, :, 64 * i:64 * i + n])
+                assert not dl[page][:, n:].any()
+
+
+def run(w, smooth=True, v_scale=1.0):
+    from paper_2609_33135_b200 import decode_cache
+    st = decode_cache.build_cache(w, smooth=smooth, v_scale=v_scale)
+    decode_cache.decode_step(st)
+    torch.cuda.synchronize()
+    assert int(st.status.item()) == 0
+    return st
+
+
+def compare(st, ref32):
+    g32 = st.out_f32.cpu().numpy()
+    g16 = st.out.view(torch.uint16).cpu().numpy()
+    d = np.abs(g32 - ref32)
+    assert np.isfinite(g32).all()
+    assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (float(d.max()), float(d.mean()))
+    assert np.array_equal(g16, torch.from_numpy(g32.copy()).to(torch.bfloat16).view(torch.uint16).numpy())
+    assert bf16_neighbours_ok(g16, ref32).all()
+
+
+@pytest.mark.parametrize("hq,hkv", [(8, 2), (10, 2), (4, 4)])
+def test_decode_matches_oracle(hq, hkv):
+    # lengths that hit the edges: one key, one page, one block + 1, one partition + 1, ragged multi-partition
+    w = wl.decode_workload("dec_small", 61 + hq, 5, hq, hkv, 1, 2600, seq_lens=[1, 64, 129, 1025, 2600])
+    ref32, ref16, caches = oracle_decode(w)
+    st = run(w)
+    check_cache(st, w, caches)
+    compare(st, ref32)
+
+
+def test_decode_direct_variant_and_v_scale():
+    w = wl.decode_workload("dec_direct", 71, 3, 8, 2, 300, 3000)
+    ref32, _, caches = oracle_decode(w, smooth=False, v_scale=0.5)
+    st = run(w, smooth=False, v_scale=0.5)
+    check_cache(st, w, caches, smooth=False)
+    compare(st, ref32)
+
+
+def test_decode_independent_of_page_permutation_and_repeatable():
+    w1 = wl.decode_workload("dec_perm", 72, 3, 8, 2, 500, 2500, shuffle_pages=True)
+    w2 = wl.decode_workload("dec_perm", 72, 3, 8, 2, 500, 2500, shuffle_pages=False)
+    assert not torch.equal(w1.page_table, w2.page_table)
+    a, b = run(w1), run(w2)
+    assert torch.equal(a.out, b.out) and torch.equal(a.out_f32, b.out_f32)
+    from paper_2609_33135_b200 import decode_cache
+    first = a.out_f32.clone()
+    decode_cache.decode_step(a)
+    torch.cuda.synchronize()
+    assert torch.equal(first, a.out_f32)
+
+
+def test_decode_bad_page_is_reported_not_followed():
+    from paper_2609_33135_b200 import decode_cache
+    w = wl.decode_workload("dec_bad", 73, 2, 8, 2, 200, 400)
+    st = run(w)
+    st.page_table[1, 1] = st.kv.num_pages + 5
+    st.status.zero_()
+    decode_cache.decode_step(st)
+    torch.cuda.synchronize()
+    assert int(st.status.item()) & 2
+    assert torch.isfinite(st.out_f32).all()
