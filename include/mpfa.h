@@ -134,6 +134,29 @@ mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, int B, int 
                              mpfa_fp4_tensor *h_k_out, void *delta_s_bf16, void *workspace,
                              size_t workspace_bytes, void *stream);
 
+/* (No counterpart in the paper: a convenience for embedders.)
+ * mpfa_quantize_qk for callers that cannot hand the library any scratch memory - code
+ * that runs where device allocation is forbidden or unavailable: inside a serving loop
+ * whose memory pool is fully pre-assigned, in a plugin that is given only its input and
+ * output tensors, or after the process has dropped the right to call the allocator.
+ * Arguments and results are exactly those of mpfa_quantize_qk without the workspace pair.
+ * The column sums and maxima live in a fixed MPFA_STATIC_SCRATCH_BYTES buffer that is
+ * part of the library image: every GPU that loads the library carries it until the
+ * process exits.  Shapes whose statistics need more (mpfa_quantize_workspace_bytes(B, H_q,
+ * H_kv) > MPFA_STATIC_SCRATCH_BYTES, i.e. roughly B * (H_q + H_kv) > 500) are rejected
+ * with MPFA_ERR_WORKSPACE and nothing is launched.  The call allocates nothing and frees
+ * nothing.  The first call on each device looks up the buffer's device address (with that
+ * device current); make that first call before starting any stream capture.  All calls on
+ * a device share the one buffer, which keeps whatever the previous call left in it: each
+ * call clears what it needs on `stream` before use, and two calls whose GPU work overlaps
+ * (different streams, or different host threads on different streams) race on it - keep
+ * them on one stream or order them yourself. */
+#define MPFA_STATIC_SCRATCH_BYTES (512 * 1024)
+mpfa_status mpfa_quantize_qk_static(const void *q_bf16, const void *k_bf16, int B, int N_q, int N_kv, int H_q,
+                                    int H_kv, int flags, mpfa_stats *h_stats, mpfa_fp4_tensor *h_q_out,
+                                    mpfa_fp4_tensor *h_k_out, void *delta_s_bf16, void *stream);
+size_t mpfa_static_scratch_bytes(void);
+
 /* Algorithm 1 line 4: V is not centered; code = E4M3(v / v_scale), round to nearest even,
  * saturating at +-448.  v_bf16 [B, N_kv, H_kv, 128] -> v_fp8 [B, H_kv, N_kv_pad, 128]
  * (1024-byte aligned).  v_scale = 1.0f is the plain cast. */

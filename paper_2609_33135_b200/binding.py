@@ -75,6 +75,10 @@ def lib() -> ctypes.CDLL:
         L.mpfa_quantize_qk.restype = i
         L.mpfa_quantize_qk.argtypes = [vp, vp, i, i, i, i, i, i, ctypes.POINTER(_Stats), ctypes.POINTER(_Fp4),
                                        ctypes.POINTER(_Fp4), vp, vp, sz, vp]
+        L.mpfa_quantize_qk_static.restype = i
+        L.mpfa_quantize_qk_static.argtypes = [vp, vp, i, i, i, i, i, i, ctypes.POINTER(_Stats), ctypes.POINTER(_Fp4),
+                                              ctypes.POINTER(_Fp4), vp, vp]
+        L.mpfa_static_scratch_bytes.restype = sz
         L.mpfa_quantize_v.restype = i
         L.mpfa_quantize_v.argtypes = [vp, i, i, i, f, vp, vp]
         L.mpfa_quantize_kv_paged.restype = i
@@ -210,6 +214,28 @@ def mpfa_quantize_qk(q: Optional[torch.Tensor], k: Optional[torch.Tensor], flags
                                 ctypes.byref(kc) if kc is not None else None, _ptr(delta), _ptr(workspace),
                                 0 if workspace is None else workspace.numel(), _stream())
     _check(rc, "mpfa_quantize_qk")
+
+
+def mpfa_quantize_qk_static(q: Optional[torch.Tensor], k: Optional[torch.Tensor], flags: int, stats: Stats,
+                            q_out: Optional[Fp4Tensor], k_out: Optional[Fp4Tensor],
+                            delta: Optional[torch.Tensor]) -> None:
+    """mpfa_quantize_qk without a workspace argument: for callers that may not allocate device
+    memory.  The library's own fixed scratch buffer is used; shapes that need more than
+    mpfa_static_scratch_bytes() raise MpfaError("workspace too small").  This wrapper itself
+    allocates nothing on the device.  Calls overlapping on the GPU share that buffer and race."""
+    ref = q if q is not None else k
+    B = ref.shape[0]
+    N_q = q.shape[1] if q is not None else 0
+    N_kv = k.shape[1] if k is not None else 0
+    H_q = q.shape[2] if q is not None else stats.q_mean.shape[1]
+    H_kv = k.shape[2] if k is not None else stats.k_mean.shape[1]
+    sc = stats.c()
+    qc = q_out.c() if q_out is not None else None
+    kc = k_out.c() if k_out is not None else None
+    rc = lib().mpfa_quantize_qk_static(_ptr(q), _ptr(k), B, N_q, N_kv, H_q, H_kv, flags, ctypes.byref(sc),
+                                       ctypes.byref(qc) if qc is not None else None,
+                                       ctypes.byref(kc) if kc is not None else None, _ptr(delta), _stream())
+    _check(rc, "mpfa_quantize_qk_static")
 
 
 def mpfa_quantize_v(v: torch.Tensor, v_scale: float, out: torch.Tensor) -> None:

@@ -11,6 +11,8 @@
 #include <cuda_fp4.h>
 #include <cuda_fp8.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mpfa {
@@ -501,4 +503,51 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
     MPFA_LAUNCH_OK();
   }
   return MPFA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// mpfa_quantize_qk_static: the same stage-1 call for callers that cannot provide scratch.
+// ---------------------------------------------------------------------------------------
+namespace mpfa {
+namespace {
+
+// Scratch for the column sums and maxima, resident in every device that loads the library.
+constexpr size_t STATIC_SCRATCH_BYTES = MPFA_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+void *g_static_scratch_addr[MAX_DEVICES] = {};
+std::mutex g_static_scratch_mutex;
+
+// In host code the array's name is only a handle; the device address has to be asked for,
+// once per device, with that device current.
+mpfa_status static_scratch_address(void **out) {
+  int dev = 0;
+  MPFA_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= MAX_DEVICES) return MPFA_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (!g_static_scratch_addr[dev]) {
+    void *ptr = nullptr;
+    MPFA_CUDA_OK(cudaGetSymbolAddress(&ptr, g_static_scratch));
+    g_static_scratch_addr[dev] = ptr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return MPFA_OK;
+}
+
+}  // namespace
+}  // namespace mpfa
+
+extern "C" size_t mpfa_static_scratch_bytes(void) { return STATIC_SCRATCH_BYTES; }
+
+extern "C" mpfa_status mpfa_quantize_qk_static(const void *q_bf16, const void *k_bf16, int B, int N_q, int N_kv,
+                                               int H_q, int H_kv, int flags, mpfa_stats *st, mpfa_fp4_tensor *q_out,
+                                               mpfa_fp4_tensor *k_out, void *delta_s_bf16, void *stream) {
+  if (B <= 0 || H_q <= 0 || H_kv <= 0) return MPFA_ERR_INVALID_ARG;
+  if (carve(nullptr, B, H_q, H_kv).bytes > STATIC_SCRATCH_BYTES) return MPFA_ERR_WORKSPACE;
+  void *scratch = nullptr;
+  mpfa_status rc = static_scratch_address(&scratch);
+  if (rc != MPFA_OK) return rc;
+  return mpfa_quantize_qk(q_bf16, k_bf16, B, N_q, N_kv, H_q, H_kv, flags, st, q_out, k_out, delta_s_bf16, scratch,
+                          STATIC_SCRATCH_BYTES, stream);
 }
