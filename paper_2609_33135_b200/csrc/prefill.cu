@@ -1,22 +1,30 @@
 // QK4PV8 prefill (Algorithm 1 lines 6-20) for sm_100a.
 //
 // One CTA owns one 128-row query tile of one q head and walks its KV blocks (128 keys)
-// from the last visible block down to block 0 (Section 4.1).  Roles:
-//   warp 0      TMA producer: K codes (tensor map, 64B swizzle), K scale factors and
-//               Delta_S (bulk copies) and V (tensor map, 128B swizzle) into a 3-stage ring;
-//   warp 1      MMA issuer: per block a rank-one BF16 MMA seeds S with 1 x Delta_S
-//               (Eq. 11), two block-scaled FP4 MMAs (K = 64 each) accumulate Q K^T into
-//               the same TMEM columns, and four FP8 MMAs (A = P_hat from TMEM, B = V from
-//               shared memory, MN-major) accumulate P V into O;
-//   warps 4-7   softmax: one thread per row; mask, running max, 2^(lam S - lam m), row sum
-//               from the unquantized P, P -> E4M3 at the fixed scale 448 written back over
-//               the first 32 columns of the score buffer (Algorithm 1 lines 11-14);
-//   warps 8-11  correction + epilogue: O *= alpha whenever a row's maximum moved
-//               (Eq. 6), final O / (448 l) * v_scale -> BF16.
-// Tensor memory (512 columns): S0 [0,128) S1 [128,256) O [256,384), scale factors of Q
-// [384,392) and of the two in-flight K blocks [392,400) [400,408).  The score buffer is
-// double-buffered over KV blocks so Q K^T of block t+1 overlaps the softmax of block t and
-// P V of block t overlaps the softmax of block t+1.
+// from the last visible block down to block 0 (Section 4.1).  Roles (512 threads):
+//   warp 0       TMA producer: K codes (tensor map, 64B swizzle), K scale factors and
+//                Delta_S (bulk copies) and V (tensor map, 128B swizzle) into 3-stage rings;
+//   warp 1       Q K^T issuer: per block a rank-one BF16 MMA seeds S with 1 x Delta_S
+//                (Eq. 11) and two block-scaled FP4 MMAs (K = 64 each) accumulate Q K^T into
+//                the same TMEM columns;
+//   warp 3       P V issuer: four FP8 MMAs per block (A = P_hat from TMEM, B = V from
+//                shared memory, MN-major) accumulate P V into O;
+//   warps 4-7    softmax of the even-numbered blocks of the traversal (score buffer S0);
+//   warps 8-11   softmax of the odd-numbered blocks (score buffer S1).  One thread per row:
+//                the whole 128-column row is read into registers once; mask, row maximum,
+//                running maximum handed from one group to the other through shared memory
+//                (only the maximum is loop-carried, so the exponentials of block t overlap
+//                the maximum pass and exponentials of block t+1), 2^(lam S - lam m), row sum
+//                from the unquantized P, P -> E4M3 at the fixed scale 448 written to its own
+//                32 TMEM columns (Algorithm 1 lines 11-14).  The score buffer is handed back to
+//                the MMA warp as soon as the row is in registers, so Q K^T runs two blocks
+//                ahead of P V and a softmax group never waits for its next scores;
+//   warps 12-15  correction + epilogue: O *= alpha whenever a row's maximum moved
+//                (Eq. 6), final O / (448 l) * v_scale -> BF16.
+// Tensor memory (512 columns): S0 [0,128) S1 [128,256) O [256,384), P_hat0 [384,416)
+// P_hat1 [416,448), scale factors of Q [448,456) and of the two in-flight K blocks
+// [456,464) [464,472).
+// Register budget is moved between the roles with setmaxnreg (88 / 168 / 168 / 88).
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises MPFA_DEV_TIMEOUT in
 // *device_status, all roles leave their loops, outstanding TMA copies are drained and
@@ -31,10 +39,11 @@
 namespace mpfa {
 namespace {
 
-constexpr int KSTAGES = 3;
+constexpr int KSTAGES = 4;
 constexpr int VSTAGES = 3;
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // 2 s: far beyond any legitimate wait
-constexpr int NTHREADS = 384;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM clock: far beyond any legitimate wait
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;       // drain path only
+constexpr int NTHREADS = 512;
 
 constexpr uint32_t OFF_Q = 0;
 constexpr uint32_t OFF_K = OFF_Q + 8192;
@@ -43,9 +52,10 @@ constexpr uint32_t OFF_DELTA = OFF_V + VSTAGES * 16384;
 constexpr uint32_t OFF_ONES = OFF_DELTA + KSTAGES * 4096;
 constexpr uint32_t OFF_SFQ = OFF_ONES + 4096;
 constexpr uint32_t OFF_SFK = OFF_SFQ + 1024;
-constexpr uint32_t OFF_ALPHA = OFF_SFK + KSTAGES * 1024;
-constexpr uint32_t OFF_L = OFF_ALPHA + 2 * 128 * 4;
-constexpr uint32_t OFF_BAR = OFF_L + 128 * 4;
+constexpr uint32_t OFF_ALPHA = OFF_SFK + KSTAGES * 1024;   // alpha[2][128]
+constexpr uint32_t OFF_M = OFF_ALPHA + 2 * 128 * 4;        // running maximum after block t, [t & 1][128]
+constexpr uint32_t OFF_L = OFF_M + 2 * 128 * 4;            // final (l, m) of the two softmax groups, [2][2][128]
+constexpr uint32_t OFF_BAR = OFF_L + 4 * 128 * 4;
 enum {
   BAR_Q_FULL = 0,
   BAR_K_FULL = 1,
@@ -54,8 +64,10 @@ enum {
   BAR_V_EMPTY = BAR_V_FULL + VSTAGES,
   BAR_S_FULL = BAR_V_EMPTY + VSTAGES,
   BAR_P_FULL = BAR_S_FULL + 2,
-  BAR_A_FULL = BAR_P_FULL + 2,
-  BAR_O_FULL = BAR_A_FULL + 2,
+  BAR_S_EMPTY = BAR_P_FULL + 2,  // score buffer read into registers, free for the next Q K^T
+  BAR_P_EMPTY = BAR_S_EMPTY + 2, // P V has consumed this P_hat buffer
+  BAR_M_FULL = BAR_P_EMPTY + 2,  // running maximum and alpha of block t published
+  BAR_O_FULL = BAR_M_FULL + 2,
   BAR_O_READY = BAR_O_FULL + 1,
   BAR_L_FULL = BAR_O_READY + 1,
   NUM_BARS = BAR_L_FULL + 1
@@ -63,7 +75,8 @@ enum {
 constexpr uint32_t OFF_MISC = OFF_BAR + NUM_BARS * 8;   // tmem base, abort flag
 constexpr uint32_t SMEM_BYTES = OFF_MISC + 16 + 1024;   // + slack for the 1024-byte alignment
 
-constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_O = 256, TM_SFQ = 384, TM_SFK0 = 392, TM_SFK1 = 400;
+constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_O = 256, TM_P0 = 384, TM_P1 = 416, TM_SFQ = 448, TM_SFK0 = 456,
+                   TM_SFK1 = 464;
 constexpr uint32_t TMEM_COLS = 512;
 
 struct PrefillParams {
@@ -86,22 +99,55 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+// Optional timeline capture for tuning (compiled in only with -DMPFA_TRACE): one CTA records
+// clock64() at fixed points of every role, [role][block][event].
+#ifdef MPFA_TRACE
+__device__ long long *g_trace = nullptr;
+__device__ int g_trace_cta = 0;
+#define TR_INIT() long long *tr_buf = ((int)blockIdx.x == g_trace_cta && lane == 0) ? g_trace : nullptr
+#define TR(role, t, ev)                                                              \
+  do {                                                                               \
+    if (tr_buf && (t) < 256) tr_buf[((role) * 256 + (t)) * 8 + (ev)] = clock64();    \
+  } while (0)
+#else
+#define TR_INIT() do {} while (0)
+#define TR(role, t, ev) do {} while (0)
+#endif
+
 struct Ctx {
   uint32_t bars;      // shared address of barrier 0
   volatile int *abort_flag;
   int32_t *status;
   __device__ __forceinline__ uint32_t bar(int i) const { return bars + 8u * (uint32_t)i; }
-  // Wait bounded in wall-clock time (try_wait itself may suspend the thread for a
-  // system-dependent interval, so an iteration count alone does not bound the wait).
-  // Also gives up as soon as another role has failed.
+  // Bounded wait.  try_wait may itself suspend the thread for a system-dependent interval, so
+  // the bound is on elapsed SM clock cycles (about 2 s), checked once per 32 polls to keep the
+  // hand-off latency at the cost of a poll.  Also gives up as soon as another role has failed.
   __device__ __forceinline__ bool wait(int i, uint32_t parity) const {
     const uint32_t a = bar(i);
     if (mbar_try_wait(a, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+    const long long t0 = clock64();
     for (;;) {
-      if (mbar_try_wait(a, parity)) return true;
+#pragma unroll 1
+      for (int k = 0; k < 32; ++k) {
+        if (mbar_try_wait(a, parity)) return true;
+        __nanosleep(20);
+      }
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) break;
+      if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
     }
     *abort_flag = 1;
     atomicOr(status, MPFA_DEV_TIMEOUT);
@@ -150,11 +196,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     for (int i = 0; i < 2; ++i) {
       mbar_init(cx.bar(BAR_S_FULL + i), 1);
       mbar_init(cx.bar(BAR_P_FULL + i), 128);
-      mbar_init(cx.bar(BAR_A_FULL + i), 128);
+      mbar_init(cx.bar(BAR_M_FULL + i), 128);
+      mbar_init(cx.bar(BAR_S_EMPTY + i), 128);
+      mbar_init(cx.bar(BAR_P_EMPTY + i), 1);
     }
     mbar_init(cx.bar(BAR_O_FULL), 1);
     mbar_init(cx.bar(BAR_O_READY), 128);
-    mbar_init(cx.bar(BAR_L_FULL), 128);
+    mbar_init(cx.bar(BAR_L_FULL), 256);
     mbar_init_fence();
     prefetch_tmap(&tm_q);
     prefetch_tmap(&tm_k);
@@ -177,36 +225,48 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const uint32_t tm = *tmem_slot;
 
   const bool has_delta = p.delta != nullptr;
+  TR_INIT();
   const size_t q_row = ((size_t)b * p.H_q + hq) * (size_t)(p.nq_tiles * TILE) + row0;
   const size_t k_row = ((size_t)b * p.H_kv + hk) * (size_t)(p.nk_tiles * TILE);
 
+  if (warp < 4) setmaxnreg_dec<88>();
   if (warp == 0) {
     // =========================== TMA producer ===========================
-    if (lane == 0 && T > 0) {
+    // The whole warp runs the loop (uniform control flow keeps addresses and barrier handles in
+    // uniform registers); a single elected lane issues each copy.
+    if (T > 0) {
       int armed = 0;
-      mbar_expect_tx(cx.bar(BAR_Q_FULL), 8192 + 1024);
-      tma_load_2d(sbase + OFF_Q, &tm_q, 0, (int)q_row, cx.bar(BAR_Q_FULL));
-      bulk_load(sbase + OFF_SFQ, p.q_sf + (((size_t)b * p.H_q + hq) * p.nq_tiles + qt) * 1024, 1024,
-                cx.bar(BAR_Q_FULL));
+      if (elect_one()) {
+        mbar_expect_tx(cx.bar(BAR_Q_FULL), 8192 + 1024);
+        tma_load_2d(sbase + OFF_Q, &tm_q, 0, (int)q_row, cx.bar(BAR_Q_FULL));
+        bulk_load(sbase + OFF_SFQ, p.q_sf + (((size_t)b * p.H_q + hq) * p.nq_tiles + qt) * 1024, 1024,
+                  cx.bar(BAR_Q_FULL));
+      }
       bool ok = true;
       for (int t = 0; t < T && ok; ++t) {
         const int jb = T - 1 - t;
         const int ks = t % KSTAGES, vs = t % VSTAGES;
         if (t >= KSTAGES) ok = cx.wait(BAR_K_EMPTY + ks, (uint32_t)(t / KSTAGES - 1) & 1u);
         if (!ok) break;
-        mbar_expect_tx(cx.bar(BAR_K_FULL + ks), 8192 + 1024 + (has_delta ? 256 : 0));
-        tma_load_2d(sbase + OFF_K + ks * 8192, &tm_k, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_K_FULL + ks));
-        bulk_load(sbase + OFF_SFK + ks * 1024, p.k_sf + (((size_t)b * p.H_kv + hk) * p.nk_tiles + jb) * 1024, 1024,
-                  cx.bar(BAR_K_FULL + ks));
-        if (has_delta) {
-          const __nv_bfloat16 *d = p.delta + ((size_t)b * p.H_q + hq) * (size_t)(p.nk_tiles * TILE) + (size_t)jb * TILE;
-          bulk_load(sbase + OFF_DELTA + ks * 4096, d, 128, cx.bar(BAR_K_FULL + ks));
-          bulk_load(sbase + OFF_DELTA + ks * 4096 + 2048, d + 64, 128, cx.bar(BAR_K_FULL + ks));
+        TR(0, t, 0);
+        if (elect_one()) {
+          mbar_expect_tx(cx.bar(BAR_K_FULL + ks), 8192 + 1024 + (has_delta ? 256 : 0));
+          tma_load_2d(sbase + OFF_K + ks * 8192, &tm_k, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_K_FULL + ks));
+          bulk_load(sbase + OFF_SFK + ks * 1024, p.k_sf + (((size_t)b * p.H_kv + hk) * p.nk_tiles + jb) * 1024, 1024,
+                    cx.bar(BAR_K_FULL + ks));
+          if (has_delta) {
+            const __nv_bfloat16 *d = p.delta + ((size_t)b * p.H_q + hq) * (size_t)(p.nk_tiles * TILE) + (size_t)jb * TILE;
+            bulk_load(sbase + OFF_DELTA + ks * 4096, d, 128, cx.bar(BAR_K_FULL + ks));
+            bulk_load(sbase + OFF_DELTA + ks * 4096 + 2048, d + 64, 128, cx.bar(BAR_K_FULL + ks));
+          }
         }
         if (t >= VSTAGES) ok = cx.wait(BAR_V_EMPTY + vs, (uint32_t)(t / VSTAGES - 1) & 1u);
         if (!ok) { armed = -(t + 1); break; }   // K of block t armed, V not
-        mbar_expect_tx(cx.bar(BAR_V_FULL + vs), 16384);
-        tma_load_2d(sbase + OFF_V + vs * 16384, &tm_v, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
+        TR(0, t, 1);
+        if (elect_one()) {
+          mbar_expect_tx(cx.bar(BAR_V_FULL + vs), 16384);
+          tma_load_2d(sbase + OFF_V + vs * 16384, &tm_v, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
+        }
         armed = t + 1;
       }
       if (*cx.abort_flag) {
@@ -220,136 +280,215 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
     }
   } else if (warp == 1) {
-    // =========================== MMA issuer ===========================
-    if (lane == 0 && T > 0) {
+    // =========================== Q K^T issuer ===========================
+    // Whole warp in uniform control flow; lane 0 (always the elected lane of a full warp) issues
+    // every tcgen05 instruction, so the commits track the MMAs of the same thread.  This warp
+    // only waits for operands (K block in shared memory, score buffer handed back by its
+    // softmax group), so it runs up to two blocks ahead of the P V issuer (warp 3).
+    if (T > 0) {
       const uint32_t id_fp4 = idesc_nvfp4(128, 128);
       const uint32_t id_bf16 = idesc_bf16(128, 128, 1, 1);
-      const uint32_t id_fp8 = idesc_e4m3(128, 128, 0, 1);
+      // All shared-memory descriptors are built once; a ring stage or K step only adds a
+      // constant to the 14-bit start-address field (shared addresses stay below 256 KB).
       const uint64_t d_ones = smem_desc(sbase + OFF_ONES, 2048, 1024, SWZ_128B);
+      const uint64_t d_delta0 = smem_desc(sbase + OFF_DELTA, 2048, 1024, SWZ_128B);
+      const uint64_t d_q0 = smem_desc(sbase + OFF_Q, 16, 512, SWZ_64B);
+      const uint64_t d_k0 = smem_desc(sbase + OFF_K, 16, 512, SWZ_64B);
+      const uint64_t d_sfq0 = smem_desc(sbase + OFF_SFQ, 0, 128, SWZ_NONE);
+      const uint64_t d_sfk0 = smem_desc(sbase + OFF_SFK, 0, 128, SWZ_NONE);
       bool ok = cx.wait(BAR_Q_FULL, 0);
       if (ok) {
         tc_fence_after();
-        for (int kc = 0; kc < 2; ++kc)
-          tmem_cp_32x128b_warpx4(tm + TM_SFQ + 4 * kc, smem_desc(sbase + OFF_SFQ + 512 * kc, 0, 128, SWZ_NONE));
+        if (elect_one()) {
+          tmem_cp_32x128b_warpx4(tm + TM_SFQ, d_sfq0);
+          tmem_cp_32x128b_warpx4(tm + TM_SFQ + 4, d_sfq0 + (512 >> 4));
+        }
       }
-      auto issue_qk = [&](int t) -> bool {
+      for (int t = 0; t < T && ok; ++t) {
         const int ks = t % KSTAGES, sb = t & 1;
-        if (!cx.wait(BAR_K_FULL + ks, (uint32_t)(t / KSTAGES) & 1u)) return false;
+        TR(5, t, 0);
+        ok = cx.wait(BAR_K_FULL + ks, (uint32_t)(t / KSTAGES) & 1u);
+        // the softmax group that owns this score buffer has read block t-2 out of it
+        if (ok && t >= 2) ok = cx.wait(BAR_S_EMPTY + sb, (uint32_t)((t >> 1) - 1) & 1u);
+        if (!ok) break;
+        TR(5, t, 1);
         tc_fence_after();
         const uint32_t tS = tm + (sb ? TM_S1 : TM_S0);
         const uint32_t tSFK = tm + (sb ? TM_SFK1 : TM_SFK0);
-        for (int kc = 0; kc < 2; ++kc)
-          tmem_cp_32x128b_warpx4(tSFK + 4 * kc, smem_desc(sbase + OFF_SFK + ks * 1024 + 512 * kc, 0, 128, SWZ_NONE));
-        uint32_t acc = 0;
-        if (has_delta) {
-          mma_bf16_ss(tS, d_ones, smem_desc(sbase + OFF_DELTA + ks * 4096, 2048, 1024, SWZ_128B), id_bf16, 0);
-          acc = 1;
+        const uint64_t d_sfk = d_sfk0 + (uint64_t)((ks * 1024) >> 4);
+        const uint64_t d_k = d_k0 + (uint64_t)((ks * 8192) >> 4);
+        const uint64_t d_delta = d_delta0 + (uint64_t)((ks * 4096) >> 4);
+        if (elect_one()) {
+          tmem_cp_32x128b_warpx4(tSFK, d_sfk);
+          tmem_cp_32x128b_warpx4(tSFK + 4, d_sfk + (512 >> 4));
+          if (has_delta) mma_bf16_ss(tS, d_ones, d_delta, id_bf16, 0);
+          mma_nvfp4_ss(tS, d_q0, d_k, id_fp4, tm + TM_SFQ, tSFK, has_delta ? 1u : 0u);
+          mma_nvfp4_ss(tS, d_q0 + (32 >> 4), d_k + (32 >> 4), id_fp4, tm + TM_SFQ + 4, tSFK + 4, 1u);
+          mma_commit(cx.bar(BAR_K_EMPTY + ks));
+          mma_commit(cx.bar(BAR_S_FULL + sb));
         }
-        for (int kc = 0; kc < 2; ++kc) {
-          mma_nvfp4_ss(tS, smem_desc(sbase + OFF_Q + 32 * kc, 16, 512, SWZ_64B),
-                       smem_desc(sbase + OFF_K + ks * 8192 + 32 * kc, 16, 512, SWZ_64B), id_fp4,
-                       tm + TM_SFQ + 4 * kc, tSFK + 4 * kc, acc);
-          acc = 1;
-        }
-        mma_commit(cx.bar(BAR_K_EMPTY + ks));
-        mma_commit(cx.bar(BAR_S_FULL + sb));
-        return true;
-      };
-      if (ok) ok = issue_qk(0);
-      for (int t = 0; t < T && ok; ++t) {
-        if (t + 1 < T) ok = issue_qk(t + 1);
-        if (!ok) break;
-        const int sb = t & 1, vs = t % VSTAGES;
-        ok = cx.wait(BAR_P_FULL + sb, (uint32_t)(t >> 1) & 1u) && cx.wait(BAR_O_READY, (uint32_t)t & 1u) &&
-             cx.wait(BAR_V_FULL + vs, (uint32_t)(t / VSTAGES) & 1u);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t tP = tm + (sb ? TM_S1 : TM_S0);
-        for (int k4 = 0; k4 < 4; ++k4)
-          mma_e4m3_ts(tm + TM_O, tP + 8 * k4, smem_desc(sbase + OFF_V + vs * 16384 + 4096 * k4, 16, 1024, SWZ_128B),
-                      id_fp8, (t > 0 || k4 > 0) ? 1u : 0u);
-        mma_commit(cx.bar(BAR_V_EMPTY + vs));
-        mma_commit(cx.bar(BAR_O_FULL));
+        TR(5, t, 5);
       }
     }
-  } else if (warp >= 4 && warp < 8) {
-    // =========================== softmax ===========================
-    const int row = (warp - 4) * 32 + lane;
+  } else if (warp == 3) {
+    // =========================== P V issuer ===========================
+    if (T > 0) {
+      const uint32_t id_fp8 = idesc_e4m3(128, 128, 0, 1);
+      const uint64_t d_v0 = smem_desc(sbase + OFF_V, 16, 1024, SWZ_128B);
+      bool ok = true;
+      for (int t = 0; t < T && ok; ++t) {
+        TR(1, t, 0);
+        const int sb = t & 1, vs = t % VSTAGES;
+        ok = cx.wait(BAR_V_FULL + vs, (uint32_t)(t / VSTAGES) & 1u);
+        TR(1, t, 1);
+        ok = ok && cx.wait(BAR_O_READY, (uint32_t)t & 1u);
+        TR(1, t, 2);
+        ok = ok && cx.wait(BAR_P_FULL + sb, (uint32_t)(t >> 1) & 1u);
+        TR(1, t, 3);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tP = tm + (sb ? TM_P1 : TM_P0);
+        const uint64_t d_v = d_v0 + (uint64_t)((vs * 16384) >> 4);
+        if (elect_one()) {
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            mma_e4m3_ts(tm + TM_O, tP + 8 * k4, d_v + (uint64_t)((4096 * k4) >> 4), id_fp8, (t > 0 || k4 > 0) ? 1u : 0u);
+          mma_commit(cx.bar(BAR_V_EMPTY + vs));
+          mma_commit(cx.bar(BAR_P_EMPTY + sb));
+          mma_commit(cx.bar(BAR_O_FULL));
+        }
+        TR(1, t, 5);
+      }
+    }
+  } else if (warp >= 4 && warp < 12) {
+    // =========================== softmax (two groups alternating over KV blocks) ===========
+    setmaxnreg_inc<168>();
+    const int grp = (warp - 4) >> 2;                 // 0: even blocks / S0, 1: odd blocks / S1
+    const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const int r_abs = row0 + row;
     const int limit = p.causal ? min(p.N_kv - 1, r_abs + off) : p.N_kv - 1;   // last visible key
     const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[b]), p.k_gscale[b]);
-    float m = -INFINITY, l = 0.0f;
+    float m_own = -INFINITY;   // running maximum after this group's previous block
+    float l_own = 0.0f;        // sum of P over this group's blocks, relative to m_own
     float *s_alpha = reinterpret_cast<float *>(smem + OFF_ALPHA);
-    bool ok = true;
-    for (int t = 0; t < T; ++t) {
-      const int sb = t & 1;
+    float *s_m = reinterpret_cast<float *>(smem + OFF_M);
+    const uint32_t tS = tm + (grp ? TM_S1 : TM_S0) + lane_off;
+    const uint32_t tP = tm + (grp ? TM_P1 : TM_P0) + lane_off;
+    for (int t = grp; t < T; t += 2) {
       const int key0 = (T - 1 - t) * TILE;
-      ok = __all_sync(0xffffffffu, cx.wait(BAR_S_FULL + sb, (uint32_t)(t >> 1) & 1u));
-      if (!ok) break;
+      TR(2 + grp, t, 0);
+      if (!__all_sync(0xffffffffu, cx.wait(BAR_S_FULL + grp, (uint32_t)(t >> 1) & 1u))) break;
+      TR(2 + grp, t, 1);
       tc_fence_after();
-      const uint32_t tS = tm + (sb ? TM_S1 : TM_S0) + lane_off;
-      const bool need_mask = key0 + TILE - 1 > limit;
-      // pass 1: row maximum (Eq. 3)
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c0 = 0; c0 < TILE; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tS + c0, r);
+      uint32_t s[128];
+      {
+        uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
+        uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
+        uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
+        uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
+        tmem_ld32(tS, s0);
+        tmem_ld32(tS + 32, s1);
+        tmem_ld32(tS + 64, s2);
+        tmem_ld32(tS + 96, s3);
         tmem_ld_wait();
-        if (need_mask) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (key0 + c0 + i > limit) r[i] = 0xFF800000u;   // -inf
-        }
-#pragma unroll
-        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
       }
-      const float m_new = fmaxf(m, mx);
-      const float alpha = (m_new == m) ? 1.0f : ex2_approx(__fmul_rn(m - m_new, lam));
-      s_alpha[sb * 128 + row] = alpha;
-      mbar_arrive(cx.bar(BAR_A_FULL + sb));
-      const float neg_mlam = (m_new == -INFINITY) ? 0.0f : -__fmul_rn(m_new, lam);
-      // pass 2: P = 2^(lam S - lam m) (Eq. 4), row sum of the unquantized P (Eq. 5),
-      // P_hat = E4M3(448 P) written over the first 32 columns of this score buffer.
+      tc_fence_before();
+      mbar_arrive(cx.bar(BAR_S_EMPTY + grp));   // the row is in registers: Q K^T of block t+2 may overwrite it
+      TR(2 + grp, t, 2);
+      if (key0 + TILE - 1 > limit) {   // diagonal / ragged block only
+#pragma unroll
+        for (int i = 0; i < 128; ++i)
+          if (key0 + i > limit) s[i] = 0xFF800000u;   // -inf
+      }
+      // row maximum (Eq. 3)
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 128; i += 8) {
+        mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+        mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+        mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+      }
+#ifdef MPFA_ABLATE_NO_MAX
+      const float mx = fmaxf(__uint_as_float(s[0]), __uint_as_float(s[127])) + 30.0f;
+#else
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+#endif
+      // running maximum: the other group owns block t-1
+      float m_prev = -INFINITY;
+#ifdef MPFA_ABLATE_NO_MHAND
+      m_prev = m_own;
+      if (false) {
+#else
+      if (t > 0) {
+#endif
+        if (!__all_sync(0xffffffffu, cx.wait(BAR_M_FULL + (grp ^ 1), (uint32_t)((t - 1) >> 1) & 1u))) break;
+        m_prev = s_m[(grp ^ 1) * 128 + row];
+      }
+      TR(2 + grp, t, 3);
+      const float m_t = fmaxf(m_prev, mx);
+      s_m[grp * 128 + row] = m_t;
+      s_alpha[grp * 128 + row] = (m_t == m_prev) ? 1.0f : ex2_approx(__fmul_rn(m_prev - m_t, lam));
+      mbar_arrive(cx.bar(BAR_M_FULL + grp));
+      TR(2 + grp, t, 4);
+      const float a_own = (m_t == m_own) ? 1.0f : ex2_approx(__fmul_rn(m_own - m_t, lam));
+      // P = 2^(lam S - lam m) (Eq. 4)
+      const float c = (m_t == -INFINITY) ? 0.0f : -__fmul_rn(m_t, lam);
+      // P V of block t-2 must have consumed this group's P_hat columns
+      if (t >= 2 && !__all_sync(0xffffffffu, cx.wait(BAR_P_EMPTY + grp, (uint32_t)((t >> 1) - 1) & 1u))) break;
       float sum0 = 0.0f, sum1 = 0.0f, sum2 = 0.0f, sum3 = 0.0f;
+#ifdef MPFA_ABLATE_NO_SOFTMAX
+      sum0 = __uint_as_float(s[5]);
+      if (false)
+#endif
 #pragma unroll
-      for (int c0 = 0; c0 < TILE; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tS + c0, r);
-        tmem_ld_wait();
-        if (need_mask) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (key0 + c0 + i > limit) r[i] = 0xFF800000u;
-        }
+      for (int c0 = 0; c0 < 128; c0 += 32) {
         uint32_t packed[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float p0 = ex2_approx(__fmaf_rn(__uint_as_float(r[4 * i]), lam, neg_mlam));
-          const float p1 = ex2_approx(__fmaf_rn(__uint_as_float(r[4 * i + 1]), lam, neg_mlam));
-          const float p2 = ex2_approx(__fmaf_rn(__uint_as_float(r[4 * i + 2]), lam, neg_mlam));
-          const float p3 = ex2_approx(__fmaf_rn(__uint_as_float(r[4 * i + 3]), lam, neg_mlam));
-          sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+#ifdef MPFA_ABLATE_NO_EXP
+#define EX2_(x) (x)
+#else
+#define EX2_(x) ex2_approx(x)
+#endif
+          const float p0 = EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i]), lam, c));
+          const float p1 = EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 1]), lam, c));
+          const float p2 = EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 2]), lam, c));
+          const float p3 = EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 3]), lam, c));
+          sum0 += p0;
+          sum1 += p1;
+          sum2 += p2;
+          sum3 += p3;
+          // 448 P is the E4M3 operand (Section 4.1)
           const uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(p0, 448.0f), __fmul_rn(p1, 448.0f)),
                                                                  __NV_SATFINITE, __NV_E4M3);
           const uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(p2, 448.0f), __fmul_rn(p3, 448.0f)),
                                                                  __NV_SATFINITE, __NV_E4M3);
           packed[i] = (lo & 0xFFFFu) | (hi << 16);
         }
-        tmem_st8(tS + (c0 >> 2), packed);
+#ifndef MPFA_ABLATE_NO_PST
+        tmem_st8(tP + (c0 >> 2), packed);
+#else
+        if (packed[0] == 0x12345u && packed[7] == 77u) tmem_st8(tP + (c0 >> 2), packed);
+#endif
       }
-      l = __fadd_rn(__fmul_rn(alpha, l), (sum0 + sum1) + (sum2 + sum3));
-      m = m_new;
+      l_own = __fadd_rn(__fmul_rn(a_own, l_own), (sum0 + sum1) + (sum2 + sum3));
+      m_own = m_t;
+      TR(2 + grp, t, 5);
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(cx.bar(BAR_P_FULL + sb));
+      mbar_arrive(cx.bar(BAR_P_FULL + grp));
+      TR(2 + grp, t, 6);
     }
-    reinterpret_cast<float *>(smem + OFF_L)[row] = l;
+    float *s_fin = reinterpret_cast<float *>(smem + OFF_L);
+    s_fin[(grp * 2 + 0) * 128 + row] = l_own;
+    s_fin[(grp * 2 + 1) * 128 + row] = m_own;
     mbar_arrive(cx.bar(BAR_L_FULL));
-  } else if (warp >= 8) {
+  } else if (warp >= 12) {
     // =========================== correction + epilogue ===========================
-    const int row = (warp - 8) * 32 + lane;
+    setmaxnreg_dec<88>();
+    const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const int r_abs = row0 + row;
     const float *s_alpha = reinterpret_cast<const float *>(smem + OFF_ALPHA);
@@ -357,14 +496,21 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     bool ok = true;
     for (int t = 0; t < T; ++t) {
       const int sb = t & 1;
-      ok = __all_sync(0xffffffffu, cx.wait(BAR_A_FULL + sb, (uint32_t)(t >> 1) & 1u));
+      TR(4, t, 0);
+      ok = __all_sync(0xffffffffu, cx.wait(BAR_M_FULL + sb, (uint32_t)(t >> 1) & 1u));
       if (!ok) break;
+      TR(4, t, 1);
       const float alpha = s_alpha[sb * 128 + row];
       if (t > 0) {
         ok = __all_sync(0xffffffffu, cx.wait(BAR_O_FULL, (uint32_t)(t - 1) & 1u));
         if (!ok) break;
+        TR(4, t, 2);
         tc_fence_after();
+#ifdef MPFA_ABLATE_NO_CORR
+        if (false) {
+#else
         if (__any_sync(0xffffffffu, alpha != 1.0f)) {   // identical result when every alpha is exactly 1
+#endif
 #pragma unroll
           for (int c0 = 0; c0 < HEAD_DIM; c0 += 32) {
             uint32_t r[32];
@@ -378,14 +524,27 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         tc_fence_before();
       }
+      TR(4, t, 3);
       mbar_arrive(cx.bar(BAR_O_READY));
     }
-    // final normalisation (Algorithm 1 line 17): O / (448 l) * v_scale -> BF16
+    // final normalisation (Algorithm 1 line 17): O / (448 l) * v_scale -> BF16.  The two softmax
+    // groups hold partial sums relative to their own last maximum; bring both to the final one.
     float l = 0.0f;
     if (T > 0 && ok) {
       ok = cx.wait(BAR_O_FULL, (uint32_t)(T - 1) & 1u) && cx.wait(BAR_L_FULL, 0);
       tc_fence_after();
-      if (ok) l = reinterpret_cast<const float *>(smem + OFF_L)[row];
+      if (ok) {
+        const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[b]), p.k_gscale[b]);
+        const float *s_fin = reinterpret_cast<const float *>(smem + OFF_L);
+        const float l0 = s_fin[0 * 128 + row], m0 = s_fin[1 * 128 + row];
+        const float l1 = s_fin[2 * 128 + row], m1 = s_fin[3 * 128 + row];
+        const float mf = fmaxf(m0, m1);
+        if (mf != -INFINITY) {
+          const float w0 = (m0 == mf) ? 1.0f : ex2_approx(__fmul_rn(m0 - mf, lam));
+          const float w1 = (m1 == mf) ? 1.0f : ex2_approx(__fmul_rn(m1 - mf, lam));
+          l = __fadd_rn(__fmul_rn(w0, l0), __fmul_rn(w1, l1));
+        }
+      }
     }
     // tcgen05.ld is warp-collective: every lane loads, only the stores are predicated.
     const bool warp_ok = __all_sync(0xffffffffu, ok);
@@ -464,6 +623,14 @@ mpfa_status make_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, uint64
 }  // namespace mpfa
 
 using namespace mpfa;
+
+#ifdef MPFA_TRACE
+extern "C" int mpfa_debug_set_trace(long long *buf, int cta) {
+  if (cudaMemcpyToSymbol(g_trace, &buf, sizeof(buf)) != cudaSuccess) return -1;
+  if (cudaMemcpyToSymbol(g_trace_cta, &cta, sizeof(cta)) != cudaSuccess) return -1;
+  return 0;
+}
+#endif
 
 extern "C" mpfa_status mpfa_prefill(const mpfa_fp4_tensor *q, const mpfa_fp4_tensor *k, const uint8_t *v_fp8,
                                     const void *delta_s_bf16, const mpfa_stats *st, float v_scale, int causal,
