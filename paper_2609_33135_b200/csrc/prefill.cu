@@ -9,8 +9,8 @@
 //                the same TMEM columns;
 //   warp 3       P V issuer: four FP8 MMAs per block (A = P_hat from TMEM, B = V from
 //                shared memory, MN-major) accumulate P V into O;
-//   warps 4-7    softmax of the even-numbered blocks of the traversal (score buffer S0);
-//   warps 8-11   softmax of the odd-numbered blocks (score buffer S1).  One thread per row:
+//   warps 4-7    softmax of the even-numbered blocks of the traversal;
+//   warps 8-11   softmax of the odd-numbered blocks.  One thread per row:
 //                the whole 128-column row is read into registers once; mask, row maximum,
 //                running maximum handed from one group to the other through shared memory
 //                (only the maximum is loop-carried, so the exponentials of block t overlap
@@ -19,11 +19,13 @@
 //                32 TMEM columns (Algorithm 1 lines 11-14).  The score buffer is handed back to
 //                the MMA warp as soon as the row is in registers, so Q K^T runs two blocks
 //                ahead of P V and a softmax group never waits for its next scores;
-//   warps 12-15  correction + epilogue: O *= alpha whenever a row's maximum moved
-//                (Eq. 6), final O / (448 l) * v_scale -> BF16.
-// Tensor memory (512 columns): S0 [0,128) S1 [128,256) O [256,384), P_hat0 [384,416)
-// P_hat1 [416,448), scale factors of Q [448,456) and of the two in-flight K blocks
-// [456,464) [464,472).
+//   warps 12-15  correction + epilogue.  Even blocks accumulate into O0, odd blocks into O1,
+//                so the rescale of an accumulator (Eq. 6, by alpha_t * alpha_{t-1}, only when
+//                some row's maximum moved) has a whole block of slack instead of sitting
+//                between two dependent MMAs; the epilogue adds the two accumulators
+//                (the older one times the last alpha) and writes O / (448 l) * v_scale as BF16.
+// Tensor memory (512 columns): S [0,128) O0 [128,256) O1 [256,384), P_hat0 [384,416)
+// P_hat1 [416,448), scale factors of Q [448,456) and of two K blocks [456,464) [464,472).
 // Register budget is moved between the roles with setmaxnreg (88 / 168 / 168 / 88).
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises MPFA_DEV_TIMEOUT in
@@ -62,20 +64,21 @@ enum {
   BAR_K_EMPTY = BAR_K_FULL + KSTAGES,
   BAR_V_FULL = BAR_K_EMPTY + KSTAGES,
   BAR_V_EMPTY = BAR_V_FULL + VSTAGES,
-  BAR_S_FULL = BAR_V_EMPTY + VSTAGES,
-  BAR_P_FULL = BAR_S_FULL + 2,
-  BAR_S_EMPTY = BAR_P_FULL + 2,  // score buffer read into registers, free for the next Q K^T
-  BAR_P_EMPTY = BAR_S_EMPTY + 2, // P V has consumed this P_hat buffer
-  BAR_M_FULL = BAR_P_EMPTY + 2,  // running maximum and alpha of block t published
-  BAR_O_FULL = BAR_M_FULL + 2,
-  BAR_O_READY = BAR_O_FULL + 1,
-  BAR_L_FULL = BAR_O_READY + 1,
+  BAR_S_FULL = BAR_V_EMPTY + VSTAGES,   // [2] scores of block t in TMEM (one buffer, one barrier per
+                                        //     softmax group so that each group's first wait is on phase 0)
+  BAR_S_EMPTY = BAR_S_FULL + 2,         // scores read into registers, buffer free for block t+1
+  BAR_P_FULL = BAR_S_EMPTY + 1,         // [2] P_hat of block t written
+  BAR_P_EMPTY = BAR_P_FULL + 2,         // [2] P V of block t has consumed P_hat
+  BAR_M_FULL = BAR_P_EMPTY + 2,         // [2] running maximum and alpha of block t published
+  BAR_O_FULL = BAR_M_FULL + 2,          // [2] P V of block t accumulated into O[t & 1]
+  BAR_O_READY = BAR_O_FULL + 2,         // [2] O[t & 1] rescaled for block t
+  BAR_L_FULL = BAR_O_READY + 2,
   NUM_BARS = BAR_L_FULL + 1
 };
 constexpr uint32_t OFF_MISC = OFF_BAR + NUM_BARS * 8;   // tmem base, abort flag
 constexpr uint32_t SMEM_BYTES = OFF_MISC + 16 + 1024;   // + slack for the 1024-byte alignment
 
-constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_O = 256, TM_P0 = 384, TM_P1 = 416, TM_SFQ = 448, TM_SFK0 = 456,
+constexpr uint32_t TM_S = 0, TM_O0 = 128, TM_O1 = 256, TM_P0 = 384, TM_P1 = 416, TM_SFQ = 448, TM_SFK0 = 456,
                    TM_SFK1 = 464;
 constexpr uint32_t TMEM_COLS = 512;
 
@@ -128,11 +131,19 @@ __device__ int g_trace_cta = 0;
 #define TR(role, t, ev) do {} while (0)
 #endif
 
+// One arrival per warp: every lane's earlier shared-memory writes and tensor-memory accesses are
+// ordered before it by the warp-level barrier.
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
+}
+
 struct Ctx {
   uint32_t bars;      // shared address of barrier 0
   volatile int *abort_flag;
   int32_t *status;
   __device__ __forceinline__ uint32_t bar(int i) const { return bars + 8u * (uint32_t)i; }
+  __device__ __forceinline__ bool probe(int i, uint32_t parity) const { return mbar_try_wait(bar(i), parity); }
   // Bounded wait.  try_wait may itself suspend the thread for a system-dependent interval, so
   // the bound is on elapsed SM clock cycles (about 2 s), checked once per 32 polls to keep the
   // hand-off latency at the cost of a poll.  Also gives up as soon as another role has failed.
@@ -181,6 +192,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const int last_key = p.causal ? min(p.N_kv - 1, last_row + off) : p.N_kv - 1;
   const int T = last_key < 0 ? 0 : last_key / TILE + 1;   // KV blocks to visit
 
+#ifdef MPFA_TRACE
+  if ((int)blockIdx.x == g_trace_cta && tid == 12 * 32 && g_trace) g_trace[((0) * 256 + 255) * 8 + 1] = clock64();   // kernel entry
+#endif
   Ctx cx;
   cx.bars = sbase + OFF_BAR;
   cx.abort_flag = reinterpret_cast<volatile int *>(smem + OFF_MISC + 4);
@@ -193,16 +207,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     mbar_init(cx.bar(BAR_Q_FULL), 1);
     for (int i = 0; i < KSTAGES; ++i) { mbar_init(cx.bar(BAR_K_FULL + i), 1); mbar_init(cx.bar(BAR_K_EMPTY + i), 1); }
     for (int i = 0; i < VSTAGES; ++i) { mbar_init(cx.bar(BAR_V_FULL + i), 1); mbar_init(cx.bar(BAR_V_EMPTY + i), 1); }
+    mbar_init(cx.bar(BAR_S_FULL), 1);
+    mbar_init(cx.bar(BAR_S_FULL + 1), 1);
+    mbar_init(cx.bar(BAR_S_EMPTY), 4);   // one arrival per warp (lane 0 after __syncwarp)
     for (int i = 0; i < 2; ++i) {
-      mbar_init(cx.bar(BAR_S_FULL + i), 1);
-      mbar_init(cx.bar(BAR_P_FULL + i), 128);
-      mbar_init(cx.bar(BAR_M_FULL + i), 128);
-      mbar_init(cx.bar(BAR_S_EMPTY + i), 128);
+      mbar_init(cx.bar(BAR_P_FULL + i), 4);
       mbar_init(cx.bar(BAR_P_EMPTY + i), 1);
+      mbar_init(cx.bar(BAR_M_FULL + i), 4);
+      mbar_init(cx.bar(BAR_O_FULL + i), 1);
+      mbar_init(cx.bar(BAR_O_READY + i), 4);
     }
-    mbar_init(cx.bar(BAR_O_FULL), 1);
-    mbar_init(cx.bar(BAR_O_READY), 128);
-    mbar_init(cx.bar(BAR_L_FULL), 256);
+    mbar_init(cx.bar(BAR_L_FULL), 8);
     mbar_init_fence();
     prefetch_tmap(&tm_q);
     prefetch_tmap(&tm_k);
@@ -226,6 +241,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
   const bool has_delta = p.delta != nullptr;
   TR_INIT();
+  if (warp == 12) TR(0, 255, 2);   // roles start (after setup)
   const size_t q_row = ((size_t)b * p.H_q + hq) * (size_t)(p.nq_tiles * TILE) + row0;
   const size_t k_row = ((size_t)b * p.H_kv + hk) * (size_t)(p.nk_tiles * TILE);
 
@@ -308,24 +324,27 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int ks = t % KSTAGES, sb = t & 1;
         TR(5, t, 0);
         ok = cx.wait(BAR_K_FULL + ks, (uint32_t)(t / KSTAGES) & 1u);
-        // the softmax group that owns this score buffer has read block t-2 out of it
-        if (ok && t >= 2) ok = cx.wait(BAR_S_EMPTY + sb, (uint32_t)((t >> 1) - 1) & 1u);
         if (!ok) break;
-        TR(5, t, 1);
-        tc_fence_after();
-        const uint32_t tS = tm + (sb ? TM_S1 : TM_S0);
         const uint32_t tSFK = tm + (sb ? TM_SFK1 : TM_SFK0);
         const uint64_t d_sfk = d_sfk0 + (uint64_t)((ks * 1024) >> 4);
         const uint64_t d_k = d_k0 + (uint64_t)((ks * 8192) >> 4);
         const uint64_t d_delta = d_delta0 + (uint64_t)((ks * 4096) >> 4);
-        if (elect_one()) {
+        tc_fence_after();
+        if (elect_one()) {   // scale factors first: their TMEM columns were last used by block t-2
           tmem_cp_32x128b_warpx4(tSFK, d_sfk);
           tmem_cp_32x128b_warpx4(tSFK + 4, d_sfk + (512 >> 4));
-          if (has_delta) mma_bf16_ss(tS, d_ones, d_delta, id_bf16, 0);
-          mma_nvfp4_ss(tS, d_q0, d_k, id_fp4, tm + TM_SFQ, tSFK, has_delta ? 1u : 0u);
-          mma_nvfp4_ss(tS, d_q0 + (32 >> 4), d_k + (32 >> 4), id_fp4, tm + TM_SFQ + 4, tSFK + 4, 1u);
-          mma_commit(cx.bar(BAR_K_EMPTY + ks));
+        }
+        // the softmax group of block t-1 has read its scores out of the buffer
+        if (t >= 1) ok = cx.wait(BAR_S_EMPTY, (uint32_t)(t - 1) & 1u);
+        if (!ok) break;
+        TR(5, t, 1);
+        tc_fence_after();
+        if (elect_one()) {
+          if (has_delta) mma_bf16_ss(tm + TM_S, d_ones, d_delta, id_bf16, 0);
+          mma_nvfp4_ss(tm + TM_S, d_q0, d_k, id_fp4, tm + TM_SFQ, tSFK, has_delta ? 1u : 0u);
+          mma_nvfp4_ss(tm + TM_S, d_q0 + (32 >> 4), d_k + (32 >> 4), id_fp4, tm + TM_SFQ + 4, tSFK + 4, 1u);
           mma_commit(cx.bar(BAR_S_FULL + sb));
+          mma_commit(cx.bar(BAR_K_EMPTY + ks));
         }
         TR(5, t, 5);
       }
@@ -341,21 +360,22 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int sb = t & 1, vs = t % VSTAGES;
         ok = cx.wait(BAR_V_FULL + vs, (uint32_t)(t / VSTAGES) & 1u);
         TR(1, t, 1);
-        ok = ok && cx.wait(BAR_O_READY, (uint32_t)t & 1u);
+        ok = ok && cx.wait(BAR_O_READY + sb, (uint32_t)(t >> 1) & 1u);
         TR(1, t, 2);
         ok = ok && cx.wait(BAR_P_FULL + sb, (uint32_t)(t >> 1) & 1u);
         TR(1, t, 3);
         if (!ok) break;
         tc_fence_after();
         const uint32_t tP = tm + (sb ? TM_P1 : TM_P0);
+        const uint32_t tOacc = tm + (sb ? TM_O1 : TM_O0);
         const uint64_t d_v = d_v0 + (uint64_t)((vs * 16384) >> 4);
         if (elect_one()) {
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
-            mma_e4m3_ts(tm + TM_O, tP + 8 * k4, d_v + (uint64_t)((4096 * k4) >> 4), id_fp8, (t > 0 || k4 > 0) ? 1u : 0u);
-          mma_commit(cx.bar(BAR_V_EMPTY + vs));
+            mma_e4m3_ts(tOacc, tP + 8 * k4, d_v + (uint64_t)((4096 * k4) >> 4), id_fp8, (t >= 2 || k4 > 0) ? 1u : 0u);
+          mma_commit(cx.bar(BAR_O_FULL + sb));
           mma_commit(cx.bar(BAR_P_EMPTY + sb));
-          mma_commit(cx.bar(BAR_O_FULL));
+          mma_commit(cx.bar(BAR_V_EMPTY + vs));
         }
         TR(1, t, 5);
       }
@@ -371,9 +391,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[b]), p.k_gscale[b]);
     float m_own = -INFINITY;   // running maximum after this group's previous block
     float l_own = 0.0f;        // sum of P over this group's blocks, relative to m_own
-    float *s_alpha = reinterpret_cast<float *>(smem + OFF_ALPHA);
     float *s_m = reinterpret_cast<float *>(smem + OFF_M);
-    const uint32_t tS = tm + (grp ? TM_S1 : TM_S0) + lane_off;
+    const uint32_t tS = tm + TM_S + lane_off;
     const uint32_t tP = tm + (grp ? TM_P1 : TM_P0) + lane_off;
     for (int t = grp; t < T; t += 2) {
       const int key0 = (T - 1 - t) * TILE;
@@ -391,10 +410,25 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         tmem_ld32(tS + 32, s1);
         tmem_ld32(tS + 64, s2);
         tmem_ld32(tS + 96, s3);
-        tmem_ld_wait();
       }
+      // While the scores are on their way: P V of block t-2 must have consumed this group's P_hat
+      // columns (this also means the correction warps have read the maximum this group published
+      // two blocks ago, so its slot may be overwritten), and the other group's maximum of block
+      // t-1 is usually already there.
+      if (t >= 2 && !__all_sync(0xffffffffu, cx.wait(BAR_P_EMPTY + grp, (uint32_t)((t >> 1) - 1) & 1u))) break;
+      float m_prev = -INFINITY;
+      bool have_prev = (t == 0);
+#ifdef MPFA_ABLATE_NO_MHAND
+      have_prev = true;
+      m_prev = m_own;
+#endif
+      if (!have_prev && __all_sync(0xffffffffu, cx.probe(BAR_M_FULL + (grp ^ 1), (uint32_t)((t - 1) >> 1) & 1u))) {
+        m_prev = s_m[(grp ^ 1) * 128 + row];
+        have_prev = true;
+      }
+      tmem_ld_wait();
       tc_fence_before();
-      mbar_arrive(cx.bar(BAR_S_EMPTY + grp));   // the row is in registers: Q K^T of block t+2 may overwrite it
+      warp_arrive(cx.bar(BAR_S_EMPTY), lane);   // the row is in registers: Q K^T of block t+1 may overwrite it
       TR(2 + grp, t, 2);
       if (key0 + TILE - 1 > limit) {   // diagonal / ragged block only
 #pragma unroll
@@ -416,27 +450,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
 #endif
       // running maximum: the other group owns block t-1
-      float m_prev = -INFINITY;
-#ifdef MPFA_ABLATE_NO_MHAND
-      m_prev = m_own;
-      if (false) {
-#else
-      if (t > 0) {
-#endif
+      if (!have_prev) {
         if (!__all_sync(0xffffffffu, cx.wait(BAR_M_FULL + (grp ^ 1), (uint32_t)((t - 1) >> 1) & 1u))) break;
         m_prev = s_m[(grp ^ 1) * 128 + row];
       }
       TR(2 + grp, t, 3);
       const float m_t = fmaxf(m_prev, mx);
       s_m[grp * 128 + row] = m_t;
-      s_alpha[grp * 128 + row] = (m_t == m_prev) ? 1.0f : ex2_approx(__fmul_rn(m_prev - m_t, lam));
-      mbar_arrive(cx.bar(BAR_M_FULL + grp));
+      warp_arrive(cx.bar(BAR_M_FULL + grp), lane);
       TR(2 + grp, t, 4);
       const float a_own = (m_t == m_own) ? 1.0f : ex2_approx(__fmul_rn(m_own - m_t, lam));
       // P = 2^(lam S - lam m) (Eq. 4)
       const float c = (m_t == -INFINITY) ? 0.0f : -__fmul_rn(m_t, lam);
-      // P V of block t-2 must have consumed this group's P_hat columns
-      if (t >= 2 && !__all_sync(0xffffffffu, cx.wait(BAR_P_EMPTY + grp, (uint32_t)((t >> 1) - 1) & 1u))) break;
       float sum0 = 0.0f, sum1 = 0.0f, sum2 = 0.0f, sum3 = 0.0f;
 #ifdef MPFA_ABLATE_NO_SOFTMAX
       sum0 = __uint_as_float(s[5]);
@@ -478,63 +503,76 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       TR(2 + grp, t, 5);
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(cx.bar(BAR_P_FULL + grp));
+      warp_arrive(cx.bar(BAR_P_FULL + grp), lane);
       TR(2 + grp, t, 6);
     }
     float *s_fin = reinterpret_cast<float *>(smem + OFF_L);
     s_fin[(grp * 2 + 0) * 128 + row] = l_own;
     s_fin[(grp * 2 + 1) * 128 + row] = m_own;
-    mbar_arrive(cx.bar(BAR_L_FULL));
+    warp_arrive(cx.bar(BAR_L_FULL), lane);
   } else if (warp >= 12) {
     // =========================== correction + epilogue ===========================
     setmaxnreg_dec<88>();
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const int r_abs = row0 + row;
-    const float *s_alpha = reinterpret_cast<const float *>(smem + OFF_ALPHA);
-    const uint32_t tO = tm + TM_O + lane_off;
+    const float *s_m = reinterpret_cast<const float *>(smem + OFF_M);
+    const uint32_t tO0 = tm + TM_O0 + lane_off, tO1 = tm + TM_O1 + lane_off;
+    const float lam_c = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[b]), p.k_gscale[b]);
     bool ok = true;
+    float alpha_prev = 1.0f, alpha = 1.0f, m_before = -INFINITY;
     for (int t = 0; t < T; ++t) {
       const int sb = t & 1;
       TR(4, t, 0);
       ok = __all_sync(0xffffffffu, cx.wait(BAR_M_FULL + sb, (uint32_t)(t >> 1) & 1u));
       if (!ok) break;
       TR(4, t, 1);
-      const float alpha = s_alpha[sb * 128 + row];
-      if (t > 0) {
-        ok = __all_sync(0xffffffffu, cx.wait(BAR_O_FULL, (uint32_t)(t - 1) & 1u));
+      // alpha_t = 2^(lam (m_{t-1} - m_t)) (Eq. 5/6), from the running maxima the softmax groups publish
+      const float m_now = s_m[sb * 128 + row];
+      alpha = (m_now == m_before) ? 1.0f : ex2_approx(__fmul_rn(m_before - m_now, lam_c));
+      m_before = m_now;
+      if (t >= 2) {
+        // O[sb] holds blocks t-2, t-4, ... relative to the maximum after block t-2
+        const float scale = __fmul_rn(alpha, alpha_prev);
+        ok = __all_sync(0xffffffffu, cx.wait(BAR_O_FULL + sb, (uint32_t)((t >> 1) - 1) & 1u));
         if (!ok) break;
         TR(4, t, 2);
         tc_fence_after();
 #ifdef MPFA_ABLATE_NO_CORR
         if (false) {
 #else
-        if (__any_sync(0xffffffffu, alpha != 1.0f)) {   // identical result when every alpha is exactly 1
+        if (__any_sync(0xffffffffu, scale != 1.0f)) {   // identical result when every factor is exactly 1
 #endif
+          const uint32_t tO = sb ? tO1 : tO0;
 #pragma unroll
           for (int c0 = 0; c0 < HEAD_DIM; c0 += 32) {
             uint32_t r[32];
             tmem_ld32(tO + c0, r);
             tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__fmul_rn(__uint_as_float(r[i]), alpha));
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__fmul_rn(__uint_as_float(r[i]), scale));
             tmem_st32(tO + c0, r);
           }
           tmem_st_wait();
         }
         tc_fence_before();
       }
+      alpha_prev = alpha;
       TR(4, t, 3);
-      mbar_arrive(cx.bar(BAR_O_READY));
+      warp_arrive(cx.bar(BAR_O_READY + sb), lane);
     }
     // final normalisation (Algorithm 1 line 17): O / (448 l) * v_scale -> BF16.  The two softmax
     // groups hold partial sums relative to their own last maximum; bring both to the final one.
-    float l = 0.0f;
+    // The accumulator of the last block is current; the other one is one alpha behind.
+    const int last = (T - 1) & 1;
+    float l = 0.0f, a_other = 0.0f;
     if (T > 0 && ok) {
-      ok = cx.wait(BAR_O_FULL, (uint32_t)(T - 1) & 1u) && cx.wait(BAR_L_FULL, 0);
+      ok = cx.wait(BAR_O_FULL + last, (uint32_t)((T - 1) >> 1) & 1u);
+      if (ok && T > 1) ok = cx.wait(BAR_O_FULL + (last ^ 1), (uint32_t)((T - 2) >> 1) & 1u);
+      ok = ok && cx.wait(BAR_L_FULL, 0);
       tc_fence_after();
       if (ok) {
-        const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[b]), p.k_gscale[b]);
+        const float lam = lam_c;
         const float *s_fin = reinterpret_cast<const float *>(smem + OFF_L);
         const float l0 = s_fin[0 * 128 + row], m0 = s_fin[1 * 128 + row];
         const float l1 = s_fin[2 * 128 + row], m1 = s_fin[3 * 128 + row];
@@ -544,31 +582,38 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           const float w1 = (m1 == mf) ? 1.0f : ex2_approx(__fmul_rn(m1 - mf, lam));
           l = __fadd_rn(__fmul_rn(w0, l0), __fmul_rn(w1, l1));
         }
+        if (T > 1) a_other = alpha;   // alpha of the last block
       }
     }
     // tcgen05.ld is warp-collective: every lane loads, only the stores are predicated.
     const bool warp_ok = __all_sync(0xffffffffu, ok);
     const bool store = r_abs < p.N_q && (warp_ok || T == 0);
     const size_t o_off = (((size_t)b * p.N_q + (store ? r_abs : 0)) * p.H_q + hq) * HEAD_DIM;
-    const float denom = __fmul_rn(448.0f, l);
-#pragma unroll
-    for (int c0 = 0; c0 < HEAD_DIM; c0 += 32) {
-      uint32_t r[32];
+    // one IEEE reciprocal per row; 128 divisions per thread would cost more than ten KV blocks
+    const float inv_denom = (l > 0.0f) ? __frcp_rn(__fmul_rn(448.0f, l)) : 0.0f;
+    const uint32_t tOl = last ? tO1 : tO0, tOo = last ? tO0 : tO1;
+#pragma unroll 1
+    for (int c0 = 0; c0 < HEAD_DIM; c0 += 16) {
+      uint32_t r[16], ro[16];
       if (T > 0 && warp_ok) {
-        tmem_ld32(tO + c0, r);
+        tmem_ld16(tOl + c0, r);
+        if (T > 1) tmem_ld16(tOo + c0, ro);
         tmem_ld_wait();
       }
 #pragma unroll
-      for (int i = 0; i < 32; ++i)
-        r[i] = (l > 0.0f) ? __float_as_uint(__fmul_rn(__fdiv_rn(__uint_as_float(r[i]), denom), p.v_scale)) : 0u;
+      for (int i = 0; i < 16; ++i) {
+        float acc = __uint_as_float(r[i]);
+        if (T > 1) acc = __fadd_rn(acc, __fmul_rn(a_other, __uint_as_float(ro[i])));
+        r[i] = (l > 0.0f) ? __float_as_uint(__fmul_rn(__fmul_rn(acc, inv_denom), p.v_scale)) : 0u;
+      }
       if (store) {
         if (p.out_f32) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 4)
+          for (int i = 0; i < 16; i += 4)
             *reinterpret_cast<uint4 *>(p.out_f32 + o_off + c0 + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
         }
 #pragma unroll
-        for (int i = 0; i < 32; i += 8) {
+        for (int i = 0; i < 16; i += 8) {
           uint32_t h[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -580,8 +625,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
     }
   }
+  if (warp == 12) TR(0, 255, 3);   // epilogue stores issued
   tc_fence_before();
   __syncthreads();
+  if (warp == 12) TR(0, 255, 4);
   if (warp == 2) tmem_dealloc(tm, TMEM_COLS);
 }
 
