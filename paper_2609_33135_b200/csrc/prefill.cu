@@ -390,7 +390,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const int limit = p.causal ? min(p.N_kv - 1, r_abs + off) : p.N_kv - 1;   // last visible key
     const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[b]), p.k_gscale[b]);
     float m_own = -INFINITY;   // running maximum after this group's previous block
-    float l_own = 0.0f;        // sum of P over this group's blocks, relative to m_own
+    float l_own = 0.0f;        // sum of 448 P over this group's blocks, relative to m_own
     float *s_m = reinterpret_cast<float *>(smem + OFF_M);
     const uint32_t tS = tm + TM_S + lane_off;
     const uint32_t tP = tm + (grp ? TM_P1 : TM_P0) + lane_off;
@@ -411,21 +411,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         tmem_ld32(tS + 64, s2);
         tmem_ld32(tS + 96, s3);
       }
-      // While the scores are on their way: P V of block t-2 must have consumed this group's P_hat
-      // columns (this also means the correction warps have read the maximum this group published
-      // two blocks ago, so its slot may be overwritten), and the other group's maximum of block
-      // t-1 is usually already there.
-      if (t >= 2 && !__all_sync(0xffffffffu, cx.wait(BAR_P_EMPTY + grp, (uint32_t)((t >> 1) - 1) & 1u))) break;
+      // While the scores are on their way, test (without blocking) the two other conditions this
+      // block needs; the answers are consumed later, so their latency overlaps the TMEM load:
+      //  - P V of block t-2 has consumed this group's P_hat columns (this also means the
+      //    correction warps have read the maximum this group published two blocks ago);
+      //  - the other group's running maximum of block t-1 is published.
+      const uint32_t par_pe = (uint32_t)((t >> 1) - 1) & 1u, par_m = (uint32_t)((t - 1) >> 1) & 1u;
+      const bool pe_early = (t < 2) || cx.probe(BAR_P_EMPTY + grp, par_pe);
+      bool have_prev = (t == 0) || cx.probe(BAR_M_FULL + (grp ^ 1), par_m);
       float m_prev = -INFINITY;
-      bool have_prev = (t == 0);
 #ifdef MPFA_ABLATE_NO_MHAND
       have_prev = true;
-      m_prev = m_own;
 #endif
-      if (!have_prev && __all_sync(0xffffffffu, cx.probe(BAR_M_FULL + (grp ^ 1), (uint32_t)((t - 1) >> 1) & 1u))) {
-        m_prev = s_m[(grp ^ 1) * 128 + row];
-        have_prev = true;
-      }
       tmem_ld_wait();
       tc_fence_before();
       warp_arrive(cx.bar(BAR_S_EMPTY), lane);   // the row is in registers: Q K^T of block t+1 may overwrite it
@@ -450,9 +447,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
 #endif
       // running maximum: the other group owns block t-1
-      if (!have_prev) {
-        if (!__all_sync(0xffffffffu, cx.wait(BAR_M_FULL + (grp ^ 1), (uint32_t)((t - 1) >> 1) & 1u))) break;
-        m_prev = s_m[(grp ^ 1) * 128 + row];
+      if (!__all_sync(0xffffffffu, have_prev)) {
+        if (!__all_sync(0xffffffffu, cx.wait(BAR_M_FULL + (grp ^ 1), par_m))) break;
+      }
+      if (t > 0) m_prev = s_m[(grp ^ 1) * 128 + row];
+#ifdef MPFA_ABLATE_NO_MHAND
+      m_prev = m_own;
+#endif
+      if (!__all_sync(0xffffffffu, pe_early)) {
+        if (!__all_sync(0xffffffffu, cx.wait(BAR_P_EMPTY + grp, par_pe))) break;
       }
       TR(2 + grp, t, 3);
       const float m_t = fmaxf(m_prev, mx);
@@ -477,19 +480,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #else
 #define EX2_(x) ex2_approx(x)
 #endif
-          const float p0 = EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i]), lam, c));
-          const float p1 = EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 1]), lam, c));
-          const float p2 = EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 2]), lam, c));
-          const float p3 = EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 3]), lam, c));
-          sum0 += p0;
-          sum1 += p1;
-          sum2 += p2;
-          sum3 += p3;
-          // 448 P is the E4M3 operand (Section 4.1)
-          const uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(p0, 448.0f), __fmul_rn(p1, 448.0f)),
-                                                                 __NV_SATFINITE, __NV_E4M3);
-          const uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(p2, 448.0f), __fmul_rn(p3, 448.0f)),
-                                                                 __NV_SATFINITE, __NV_E4M3);
+          // q = 448 P is the E4M3 operand (Section 4.1); the row sum is taken over q and the
+          // factor 448 is divided out once in the epilogue
+          const float q0 = __fmul_rn(EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i]), lam, c)), 448.0f);
+          const float q1 = __fmul_rn(EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 1]), lam, c)), 448.0f);
+          const float q2 = __fmul_rn(EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 2]), lam, c)), 448.0f);
+          const float q3 = __fmul_rn(EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 3]), lam, c)), 448.0f);
+          sum0 += q0;
+          sum1 += q1;
+          sum2 += q2;
+          sum3 += q3;
+          const uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q0, q1), __NV_SATFINITE, __NV_E4M3);
+          const uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q2, q3), __NV_SATFINITE, __NV_E4M3);
           packed[i] = (lo & 0xFFFFu) | (hi << 16);
         }
 #ifndef MPFA_ABLATE_NO_PST
@@ -590,7 +592,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const bool store = r_abs < p.N_q && (warp_ok || T == 0);
     const size_t o_off = (((size_t)b * p.N_q + (store ? r_abs : 0)) * p.H_q + hq) * HEAD_DIM;
     // one IEEE reciprocal per row; 128 divisions per thread would cost more than ten KV blocks
-    const float inv_denom = (l > 0.0f) ? __frcp_rn(__fmul_rn(448.0f, l)) : 0.0f;
+    const float inv_denom = (l > 0.0f) ? __frcp_rn(l) : 0.0f;   // l already carries the factor 448
     const uint32_t tOl = last ? tO1 : tO0, tOo = last ? tO0 : tO1;
 #pragma unroll 1
     for (int c0 = 0; c0 < HEAD_DIM; c0 += 16) {
