@@ -306,8 +306,8 @@ def run_ours(args, rank, world, local):
 
 
 # DRAM bytes per prefill launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum);
-# filled in from profiles/ once captured, keyed by sequence length.
-NCU_TRAFFIC_BYTES = {}
+# from profiles/prefill_kernel_llama_shape.md (65,090,304 read + 81,254,400 written), keyed by sequence length.
+NCU_TRAFFIC_BYTES = {16384: 146344704}
 
 
 def main():
@@ -320,7 +320,7 @@ def main():
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--small-decode", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--cpu-rows-per-head", type=int, default=2048)
+    ap.add_argument("--cpu-rows-per-head", type=int, default=8192)
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args, int(os.environ.get("RANK", 0)))
