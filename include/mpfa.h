@@ -38,7 +38,7 @@
  *   Delta_S  BF16 [B, H_q, N_kv_pad], in units of (true logit) / (q_gscale * k_gscale).
  *   V        E4M3 [B, H_kv, N_kv_pad, 128], pad rows zero.
  *   Paged KV cache (mpfa_paged_kv): 64-token pages; within a page and kv head the bytes are
- *     ordered for the decode kernel's register fragments, see mpfa_paged_kv below.
+ *     ordered as the decode kernel's shared-memory operand tiles, see mpfa_paged_kv below.
  */
 #ifndef MPFA_H_
 #define MPFA_H_
@@ -96,15 +96,16 @@ typedef struct {
 } mpfa_fp4_tensor;
 
 /* Paged KV cache for decode: num_pages physical pages of 64 tokens, shared by all
- * requests through a page table.  Inside a (page, kv head) slab the bytes are ordered so
- * that every 16-byte load of the decode kernel is one thread's tensor-core fragment.
- * With token t (0..63) of the page:
+ * requests through a page table.  Inside a (page, kv head) slab the bytes are ordered as the
+ * decode kernel's shared-memory operand tiles (rows of 8 tokens, 16-byte chunks XOR-swizzled
+ * by the row), so that one bulk copy per slab fills a tile.  With token t (0..63) of the page:
  *   k_codes [P, H_kv, 4096]  byte j (0..7) of 16-channel block g (0..7) of token t at
- *             (t/8)*512 + ((t%8)*4 + j/2)*16 + g*2 + (j%2)
+ *             (t/8)*512 + (t%8)*64 + ((g/2) ^ ((t%8)/2))*16 + (g%2)*8 + j
  *   k_sf    [P, H_kv, 512]   block g of token t at t*8 + g
- *   v_fp8   [P, H_kv, 8192]  channel c (0..127) of token t, with u = t%32, at
- *             (t/32)*4096 + (c/16)*512 + ((c%8)*4 + (u%8)/2)*16 + ((c/8)%2)*8 + (u/16)*4 + ((u/8)%2)*2 + (u%2)
+ *   v_fp8   [P, H_kv, 8192]  channel c (0..127) of token t at
+ *             (t/8)*1024 + (t%8)*128 + ((c/16) ^ (t%8))*16 + c%16
  *   delta_s [P, H_q, 64]     BF16, token t at index t (NULL when compensation is off)
+ * Tokens of a page beyond the sequence length hold zeros (mpfa_quantize_kv_paged writes them).
  * mpfa_paged_k_offset / mpfa_paged_v_offset are these maps.  All pools 256-byte aligned. */
 typedef struct {
   uint8_t *k_codes;

@@ -31,13 +31,13 @@ extern "C" size_t mpfa_sf_offset(int H, int N, int b, int h, int token, int bloc
 }
 
 extern "C" size_t mpfa_paged_k_offset(int token, int block, int byte_in_block) {
-  return (size_t)(token / 8) * 512 + ((token % 8) * 4 + byte_in_block / 2) * 16 + block * 2 + (byte_in_block % 2);
+  const int r = token % 8;
+  return (size_t)(token / 8) * 512 + r * 64 + (((block / 2) ^ (r / 2)) * 16) + (block % 2) * 8 + byte_in_block;
 }
 
 extern "C" size_t mpfa_paged_v_offset(int token, int channel) {
-  const int u = token % 32, c = channel;
-  return (size_t)(token / 32) * 4096 + (c / 16) * 512 + ((c % 8) * 4 + (u % 8) / 2) * 16 + ((c / 8) % 2) * 8 +
-         (u / 16) * 4 + ((u / 8) % 2) * 2 + (u % 2);
+  const int r = token % 8;
+  return (size_t)(token / 8) * 1024 + r * 128 + (((channel / 16) ^ r) * 16) + channel % 16;
 }
 
 extern "C" const char *mpfa_status_string(mpfa_status s) {

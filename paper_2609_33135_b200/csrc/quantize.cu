@@ -268,8 +268,8 @@ __global__ void __launch_bounds__(256) quantize_v_tile_kernel(const __nv_bfloat1
 }
 
 // Paged cache write for one request: grid (pages, H_kv).  K and V of one (page, head) are
-// quantized into shared memory in the decode kernel's fragment order and copied out with
-// 16-byte stores.
+// quantized into shared memory in the byte order of the decode kernel's shared-memory operand
+// tiles (so that decode fills a tile with one bulk copy) and copied out with 16-byte stores.
 __global__ void __launch_bounds__(256) quantize_kv_page_kernel(const __nv_bfloat16 *__restrict__ k,
                                                                const __nv_bfloat16 *__restrict__ v,
                                                                const float *__restrict__ k_mean,
@@ -302,24 +302,12 @@ __global__ void __launch_bounds__(256) quantize_kv_page_kernel(const __nv_bfloat
       quantize_block16(xc, d, sc, c);
       vc = quantize_v16(v + ((size_t)tok * H_kv + h) * HEAD_DIM + g * 16, inv_vscale);
     }
-    // K: byte j of block g of token t at (t/8)*512 + ((t%8)*4 + j/2)*16 + g*2 + (j%2)
-    const uint32_t cw[2] = {c.x, c.y};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint16_t two = (uint16_t)(cw[q >> 1] >> (16 * (q & 1)));
-      *reinterpret_cast<uint16_t *>(sk + (t >> 3) * 512 + ((t & 7) * 4 + q) * 16 + g * 2) = two;
-    }
+    // K: the 8 code bytes of block g of token t, in the 64-byte-swizzled row order the decode
+    // kernel's tensor-core descriptor reads: (t/8)*512 + (t%8)*64 + ((g/2) ^ ((t%8)/2))*16 + (g%2)*8
+    *reinterpret_cast<uint2 *>(sk + (t >> 3) * 512 + (t & 7) * 64 + (((g >> 1) ^ ((t & 7) >> 1)) << 4) + (g & 1) * 8) = c;
     ssf[t * 8 + g] = sc;
-    // V: channel c of token t (u = t%32) at
-    // (t/32)*4096 + (c/16)*512 + ((c%8)*4 + (u%8)/2)*16 + ((c/8)%2)*8 + (u/16)*4 + ((u/8)%2)*2 + (u%2)
-    const uint32_t vw[4] = {vc.x, vc.y, vc.z, vc.w};
-    const int u = t & 31;
-    const int tbase = (t >> 5) * 4096 + g * 512 + ((u & 7) >> 1) * 16 + (u >> 4) * 4 + ((u >> 3) & 1) * 2 + (u & 1);
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int ch = i;  // channel inside the 16-channel segment g
-      sv[tbase + (ch & 7) * 64 + (ch >> 3) * 8] = (uint8_t)(vw[i >> 2] >> (8 * (i & 3)));
-    }
+    // V: channels 16g..16g+15 of token t, 128-byte-swizzled: (t/8)*1024 + (t%8)*128 + (g ^ (t%8))*16
+    *reinterpret_cast<uint4 *>(sv + (t >> 3) * 1024 + (t & 7) * 128 + ((g ^ (t & 7)) << 4)) = vc;
   }
   __syncthreads();
   const size_t slab = (size_t)page * H_kv + h;

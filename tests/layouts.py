@@ -26,13 +26,13 @@ def sf_to_logical(sf: np.ndarray, B, H, N) -> np.ndarray:
 
 
 def paged_k_offset(t, g, j):
-    return (t // 8) * 512 + ((t % 8) * 4 + j // 2) * 16 + g * 2 + (j % 2)
+    r = t % 8
+    return (t // 8) * 512 + r * 64 + ((g // 2) ^ (r // 2)) * 16 + (g % 2) * 8 + j
 
 
 def paged_v_offset(t, c):
-    u = t % 32
-    return ((t // 32) * 4096 + (c // 16) * 512 + ((c % 8) * 4 + (u % 8) // 2) * 16 + ((c // 8) % 2) * 8 +
-            (u // 16) * 4 + ((u // 8) % 2) * 2 + (u % 2))
+    r = t % 8
+    return (t // 8) * 1024 + r * 128 + ((c // 16) ^ r) * 16 + c % 16
 
 
 def paged_k_to_logical(slab: np.ndarray) -> np.ndarray:
