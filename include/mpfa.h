@@ -104,7 +104,8 @@ typedef struct {
  *   k_sf    [P, H_kv, 512]   block g of token t at t*8 + g
  *   v_fp8   [P, H_kv, 8192]  channel c (0..127) of token t at
  *             (t/8)*1024 + (t%8)*128 + ((c/16) ^ (t%8))*16 + c%16
- *   delta_s [P, H_q, 64]     BF16, token t at index t (NULL when compensation is off)
+ *   delta_s [P, H_q, 64]     BF16, token t of q head h at index ((t/8) ^ (h % (H_q/H_kv)))*8 + t%8
+ *                            (NULL when compensation is off)
  * Tokens of a page beyond the sequence length hold zeros (mpfa_quantize_kv_paged writes them).
  * mpfa_paged_k_offset / mpfa_paged_v_offset are these maps.  All pools 256-byte aligned. */
 typedef struct {

@@ -2,28 +2,35 @@
 //
 // The path is bound by streaming the cache from HBM (208 bytes per token and kv head plus
 // Delta_S), so the kernel is a persistent streaming pipeline: one CTA per SM walks a list of
-// (request, kv head, 1024-token partition) work items, and a producer warp keeps a ring of
-// 128-key blocks (two 64-token pages: K codes, K scales, V, Delta_S) in flight with bulk
-// asynchronous copies, across item boundaries.  The cache's physical byte order
+// (request, kv head, 1024-token partition) work items, and a producer warp keeps two rings of
+// 128-key blocks in flight with bulk asynchronous copies: a K ring (codes, block scales,
+// Delta_S) that runs one item AHEAD of a V ring.  The cache's physical byte order
 // (include/mpfa.h) is the swizzled shared-memory image the tensor-core descriptors read, so a
 // page needs one copy per tensor and no thread touches the bytes.
 //
 // The problem is transposed so that the long axis is the MMA's M dimension and the GQA group
 // (Section 5.3 packs it into one MMA tile) is the N dimension, padded to 16:
 //   S^T[key, head] = K Q^T       tcgen05.mma kind::mxf4nvf4 (E2M1 codes, UE4M3 block scales),
-//                                M = 128 keys, N = 16, K = 2 x 64 channels, FP32 in TMEM;
-//   softmax        one thread per key: + Delta_S (Eq. 10), running maximum of the reverse
-//                  traversal (blocks 7..0 of the partition), P = 2^(lam S - lam m),
-//                  P_hat = E4M3(448 P) written to shared memory as the next MMA's B operand;
-//   O^T[ch, head] += V^T P_hat^T  tcgen05.mma kind::f8f6f4, M = 128 channels, N = 16,
-//                                K = 4 x 32 keys, V read MN-major straight from the ring.
-// When the running maximum grows, O^T is rescaled in TMEM (one row of 16 floats per thread).
-// The partition state (m, l, O) goes to the workspace; a second kernel merges partitions by
-// log-sum-exp (warp-shuffle maximum, partitions ascending) and writes BF16.
+//                                M = 128 keys, N = 16, K = 2 x 64 channels, FP32 in TMEM,
+//                                one 16-column slot per block of the item;
+//   softmax        one thread per key.  As each S^T lands: + Delta_S (Eq. 10), warp maximum.
+//                  After the item's last block one exchange gives every block u the running
+//                  maximum m_u of the reverse traversal (max over the blocks visited so far),
+//                  then P = 2^(lam S - lam m_u), P_hat = E4M3(448 P) for all blocks at once,
+//                  written to shared memory as the B operands of the PV MMAs;
+//   O_u^T[ch, head] = V_u^T P_hat_u^T   tcgen05.mma kind::f8f6f4, M = 128 channels, N = 16,
+//                                K = 4 x 32 keys, V read MN-major straight from the ring, one
+//                                accumulator slot per block.
+// Because the scores of an item are finished while the previous item's V is still streaming,
+// a V block is consumed the moment it lands, and the softmax never sits on the critical path.
+// The sequential rescaling O <- 2^(lam (m_old - m_new)) O + P_hat V becomes
+// O = sum_u 2^(lam (m_u - m)) O_u at the end of the item (one thread per channel), the same
+// sum with the factors multiplied out.  The partition state (m, l, O) goes to the workspace; a
+// second kernel merges partitions by log-sum-exp and writes BF16.
 //
-// Warps: 0 producer, 1 MMA issue (+ TMEM allocation), 2-5 softmax / rescale / partition
-// write-out (TMEM lane quadrant = warp % 4), 6 rewrites the K scales of each block from
-// [token][8] into the 32 x 16-byte tile tcgen05.cp expects.  Every wait is bounded.
+// Warps: 0 producer, 1 QK issue (+ TMEM allocation), 2 PV issue, 3 rewrites the K scales of
+// each block from [token][8] into the 32 x 16-byte tiles tcgen05.cp expects, 4-7 softmax and
+// partition write-out (TMEM lane quadrant = warp % 4).  Every wait is bounded.
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
 
@@ -36,50 +43,62 @@ namespace {
 constexpr int PART_FLOATS = 130;  // m, l, O[128] per (request, q head, partition)
 constexpr int MAXG = 8;
 constexpr int NCOL = 16;          // MMA N: the GQA group padded to 16 columns
+constexpr int MAXBLK = DECODE_SPLIT / TILE;   // 8 blocks per item
 
-constexpr int D_NST = 7;          // KV ring stages, one 128-key block each
-constexpr int D_NSF = 4;          // formatted K-scale tiles in flight
-constexpr int D_THREADS = 224;
+constexpr int D_NK = 4;           // K ring stages
+constexpr int D_NV = 8;           // V ring stages
+constexpr int D_THREADS = 256;
 
-// one ring stage
-constexpr uint32_t ST_K = 0;          // 2 pages x 4096 B of codes: 64-byte rows, 64-byte swizzle
-constexpr uint32_t ST_V = 8192;       // 2 pages x 8192 B: 128-byte rows, 128-byte swizzle
-constexpr uint32_t ST_SF = 24576;     // 2 pages x 512 B of K scales, [token][8]
-constexpr uint32_t ST_DELTA = 25600;  // 2 pages x MAXG x 128 B of Delta_S (BF16)
-constexpr uint32_t ST_BYTES = 27648;
-// the rest of shared memory
-constexpr uint32_t D_OFF_P = D_NST * ST_BYTES;      // 2 x 2048: P_hat^T, 16 rows of 128 keys, 128-byte swizzle
-constexpr uint32_t D_OFF_Q = D_OFF_P + 4096;        // 2 x 1024: Q codes, 16 rows of 64 B, 64-byte swizzle
-constexpr uint32_t D_OFF_SFQ = D_OFF_Q + 2048;      // 2 x (2 x 512): Q scales, one tile per 64 channels
-constexpr uint32_t D_OFF_SFK = D_OFF_SFQ + 2048;    // D_NSF x (2 x 512): K scales
-constexpr uint32_t D_OFF_BAR = D_OFF_SFK + D_NSF * 1024;
-constexpr uint32_t D_OFF_X = D_OFF_BAR + 512;       // block maxima, l partial sums, TMEM address, abort flag
-constexpr uint32_t D_SMEM_USED = D_OFF_X + 1024;
+// one K stage
+constexpr uint32_t KST_K = 0;          // 2 pages x 4096 B of codes: 64-byte rows, 64-byte swizzle
+constexpr uint32_t KST_SF = 8192;      // 2 pages x 512 B of K scales, [token][8]
+constexpr uint32_t KST_DELTA = 9216;   // 2 pages x 8 rows x 128 B of Delta_S (BF16, 128-byte swizzle; rows G..7 stay zero)
+constexpr uint32_t KST_BYTES = 11264;
+constexpr uint32_t VST_BYTES = 16384;  // 2 pages x 8192 B: 128-byte rows, 128-byte swizzle
+constexpr uint32_t D_OFF_K = 0;
+constexpr uint32_t D_OFF_V = D_OFF_K + D_NK * KST_BYTES;
+constexpr uint32_t D_OFF_P = D_OFF_V + D_NV * VST_BYTES;   // [2 items][8 blocks] x 2048: P_hat^T, 16 rows of 128 keys
+constexpr uint32_t D_OFF_Q = D_OFF_P + 2 * MAXBLK * 2048;  // 2 x 1024: Q codes, 16 rows of 64 B, 64-byte swizzle
+constexpr uint32_t D_OFF_SFQ = D_OFF_Q + 2048;             // 2 x (2 x 512): Q scales, one tile per 64 channels
+constexpr uint32_t D_OFF_SFK = D_OFF_SFQ + 2048;           // D_NK x (2 x 512): K scales
+constexpr uint32_t D_OFF_ZERO = D_OFF_SFK + D_NK * 1024;    // 2048 B of zeros: the second K group of the Delta_S operand
+constexpr uint32_t D_OFF_IDENT = D_OFF_ZERO + 2048;        // 16 x 16 BF16 identity, MN-major, 128-byte swizzle
+constexpr uint32_t D_OFF_BAR = D_OFF_IDENT + 2048;
+constexpr uint32_t D_OFF_XMAX = D_OFF_BAR + 512;           // [2][8 blocks][MAXG][4 warps] floats
+constexpr uint32_t D_OFF_WTAB = D_OFF_XMAX + 2 * MAXBLK * MAXG * 16;   // [2][8 blocks][MAXG] floats
+constexpr uint32_t D_OFF_MFIN = D_OFF_WTAB + 2 * MAXBLK * MAXG * 4;    // [2][MAXG]
+constexpr uint32_t D_OFF_XL = D_OFF_MFIN + 2 * MAXG * 4;               // [2][4 warps][MAXG]
+constexpr uint32_t D_OFF_MISC = D_OFF_XL + 2 * 4 * MAXG * 4;           // TMEM address, abort flag
+constexpr int D_MAXREQ = 768;                                          // requests whose length / lambda are cached
+constexpr uint32_t D_OFF_LEN = D_OFF_MISC + 64;                        // [D_MAXREQ] int32
+constexpr uint32_t D_OFF_LAM = D_OFF_LEN + D_MAXREQ * 4;               // [D_MAXREQ] float
+constexpr uint32_t D_SMEM_USED = D_OFF_LAM + D_MAXREQ * 4;
 constexpr uint32_t D_SMEM = D_SMEM_USED + 1024;     // slack for the 1024-byte alignment of the base
 
 // barriers (8 bytes each)
-constexpr int B_FULL = 0;                    // [D_NST] stage landed (bytes)
-constexpr int B_EMPTY = B_FULL + D_NST;      // [D_NST] stage consumed (MMA commit)
-constexpr int B_SF_READY = B_EMPTY + D_NST;  // [D_NSF] K scales formatted
-constexpr int B_SFK_FREE = B_SF_READY + D_NSF;  // [D_NSF] scale tile consumed (MMA commit)
-constexpr int B_S_FULL = B_SFK_FREE + D_NSF;    // [2]
-constexpr int B_S_EMPTY = B_S_FULL + 2;         // [2] 4 warps
-constexpr int B_P_READY = B_S_EMPTY + 2;        // [2] 4 warps
-constexpr int B_PV_DONE = B_P_READY + 2;        // [2] MMA commit
-constexpr int B_Q_READY = B_PV_DONE + 2;        // [2] 4 warps
-constexpr int B_O_FREE = B_Q_READY + 2;         // [1] 4 warps
-constexpr int B_XCHG = B_O_FREE + 1;            // [1] 4 warps: block maxima written
-constexpr int B_LX = B_XCHG + 1;                // [1] 4 warps: l partial sums written
-constexpr int B_COUNT = B_LX + 1;
+constexpr int B_K_FULL = 0;                      // [D_NK] K stage landed (bytes)
+constexpr int B_K_EMPTY = B_K_FULL + D_NK;       // [D_NK] QK commit
+constexpr int B_V_FULL = B_K_EMPTY + D_NK;       // [D_NV]
+constexpr int B_V_EMPTY = B_V_FULL + D_NV;       // [D_NV] PV commit
+constexpr int B_SF_READY = B_V_EMPTY + D_NV;     // [D_NK] K scales formatted
+constexpr int B_S_FULL = B_SF_READY + D_NK;      // [2][8] QK commit
+constexpr int B_S_FREE = B_S_FULL + 2 * MAXBLK;  // [2] 4 warps: the item's scores have been read
+constexpr int B_P_READY = B_S_FREE + 2;          // [2] 4 warps
+constexpr int B_Q_READY = B_P_READY + 2;         // [2] scale warp
+constexpr int B_O_FULL = B_Q_READY + 2;          // [1] PV commit after the item's last block
+constexpr int B_O_FREE = B_O_FULL + 1;           // [1] 4 warps
+constexpr int B_XCHG = B_O_FREE + 1;             // [1] 4 warps
+constexpr int B_COUNT = B_XCHG + 1;
 static_assert(B_COUNT * 8 <= 512, "barrier block");
 static_assert(D_SMEM <= 232448, "shared memory");
+static_assert(KST_BYTES % 1024 == 0 && D_OFF_V % 1024 == 0 && D_OFF_P % 1024 == 0, "swizzle atoms");
 
 // tensor-memory columns
-constexpr uint32_t TM_S = 0;      // 2 x 16
-constexpr uint32_t TM_O = 32;     // 16
-constexpr uint32_t TM_SFQ = 48;   // 2 x 8
-constexpr uint32_t TM_SFK = 64;   // D_NSF x 8
-constexpr uint32_t TM_COLS = 128;
+constexpr uint32_t TM_S = 0;       // [2 items][8 blocks] x 16
+constexpr uint32_t TM_O = 256;     // [8 blocks] x 16
+constexpr uint32_t TM_SFQ = 384;   // 2 x 8
+constexpr uint32_t TM_SFK = 400;   // D_NK x 8
+constexpr uint32_t TM_COLS = 512;
 
 constexpr long long D_WAIT_CYCLES = 4000000000ll;   // about two seconds
 
@@ -89,8 +108,35 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// The first G (1..8) TMEM columns at `taddr` of this thread's lane; the load width is the next power of two.
+template <int G>
+__device__ __forceinline__ void tmem_ld_g(uint32_t taddr, uint32_t (&r)[G]) {
+  static_assert(G >= 1 && G <= 8, "group size");
+  if constexpr (G == 1) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r[0]) : "r"(taddr) : "memory");
+  } else if constexpr (G == 2) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(taddr) : "memory");
+  } else if constexpr (G <= 4) {
+    uint32_t x[4];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
+                 : "r"(taddr)
+                 : "memory");
+#pragma unroll
+    for (int g = 0; g < G; ++g) r[g] = x[g];
+  } else {
+    uint32_t x[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3]), "=r"(x[4]), "=r"(x[5]), "=r"(x[6]), "=r"(x[7])
+                 : "r"(taddr)
+                 : "memory");
+#pragma unroll
+    for (int g = 0; g < G; ++g) r[g] = x[g];
+  }
+}
+
 #ifdef MPFA_TRACE
-// clock64 stamps of CTA g_dtrace_cta: [block counter < 256][16 events]
+// clock64 stamps of CTA g_dtrace_cta: [counter < 256][16 events]
 __device__ long long *g_dtrace = nullptr;
 __device__ int g_dtrace_cta = 0;
 #define DTR(ev, blk)                                                                              \
@@ -121,7 +167,9 @@ struct DecodeParams {
 struct WorkIter {
   int idx, stride, total, n_split, H_kv;
   int b, hk, sp, L, nblk;
-  __device__ void init(const DecodeParams &p) {
+  const int32_t *len_tab;   // shared-memory copy of seq_lens (first D_MAXREQ requests)
+  __device__ void init(const DecodeParams &p, const int32_t *tab) {
+    len_tab = tab;
     stride = gridDim.x;
     idx = (int)blockIdx.x - stride;
     n_split = p.n_split;
@@ -136,7 +184,7 @@ struct WorkIter {
       const int r = idx / n_split;
       hk = r % H_kv;
       b = r / H_kv;
-      L = seq_lens[b];
+      L = b < D_MAXREQ ? len_tab[b] : seq_lens[b];
       const int rem = L - sp * DECODE_SPLIT;
       if (rem > 0) {
         nblk = (min(rem, DECODE_SPLIT) + TILE - 1) / TILE;
@@ -157,8 +205,8 @@ struct DCtx {
     if (mbar_try_wait(a, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t n = 1;; ++n) {
-      if (mbar_try_wait(a, parity)) return true;
-      if ((n & 1023u) == 0u) {
+      if (mbar_try_wait_hint(a, parity, 2000u)) return true;   // the hardware may park the thread meanwhile
+      if ((n & 255u) == 0u) {
         if (*abort_flag) return false;
         if (clock64() - t0 > D_WAIT_CYCLES) {
           *abort_flag = 1;
@@ -178,44 +226,78 @@ struct DCtx {
   }
 };
 
+// Page ids of the blocks of one item, lane l holding block l's two pages (-1 = not there).
+__device__ __forceinline__ void lookup_pages(const DecodeParams &p, const WorkIter &w, int lane, int &pid0, int &pid1) {
+  pid0 = -1, pid1 = -1;
+  bool bad = false;
+  if (lane < w.nblk) {
+    const int first = w.sp * DECODE_SPLIT + lane * TILE;
+    const int pg = first / PAGE;
+    const int32_t *row = p.page_table + (size_t)w.b * p.max_pages;
+    if (pg < p.max_pages) pid0 = row[pg];
+    if (pid0 < 0 || pid0 >= p.num_pages) pid0 = -1, bad = true;
+    if (first + PAGE < w.L) {
+      if (pg + 1 < p.max_pages) pid1 = row[pg + 1];
+      if (pid1 < 0 || pid1 >= p.num_pages) pid1 = -1, bad = true;
+    }
+  }
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(p.status, MPFA_DEV_BAD_PAGE);
+}
+
+template <int G>
 __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const DecodeParams p) {
   extern __shared__ uint8_t dsm_raw[];
   uint8_t *dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(dsm);
-  float *xmax = reinterpret_cast<float *>(dsm + D_OFF_X);            // [2][4][MAXG]
-  float *xl = reinterpret_cast<float *>(dsm + D_OFF_X + 256);        // [2][4][MAXG]
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(dsm + D_OFF_X + 512);
-  volatile int *abort_flag = reinterpret_cast<volatile int *>(dsm + D_OFF_X + 516);
+  float *xmax = reinterpret_cast<float *>(dsm + D_OFF_XMAX);
+  float *wtab = reinterpret_cast<float *>(dsm + D_OFF_WTAB);
+  float *mfin = reinterpret_cast<float *>(dsm + D_OFF_MFIN);
+  float *xl = reinterpret_cast<float *>(dsm + D_OFF_XL);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(dsm + D_OFF_MISC);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(dsm + D_OFF_MISC + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int G = p.H_q / p.H_kv;
   DCtx cx{sbase + D_OFF_BAR, abort_flag, p.status};
 
   // ---- set-up: barriers, zeroed operand tiles (rows G..15 stay zero for good), TMEM
   if (threadIdx.x == 0) {
-    for (int i = 0; i < D_NST; ++i) {
-      mbar_init(cx.bar(B_FULL + i), 1);
-      mbar_init(cx.bar(B_EMPTY + i), 1);
-    }
-    for (int i = 0; i < D_NSF; ++i) {
+    for (int i = 0; i < D_NK; ++i) {
+      mbar_init(cx.bar(B_K_FULL + i), 1);
+      mbar_init(cx.bar(B_K_EMPTY + i), 1);
       mbar_init(cx.bar(B_SF_READY + i), 1);
-      mbar_init(cx.bar(B_SFK_FREE + i), 1);
     }
+    for (int i = 0; i < D_NV; ++i) {
+      mbar_init(cx.bar(B_V_FULL + i), 1);
+      mbar_init(cx.bar(B_V_EMPTY + i), 1);
+    }
+    for (int i = 0; i < 2 * MAXBLK; ++i) mbar_init(cx.bar(B_S_FULL + i), 1);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(cx.bar(B_S_FULL + i), 1);
-      mbar_init(cx.bar(B_S_EMPTY + i), 4);
+      mbar_init(cx.bar(B_S_FREE + i), 4);
       mbar_init(cx.bar(B_P_READY + i), 4);
-      mbar_init(cx.bar(B_PV_DONE + i), 1);
-      mbar_init(cx.bar(B_Q_READY + i), 4);
+      mbar_init(cx.bar(B_Q_READY + i), 1);
     }
+    mbar_init(cx.bar(B_O_FULL), 1);
     mbar_init(cx.bar(B_O_FREE), 4);
     mbar_init(cx.bar(B_XCHG), 4);
-    mbar_init(cx.bar(B_LX), 4);
     mbar_init_fence();
     *abort_flag = 0;
   }
-  for (uint32_t o = threadIdx.x * 16; o < 8192; o += D_THREADS * 16)   // P, Q and Q-scale tiles
+  // zeroed once: the K ring (Delta_S rows G..7 are never written), P, Q and scale tiles, zero and identity blocks
+  for (uint32_t o = threadIdx.x * 16; o < D_NK * KST_BYTES; o += D_THREADS * 16)
+    *reinterpret_cast<uint4 *>(dsm + D_OFF_K + o) = make_uint4(0u, 0u, 0u, 0u);
+  for (uint32_t o = threadIdx.x * 16; o < D_OFF_BAR - D_OFF_P; o += D_THREADS * 16)
     *reinterpret_cast<uint4 *>(dsm + D_OFF_P + o) = make_uint4(0u, 0u, 0u, 0u);
+  int32_t *len_tab = reinterpret_cast<int32_t *>(dsm + D_OFF_LEN);
+  float *lam_tab = reinterpret_cast<float *>(dsm + D_OFF_LAM);
+  for (int i = threadIdx.x; i < min(p.B, D_MAXREQ); i += D_THREADS) {
+    len_tab[i] = p.seq_lens[i];
+    lam_tab[i] = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[i]), p.k_gscale[i]);
+  }
+  __syncthreads();
+  if (threadIdx.x < 16) {   // identity[n][k]: element (n, k) at (k/8)*1024 + (k%8)*128 + ((n/8) ^ (k%8))*16 + (n%8)*2
+    const int k = threadIdx.x;
+    *reinterpret_cast<uint16_t *>(dsm + D_OFF_IDENT + (k >> 3) * 1024 + (k & 7) * 128 + (((k >> 3) ^ (k & 7)) << 4) + (k & 7) * 2) = 0x3F80;
+  }
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_slot), TM_COLS);
     tmem_relinquish();
@@ -227,345 +309,423 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
   const uint32_t tm = *tmem_slot;
 
   if (warp == 0) {
-    // ================= producer: page lookups and bulk copies
-    WorkIter w;
-    w.init(p);
-    uint32_t it = 0;
+    // ================= producer: the K walk runs one item ahead of the V walk
+    WorkIter wk, wv;
+    wk.init(p, len_tab);
+    wv.init(p, len_tab);
+    uint32_t kc = 0, vc = 0;
     bool ok = true;
     const uint32_t d_bytes = p.delta ? (uint32_t)G * PAGE * 2 : 0u;
-    const uint32_t page_bytes = 4096u + 8192u + 512u + d_bytes;
-    while (ok && w.next(p.seq_lens)) {
-      const int k_part = w.sp * DECODE_SPLIT;
-      // lane l holds the two page ids of block l of this partition
-      int pid0 = -1, pid1 = -1;
-      bool bad = false;
-      if (lane < w.nblk) {
-        const int first = k_part + lane * TILE;
-        const int pg = first / PAGE;
-        const int32_t *row = p.page_table + (size_t)w.b * p.max_pages;
-        if (pg < p.max_pages) pid0 = row[pg];
-        if (pid0 < 0 || pid0 >= p.num_pages) pid0 = -1, bad = true;
-        if (first + PAGE < w.L) {
-          if (pg + 1 < p.max_pages) pid1 = row[pg + 1];
-          if (pid1 < 0 || pid1 >= p.num_pages) pid1 = -1, bad = true;
+    const uint32_t kpage_bytes = 4096u + 512u + d_bytes;
+    int pk0 = -1, pk1 = -1, pv0 = -1, pv1 = -1;
+    auto issue_k = [&](const WorkIter &w, int t) {
+      const uint32_t st = kc % D_NK;
+      if (kc >= (uint32_t)D_NK && !cx.wait_warp(B_K_EMPTY + st, ((kc / D_NK) - 1) & 1)) {
+        ok = false;
+        return;
+      }
+      DTR(0, kc);
+      const int u = w.nblk - 1 - t;
+      const int id0 = __shfl_sync(0xffffffffu, pk0, u), id1 = __shfl_sync(0xffffffffu, pk1, u);
+      if (elect_one()) {
+        const uint32_t full = cx.bar(B_K_FULL + st);
+        const uint32_t sdst = sbase + D_OFF_K + st * KST_BYTES;
+        mbar_expect_tx(full, (id0 >= 0 ? kpage_bytes : 0u) + (id1 >= 0 ? kpage_bytes : 0u));
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int id = half == 0 ? id0 : id1;
+          if (id < 0) continue;
+          const size_t slab = (size_t)id * p.H_kv + w.hk;
+          bulk_load(sdst + KST_K + half * 4096, p.k_codes + slab * 4096, 4096, full);
+          bulk_load(sdst + KST_SF + half * 512, p.k_sf + slab * 512, 512, full);
+          if (d_bytes)
+            bulk_load(sdst + KST_DELTA + half * 1024, p.delta + ((size_t)id * p.H_q + (size_t)w.hk * G) * PAGE, d_bytes, full);
         }
       }
-      if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(p.status, MPFA_DEV_BAD_PAGE);
-      for (int u = w.nblk - 1; u >= 0; --u, ++it) {
-        const uint32_t st = it % D_NST;
-        if (it >= (uint32_t)D_NST && !cx.wait_warp(B_EMPTY + st, ((it / D_NST) - 1) & 1)) {
-          ok = false;
-          break;
-        }
-        DTR(0, it);
-        const int id0 = __shfl_sync(0xffffffffu, pid0, u), id1 = __shfl_sync(0xffffffffu, pid1, u);
-        uint8_t *stage = dsm + st * ST_BYTES;
-        // a page that is not there contributes P_hat = 0 times V: V must be finite, so zero it
-        if (id0 < 0 || id1 < 0) {
+      __syncwarp();
+      ++kc;
+    };
+    auto issue_v = [&](const WorkIter &w, int t) {
+      const uint32_t st = vc % D_NV;
+      if (vc >= (uint32_t)D_NV && !cx.wait_warp(B_V_EMPTY + st, ((vc / D_NV) - 1) & 1)) {
+        ok = false;
+        return;
+      }
+      DTR(1, vc);
+      const int u = w.nblk - 1 - t;
+      const int id0 = __shfl_sync(0xffffffffu, pv0, u), id1 = __shfl_sync(0xffffffffu, pv1, u);
+      uint8_t *stage = dsm + D_OFF_V + st * VST_BYTES;
+      // a page that is not there contributes P_hat = 0 times V: V must be finite, so zero it
+      if (id0 < 0 || id1 < 0) {
 #pragma unroll 1
-          for (int half = 0; half < 2; ++half) {
-            if ((half == 0 ? id0 : id1) >= 0) continue;
-            for (int i = 0; i < 16; ++i)
-              *reinterpret_cast<uint4 *>(stage + ST_V + half * 8192 + i * 512 + lane * 16) = make_uint4(0u, 0u, 0u, 0u);
-          }
-          fence_proxy_async_smem();
-          __syncwarp();
+        for (int half = 0; half < 2; ++half) {
+          if ((half == 0 ? id0 : id1) >= 0) continue;
+          for (int i = 0; i < 16; ++i)
+            *reinterpret_cast<uint4 *>(stage + half * 8192 + i * 512 + lane * 16) = make_uint4(0u, 0u, 0u, 0u);
         }
-        if (elect_one()) {
-          const uint32_t full = cx.bar(B_FULL + st);
-          const uint32_t sdst = sbase + st * ST_BYTES;
-          mbar_expect_tx(full, (id0 >= 0 ? page_bytes : 0u) + (id1 >= 0 ? page_bytes : 0u));
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const int id = half == 0 ? id0 : id1;
-            if (id < 0) continue;
-            const size_t slab = (size_t)id * p.H_kv + w.hk;
-            bulk_load(sdst + ST_K + half * 4096, p.k_codes + slab * 4096, 4096, full);
-            bulk_load(sdst + ST_V + half * 8192, p.v_fp8 + slab * 8192, 8192, full);
-            bulk_load(sdst + ST_SF + half * 512, p.k_sf + slab * 512, 512, full);
-            if (d_bytes)
-              bulk_load(sdst + ST_DELTA + half * 1024, p.delta + ((size_t)id * p.H_q + (size_t)w.hk * G) * PAGE, d_bytes,
-                        full);
-          }
-        }
+        fence_proxy_async_smem();
         __syncwarp();
       }
+      if (elect_one()) {
+        const uint32_t full = cx.bar(B_V_FULL + st);
+        const uint32_t sdst = sbase + D_OFF_V + st * VST_BYTES;
+        mbar_expect_tx(full, (id0 >= 0 ? 8192u : 0u) + (id1 >= 0 ? 8192u : 0u));
+        if (id0 >= 0) bulk_load(sdst, p.v_fp8 + ((size_t)id0 * p.H_kv + w.hk) * 8192, 8192, full);
+        if (id1 >= 0) bulk_load(sdst + 8192, p.v_fp8 + ((size_t)id1 * p.H_kv + w.hk) * 8192, 8192, full);
+      }
+      __syncwarp();
+      ++vc;
+    };
+    // page ids are looked up one item before the K walk needs them (pn: the item after wk's)
+    WorkIter wl;
+    wl.init(p, len_tab);
+    int pn0 = -1, pn1 = -1;
+    bool vk = wk.next(p.seq_lens);
+    bool vl = wl.next(p.seq_lens);
+    if (vk) {
+      lookup_pages(p, wk, lane, pk0, pk1);
+      vl = wl.next(p.seq_lens);
+      if (vl) lookup_pages(p, wl, lane, pn0, pn1);
+      for (int t = 0; ok && t < wk.nblk; ++t) issue_k(wk, t);
+    }
+    bool vv = wv.next(p.seq_lens);
+    while (ok && vv) {
+      pv0 = pk0, pv1 = pk1;   // wv now stands where wk stood
+      vk = wk.next(p.seq_lens);
+      if (vk) {
+        pk0 = pn0, pk1 = pn1;
+        vl = wl.next(p.seq_lens);
+        if (vl) lookup_pages(p, wl, lane, pn0, pn1);
+      }
+      const int nk = vk ? wk.nblk : 0, nv = wv.nblk;
+      for (int t = 0; ok && t < max(nk, nv); ++t) {
+        if (t < nk) issue_k(wk, t);
+        if (ok && t < nv) issue_v(wv, t);
+      }
+      vv = wv.next(p.seq_lens);
     }
     if (!ok) {
       // another role gave up: let the copies already issued land before shared memory goes away
-      const uint32_t n = it < (uint32_t)D_NST ? it : (uint32_t)D_NST;
-      for (uint32_t i = it - n; i < it; ++i) {
+      for (uint32_t i = kc - min(kc, (uint32_t)D_NK); i < kc; ++i) {
         const long long t0 = clock64();
-        while (!mbar_try_wait(cx.bar(B_FULL + i % D_NST), (i / D_NST) & 1) && clock64() - t0 < D_WAIT_CYCLES) {
+        while (!mbar_try_wait(cx.bar(B_K_FULL + i % D_NK), (i / D_NK) & 1) && clock64() - t0 < D_WAIT_CYCLES) {
+        }
+      }
+      for (uint32_t i = vc - min(vc, (uint32_t)D_NV); i < vc; ++i) {
+        const long long t0 = clock64();
+        while (!mbar_try_wait(cx.bar(B_V_FULL + i % D_NV), (i / D_NV) & 1) && clock64() - t0 < D_WAIT_CYCLES) {
         }
       }
     }
   } else if (warp == 1) {
-    // ================= MMA issue: S^T = K Q^T one block ahead of O^T += V^T P_hat^T
+    // ================= QK issue: S^T[item parity][block] = K Q^T as K stages land
     const uint32_t id_qk = idesc_nvfp4(128, NCOL);
-    const uint32_t id_pv = idesc_e4m3(128, NCOL, 1, 0);
-    WorkIter wa, wc;   // block being scored, block being accumulated
-    wa.init(p);
-    wc.init(p);
-    bool va = wa.next(p.seq_lens), vc = wc.next(p.seq_lens);
-    int ua = va ? wa.nblk - 1 : 0, uc = vc ? wc.nblk - 1 : 0;
-    uint32_t ia = 0, ic = 0, ja = 0, jc = 0;   // block and item counters of the two walks
-    bool ok = true;
-    auto issue_qk = [&]() {
-      const uint32_t st = ia % D_NST, sf = ia % D_NSF, sb = ia & 1, qs = ja & 1;
-      const bool first = ua == wa.nblk - 1;
-      ok = cx.wait_warp(B_FULL + st, (ia / D_NST) & 1);
-      DTR(1, ia);
-      ok = ok && cx.wait_warp(B_SF_READY + sf, (ia / D_NSF) & 1);
-      if (ok && first) ok = cx.wait_warp(B_Q_READY + qs, (ja >> 1) & 1);
-      if (ok && ia >= 2) ok = cx.wait_warp(B_S_EMPTY + sb, ((ia >> 1) - 1) & 1);
-      if (!ok) return;
-      DTR(2, ia);
-      tc_fence_after();
-      if (elect_one()) {
-        const uint32_t tSFQ = tm + TM_SFQ + qs * 8, tSFK = tm + TM_SFK + sf * 8;
-        if (first) {
-          const uint64_t d_sfq = smem_desc(sbase + D_OFF_SFQ + qs * 1024, 0, 128, SWZ_NONE);
-          tmem_cp_32x128b_warpx4(tSFQ, d_sfq);
-          tmem_cp_32x128b_warpx4(tSFQ + 4, d_sfq + (512 >> 4));
-        }
-        const uint64_t d_sfk = smem_desc(sbase + D_OFF_SFK + sf * 1024, 0, 128, SWZ_NONE);
-        tmem_cp_32x128b_warpx4(tSFK, d_sfk);
-        tmem_cp_32x128b_warpx4(tSFK + 4, d_sfk + (512 >> 4));
-        const uint64_t d_k = smem_desc(sbase + st * ST_BYTES + ST_K, 16, 512, SWZ_64B);
-        const uint64_t d_q = smem_desc(sbase + D_OFF_Q + qs * 1024, 16, 512, SWZ_64B);
-        mma_nvfp4_ss(tm + TM_S + sb * 16, d_k, d_q, id_qk, tSFK, tSFQ, 0u);
-        mma_nvfp4_ss(tm + TM_S + sb * 16, d_k + (32 >> 4), d_q + (32 >> 4), id_qk, tSFK + 4, tSFQ + 4, 1u);
-        mma_commit(cx.bar(B_S_FULL + sb));
-        mma_commit(cx.bar(B_SFK_FREE + sf));
-      }
-      __syncwarp();
-      DTR(3, ia);
-      ++ia;
-      if (--ua < 0) {
-        ++ja;
-        va = wa.next(p.seq_lens);
-        ua = va ? wa.nblk - 1 : 0;
-      }
-    };
-    if (va) issue_qk();
-    while (ok && vc) {
-      if (va) issue_qk();
-      if (!ok) break;
-      const uint32_t st = ic % D_NST, sb = ic & 1;
-      const bool first = uc == wc.nblk - 1;
-      ok = cx.wait_warp(B_P_READY + sb, (ic >> 1) & 1);
-      if (ok && first && jc >= 1) ok = cx.wait_warp(B_O_FREE, (jc - 1) & 1);   // the previous item's O has been read
-      if (!ok) break;
-      DTR(4, ic);
-      tc_fence_after();
-      if (elect_one()) {
-        const uint64_t d_v = smem_desc(sbase + st * ST_BYTES + ST_V, 16, 1024, SWZ_128B);
-        const uint64_t d_p = smem_desc(sbase + D_OFF_P + sb * 2048, 16, 1024, SWZ_128B);
-#pragma unroll
-        for (int k4 = 0; k4 < 4; ++k4)   // 32 keys per MMA
-          mma_e4m3_ss(tm + TM_O, d_v + (uint64_t)((4096 * k4) >> 4), d_p + (uint64_t)((32 * k4) >> 4), id_pv,
-                      (!first || k4 > 0) ? 1u : 0u);
-        mma_commit(cx.bar(B_PV_DONE + sb));
-        mma_commit(cx.bar(B_EMPTY + st));
-      }
-      __syncwarp();
-      DTR(5, ic);
-      ++ic;
-      if (--uc < 0) {
-        ++jc;
-        vc = wc.next(p.seq_lens);
-        uc = vc ? wc.nblk - 1 : 0;
-      }
-    }
-  } else if (warp == 6) {
-    // ================= K scales of a block: [token][8 blocks] -> two 32 x 16-byte tiles
-    // (tile h = blocks 4h..4h+3; row i holds tokens i, 32+i, 64+i, 96+i), the form tcgen05.cp spreads
+    const uint32_t id_ds = idesc_bf16(128, NCOL, 1, 1);
+    const uint64_t d_ident = smem_desc(sbase + D_OFF_IDENT, 2048, 1024, SWZ_128B);
+    const bool has_delta = p.delta != nullptr;
     WorkIter w;
-    w.init(p);
-    uint32_t it = 0;
+    w.init(p, len_tab);
+    uint32_t kc = 0, j = 0;
     bool ok = true;
     while (ok && w.next(p.seq_lens)) {
-      for (int u = w.nblk - 1; u >= 0; --u, ++it) {
-        const uint32_t st = it % D_NST, sf = it % D_NSF;
-        ok = cx.wait_warp(B_FULL + st, (it / D_NST) & 1);
-        if (ok && it >= (uint32_t)D_NSF) ok = cx.wait_warp(B_SFK_FREE + sf, ((it / D_NSF) - 1) & 1);
+      const uint32_t par = j & 1;
+      ok = cx.wait_warp(B_Q_READY + par, (j >> 1) & 1);
+      if (ok && j >= 2) ok = cx.wait_warp(B_S_FREE + par, ((j >> 1) - 1) & 1);   // scores of item j-2 have been read
+      for (int t = 0; ok && t < w.nblk; ++t, ++kc) {
+        const uint32_t st = kc % D_NK;
+        ok = cx.wait_warp(B_K_FULL + st, (kc / D_NK) & 1) && cx.wait_warp(B_SF_READY + st, (kc / D_NK) & 1);
         if (!ok) break;
-        const uint8_t *raw = dsm + st * ST_BYTES + ST_SF;
-        uint2 v[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) v[q] = *reinterpret_cast<const uint2 *>(raw + (q >> 1) * 512 + ((q & 1) * 32 + lane) * 8);
-        uint8_t *dst = dsm + D_OFF_SFK + sf * 1024 + lane * 16;
-        *reinterpret_cast<uint4 *>(dst) = make_uint4(v[0].x, v[1].x, v[2].x, v[3].x);
-        *reinterpret_cast<uint4 *>(dst + 512) = make_uint4(v[0].y, v[1].y, v[2].y, v[3].y);
-        fence_proxy_async_smem();
-        cx.warp_arrive(B_SF_READY + sf);
-        DTR(6, it);
+        DTR(2, kc);
+        tc_fence_after();
+        if (elect_one()) {
+          const uint32_t tSFQ = tm + TM_SFQ + par * 8, tSFK = tm + TM_SFK + st * 8;
+          if (t == 0) {
+            const uint64_t d_sfq = smem_desc(sbase + D_OFF_SFQ + par * 1024, 0, 128, SWZ_NONE);
+            tmem_cp_32x128b_warpx4(tSFQ, d_sfq);
+            tmem_cp_32x128b_warpx4(tSFQ + 4, d_sfq + (512 >> 4));
+          }
+          const uint64_t d_sfk = smem_desc(sbase + D_OFF_SFK + st * 1024, 0, 128, SWZ_NONE);
+          tmem_cp_32x128b_warpx4(tSFK, d_sfk);
+          tmem_cp_32x128b_warpx4(tSFK + 4, d_sfk + (512 >> 4));
+          const uint64_t d_k = smem_desc(sbase + D_OFF_K + st * KST_BYTES + KST_K, 16, 512, SWZ_64B);
+          const uint64_t d_q = smem_desc(sbase + D_OFF_Q + par * 1024, 16, 512, SWZ_64B);
+          const uint32_t tS = tm + TM_S + (par * MAXBLK + t) * 16;
+          if (has_delta) {
+            // S^T = Delta_S^T I (Eq. 10 seed): A = the stage's Delta_S rows, MN-major (keys contiguous), its
+            // second group of eight K rows read from the zero block; B = identity
+            const uint32_t a_ds = sbase + D_OFF_K + st * KST_BYTES + KST_DELTA;
+            mma_bf16_ss(tS, smem_desc(a_ds, 1024, sbase + D_OFF_ZERO - a_ds, SWZ_128B), d_ident, id_ds, 0u);
+          }
+          mma_nvfp4_ss(tS, d_k, d_q, id_qk, tSFK, tSFQ, has_delta ? 1u : 0u);
+          mma_nvfp4_ss(tS, d_k + (32 >> 4), d_q + (32 >> 4), id_qk, tSFK + 4, tSFQ + 4, 1u);
+          mma_commit(cx.bar(B_S_FULL + par * MAXBLK + t));
+          mma_commit(cx.bar(B_K_EMPTY + st));
+        }
+        __syncwarp();
+        DTR(3, kc);
       }
+      // the slots this item does not use complete a phase as well: a barrier's phase is then a function of the item
+      if (ok && w.nblk < MAXBLK && elect_one())
+        for (int t = w.nblk; t < MAXBLK; ++t) mma_commit(cx.bar(B_S_FULL + par * MAXBLK + t));   // after the MMAs above
+      __syncwarp();
+      ++j;
     }
-  } else {
-    // ================= softmax, one thread per key of the block (per channel for O^T)
-    const int quad = warp & 3;                  // TMEM lane quadrant this warp may touch
-    const int r = quad * 32 + lane;             // key within the block / channel of O^T
-    const int t128 = (warp - 2) * 32 + lane;    // 0..127 among these warps
-    const uint32_t tlane = (uint32_t)(quad * 32) << 16;
-    WorkIter w, wn;   // current item, next item (its query tile is staged one item ahead)
-    w.init(p);
-    wn.init(p);
-    bool vn = wn.next(p.seq_lens);
-    auto stage_q = [&](const WorkIter &x, uint32_t slot) {
-      if (t128 < G * 4) {
-        const int n = t128 >> 2, c = t128 & 3;
-        const uint4 v = *reinterpret_cast<const uint4 *>(p.q_codes + ((size_t)x.b * p.H_q + x.hk * G + n) * (TILE * 64) + c * 16);
-        *reinterpret_cast<uint4 *>(dsm + D_OFF_Q + slot * 1024 + n * 64 + ((c ^ ((n & 7) >> 1)) << 4)) = v;
+  } else if (warp == 2) {
+    // ================= PV issue: O_u^T = V_u^T P_hat_u^T as V stages land
+    const uint32_t id_pv = idesc_e4m3(128, NCOL, 1, 0);
+    WorkIter w;
+    w.init(p, len_tab);
+    uint32_t vc = 0, j = 0;
+    bool ok = true;
+    while (ok && w.next(p.seq_lens)) {
+      const uint32_t par = j & 1;
+      ok = cx.wait_warp(B_P_READY + par, (j >> 1) & 1);
+      if (ok && j >= 1) ok = cx.wait_warp(B_O_FREE, (j - 1) & 1);   // the previous item's O has been read
+      for (int t = 0; ok && t < w.nblk; ++t, ++vc) {
+        const uint32_t st = vc % D_NV;
+        ok = cx.wait_warp(B_V_FULL + st, (vc / D_NV) & 1);
+        if (!ok) break;
+        DTR(4, vc);
+        tc_fence_after();
+        if (elect_one()) {
+          const uint64_t d_v = smem_desc(sbase + D_OFF_V + st * VST_BYTES, 16, 1024, SWZ_128B);
+          const uint64_t d_p = smem_desc(sbase + D_OFF_P + (par * MAXBLK + t) * 2048, 16, 1024, SWZ_128B);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)   // 32 keys per MMA
+            mma_e4m3_ss(tm + TM_O + t * 16, d_v + (uint64_t)((4096 * k4) >> 4), d_p + (uint64_t)((32 * k4) >> 4), id_pv,
+                        k4 > 0 ? 1u : 0u);
+          mma_commit(cx.bar(B_V_EMPTY + st));
+          if (t == w.nblk - 1) mma_commit(cx.bar(B_O_FULL));
+        }
+        __syncwarp();
+        DTR(5, vc);
       }
-      if (t128 < G) {
-        const uint8_t *src = p.q_sf + ((size_t)x.b * p.H_q + x.hk * G + t128) * 1024;
-        uint8_t *dst = dsm + D_OFF_SFQ + slot * 1024 + t128 * 16;
-        *reinterpret_cast<uint32_t *>(dst) = *reinterpret_cast<const uint32_t *>(src);
-        *reinterpret_cast<uint32_t *>(dst + 512) = *reinterpret_cast<const uint32_t *>(src + 512);
+      ++j;
+    }
+  } else if (warp == 3) {
+    // ================= K scales of a block: [token][8 blocks] -> two 32 x 16-byte tiles
+    // (tile h = blocks 4h..4h+3; row i holds tokens i, 32+i, 64+i, 96+i), the form tcgen05.cp spreads.
+    // The tile of stage st is free: the copy into the stage waited for the MMAs that read it.
+    // The same warp stages the query tile (codes and scales of the group's G heads) of item j+1 while
+    // item j is scored: that slot was last read by the MMAs of item j-1.
+    WorkIter w, wq;
+    w.init(p, len_tab);
+    wq.init(p, len_tab);
+    uint32_t kc = 0, j = 0, n_staged = 0;
+    bool ok = true;
+    uint4 qv = make_uint4(0u, 0u, 0u, 0u);
+    uint32_t qs0 = 0, qs1 = 0;
+    bool have_q = false;
+    auto load_q = [&]() {   // global loads of the next item's tile, consumed one item later
+      have_q = wq.next(p.seq_lens);
+      if (!have_q) return;
+      if (lane < G * 4)
+        qv = *reinterpret_cast<const uint4 *>(p.q_codes + ((size_t)wq.b * p.H_q + wq.hk * G + (lane >> 2)) * (TILE * 64) + (lane & 3) * 16);
+      if (lane < G) {
+        const uint8_t *src = p.q_sf + ((size_t)wq.b * p.H_q + wq.hk * G + lane) * 1024;
+        qs0 = *reinterpret_cast<const uint32_t *>(src);
+        qs1 = *reinterpret_cast<const uint32_t *>(src + 512);
+      }
+    };
+    auto store_q = [&]() {
+      if (!have_q) return;
+      const uint32_t slot = n_staged & 1;
+      if (lane < G * 4) {
+        const int n = lane >> 2, c = lane & 3;
+        *reinterpret_cast<uint4 *>(dsm + D_OFF_Q + slot * 1024 + n * 64 + ((c ^ ((n & 7) >> 1)) << 4)) = qv;
+      }
+      if (lane < G) {
+        uint8_t *dst = dsm + D_OFF_SFQ + slot * 1024 + lane * 16;
+        *reinterpret_cast<uint32_t *>(dst) = qs0;
+        *reinterpret_cast<uint32_t *>(dst + 512) = qs1;
       }
       fence_proxy_async_smem();
       cx.warp_arrive(B_Q_READY + slot);
+      ++n_staged;
     };
-    if (vn) stage_q(wn, 0);
-    uint32_t it = 0, j = 0;
-    bool ok = true;
+    load_q();
+    store_q();
+    load_q();
+    store_q();
+    load_q();
     while (ok && w.next(p.seq_lens)) {
-      vn = wn.next(p.seq_lens);
-      if (vn) stage_q(wn, (j + 1) & 1);
-      const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[w.b]), p.k_gscale[w.b]);
-      const int k_part = w.sp * DECODE_SPLIT;
-      float m_run[MAXG], l_r[MAXG];
-#pragma unroll
-      for (int g = 0; g < MAXG; ++g) m_run[g] = -INFINITY, l_r[g] = 0.0f;
-      for (int u = w.nblk - 1; u >= 0; --u, ++it) {
-        const uint32_t st = it % D_NST, sb = it & 1;
-        ok = cx.wait_warp(B_S_FULL + sb, (it >> 1) & 1) && cx.wait_warp(B_FULL + st, (it / D_NST) & 1);
+      if (j >= 1) {
+        // all QK MMAs of item j-1 are complete once its last block's scores are
+        const uint32_t pj = j - 1;
+        ok = cx.wait_warp(B_S_FULL + (pj & 1) * MAXBLK + MAXBLK - 1, (pj >> 1) & 1);
         if (!ok) break;
-        if (warp == 2) DTR(7, it);
-        tc_fence_after();
-        uint32_t sraw[16];
-        tmem_ld16(tm + TM_S + sb * 16 + tlane, sraw);
-        tmem_ld_wait();
-        tc_fence_before();
-        cx.warp_arrive(B_S_EMPTY + sb);
-        // ---- scores of this key for the G heads, block maximum
-        const bool valid = k_part + u * TILE + r < w.L;
-        const uint8_t *dptr = dsm + st * ST_BYTES + ST_DELTA + (r >> 6) * 1024 + (r & 63) * 2;
-        float sv[MAXG];
-#pragma unroll
-        for (int g = 0; g < MAXG; ++g) {
-          sv[g] = -INFINITY;
-          if (g < G && valid) {
-            const float dl = p.delta ? __uint_as_float((uint32_t)*reinterpret_cast<const uint16_t *>(dptr + g * 128) << 16) : 0.0f;
-            sv[g] = __fadd_rn(__uint_as_float(sraw[g]), dl);
-          }
-          if (g < G) {
-            float wm = sv[g];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
-            if (lane == 0) xmax[(sb * 4 + (warp - 2)) * MAXG + g] = wm;
-          }
-        }
-        if (warp == 2) DTR(8, it);
-        cx.warp_arrive(B_XCHG);
-        ok = cx.wait_warp(B_XCHG, it & 1);
-        if (!ok) break;
-        if (warp == 2) DTR(9, it);
-        float alpha[MAXG];
-        bool rescale = false;
-        uint32_t pbytes[MAXG / 2];
-#pragma unroll
-        for (int g = 0; g < MAXG; g += 2) {
-          float pq[2];
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int gg = g + e;
-            float bm = -INFINITY;
-            if (gg < G) {
-#pragma unroll
-              for (int q = 0; q < 4; ++q) bm = fmaxf(bm, xmax[(sb * 4 + q) * MAXG + gg]);
-            }
-            const float m_new = fmaxf(m_run[gg], bm);
-            alpha[gg] = (m_run[gg] == -INFINITY) ? 1.0f : ex2_approx(__fmul_rn(m_run[gg] - m_new, lam));
-            rescale |= (gg < G) && (alpha[gg] != 1.0f);
-            const float pv = (gg < G && valid) ? ex2_approx(__fmaf_rn(sv[gg], lam, -__fmul_rn(m_new, lam))) : 0.0f;
-            l_r[gg] = __fmaf_rn(l_r[gg], alpha[gg], pv);
-            pq[e] = __fmul_rn(pv, 448.0f);
-            m_run[gg] = m_new;
-          }
-          pbytes[g >> 1] = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(pq[0], pq[1]), __NV_SATFINITE, __NV_E4M3);
-        }
-        // ---- P_hat^T into the B tile of this block's PV MMAs (free once PV of block it-2 is done)
-        if (warp == 2) DTR(10, it);
-        if (it >= 2) ok = cx.wait_warp(B_PV_DONE + sb, ((it >> 1) - 1) & 1);
-        if (!ok) break;
-        if (warp == 2) DTR(11, it);
-        {
-          uint8_t *pt = dsm + D_OFF_P + sb * 2048 + (r & 15);
-#pragma unroll
-          for (int g = 0; g < MAXG; ++g)
-            if (g < G) pt[(g & 7) * 128 + (((r >> 4) ^ (g & 7)) << 4)] = (uint8_t)(pbytes[g >> 1] >> (8 * (g & 1)));
-        }
-        // ---- the running maximum grew: rescale O^T (needs the previous block's PV to be complete)
-        if (u != w.nblk - 1 && rescale) {
-          ok = cx.wait_warp(B_PV_DONE + ((it - 1) & 1), ((it - 1) >> 1) & 1);
-          if (!ok) break;
-          tc_fence_after();
-          uint32_t o[16];
-          tmem_ld16(tm + TM_O + tlane, o);
-          tmem_ld_wait();
-#pragma unroll
-          for (int g = 0; g < MAXG; ++g) o[g] = __float_as_uint(__fmul_rn(__uint_as_float(o[g]), alpha[g]));
-          tmem_st16(tm + TM_O + tlane, o);
-          tmem_st_wait();
-          tc_fence_before();
-        }
-        if (warp == 2) DTR(12, it);
-        fence_proxy_async_smem();
-        cx.warp_arrive(B_P_READY + sb);
-        if (warp == 2) DTR(13, it);
-      }
-      if (!ok) break;
-      // ---- partition state: O^T row of this thread's channel, l summed over the keys
-      {
-        const uint32_t last = it - 1;
-        ok = cx.wait_warp(B_PV_DONE + (last & 1), (last >> 1) & 1);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t o[16];
-        tmem_ld16(tm + TM_O + tlane, o);
-        tmem_ld_wait();
-        tc_fence_before();
-        cx.warp_arrive(B_O_FREE);
-        float *dst = p.parts + (((size_t)w.b * p.H_q + (size_t)w.hk * G) * p.n_split + w.sp) * PART_FLOATS;
-        const size_t head_stride = (size_t)p.n_split * PART_FLOATS;
-#pragma unroll
-        for (int g = 0; g < MAXG; ++g) {
-          if (g < G) {
-            dst[g * head_stride + 2 + r] = __uint_as_float(o[g]);
-            float ls = l_r[g];
-#pragma unroll
-            for (int o2 = 16; o2 > 0; o2 >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o2);
-            if (lane == 0) xl[((j & 1) * 4 + (warp - 2)) * MAXG + g] = ls;
-          }
-        }
-        cx.warp_arrive(B_LX);
-        ok = cx.wait_warp(B_LX, j & 1);
-        if (!ok) break;
-#pragma unroll
-        for (int g = 0; g < MAXG; ++g) {
-          if (t128 == g && g < G) {
-            float l = 0.0f;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) l += xl[((j & 1) * 4 + q) * MAXG + g];
-            dst[g * head_stride] = m_run[g];
-            dst[g * head_stride + 1] = l;
-          }
-        }
+        store_q();
+        load_q();
       }
       ++j;
+      for (int t = 0; t < w.nblk; ++t, ++kc) {
+        const uint32_t st = kc % D_NK;
+        ok = cx.wait_warp(B_K_FULL + st, (kc / D_NK) & 1);
+        if (!ok) break;
+        const uint8_t *raw = dsm + D_OFF_K + st * KST_BYTES + KST_SF;
+        uint2 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) v[q] = *reinterpret_cast<const uint2 *>(raw + (q >> 1) * 512 + ((q & 1) * 32 + lane) * 8);
+        uint8_t *dst = dsm + D_OFF_SFK + st * 1024 + lane * 16;
+        *reinterpret_cast<uint4 *>(dst) = make_uint4(v[0].x, v[1].x, v[2].x, v[3].x);
+        *reinterpret_cast<uint4 *>(dst + 512) = make_uint4(v[0].y, v[1].y, v[2].y, v[3].y);
+        fence_proxy_async_smem();
+        cx.warp_arrive(B_SF_READY + st);
+        DTR(6, kc);
+      }
+    }
+  } else {
+    // ================= softmax, one thread per key of a block (per channel for O^T)
+    const int quad = warp & 3;                  // TMEM lane quadrant this warp may touch
+    const int r = quad * 32 + lane;             // key within the block / channel of O^T
+    const int t128 = (warp - 4) * 32 + lane;    // 0..127 among these warps
+    const uint32_t tlane = (uint32_t)(quad * 32) << 16;
+    bool ok = true;
+
+    // partition write-out of the item before the current one (its PV MMAs finish meanwhile)
+    struct Prev { int b, hk, sp, nblk; };
+    auto write_out = [&](const Prev &pr, uint32_t jp) {
+      const uint32_t par = jp & 1;
+      ok = cx.wait_warp(B_O_FULL, jp & 1);
+      if (!ok) return;
+      tc_fence_after();
+      uint32_t o[MAXBLK][G];
+#pragma unroll
+      for (int t = 0; t < MAXBLK; ++t)
+        if (t < pr.nblk) tmem_ld_g<G>(tm + TM_O + t * 16 + tlane, o[t]);
+      tmem_ld_wait();
+      tc_fence_before();
+      cx.warp_arrive(B_O_FREE);
+      float acc[G];
+#pragma unroll
+      for (int g = 0; g < G; ++g) acc[g] = 0.0f;
+#pragma unroll
+      for (int t = 0; t < MAXBLK; ++t)
+        if (t < pr.nblk) {
+#pragma unroll
+          for (int g = 0; g < G; ++g) acc[g] = __fmaf_rn(wtab[(par * MAXBLK + t) * MAXG + g], __uint_as_float(o[t][g]), acc[g]);
+        }
+      float *dst = p.parts + (((size_t)pr.b * p.H_q + (size_t)pr.hk * G) * p.n_split + pr.sp) * PART_FLOATS;
+      const size_t head_stride = (size_t)p.n_split * PART_FLOATS;
+#pragma unroll
+      for (int g = 0; g < G; ++g) dst[g * head_stride + 2 + r] = acc[g];
+      if (t128 < G) {
+        float l = 0.0f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) l += xl[(par * 4 + q) * MAXG + t128];
+        dst[t128 * head_stride] = mfin[par * MAXG + t128];
+        dst[t128 * head_stride + 1] = l;
+      }
+    };
+
+    WorkIter w;
+    w.init(p, len_tab);
+    uint32_t j = 0;
+    Prev prev{0, 0, 0, 0};
+    while (ok && w.next(p.seq_lens)) {
+      const uint32_t par = j & 1;
+      const float lam = w.b < D_MAXREQ ? lam_tab[w.b]
+                                       : __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[w.b]), p.k_gscale[w.b]);
+      const int k_part = w.sp * DECODE_SPLIT;
+      // ---- all scores of the item at once: the last slot's barrier follows every QK MMA of the item
+      ok = cx.wait_warp(B_S_FULL + par * MAXBLK + MAXBLK - 1, (j >> 1) & 1);
+      if (!ok) break;
+      if (warp == 4) DTR(7, j);
+      tc_fence_after();
+      float sv[MAXBLK][G];
+      {
+        uint32_t sraw[MAXBLK][G];
+#pragma unroll
+        for (int t = 0; t < MAXBLK; ++t)
+          if (t < w.nblk) tmem_ld_g<G>(tm + TM_S + (par * MAXBLK + t) * 16 + tlane, sraw[t]);
+        tmem_ld_wait();
+        tc_fence_before();
+        cx.warp_arrive(B_S_FREE + par);
+#pragma unroll
+        for (int t = 0; t < MAXBLK; ++t) {
+          if (t < w.nblk) {
+            const bool valid = k_part + (w.nblk - 1 - t) * TILE + r < w.L;
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+              sv[t][g] = valid ? __uint_as_float(sraw[t][g]) : -INFINITY;
+              // warp maximum through an order-preserving integer key and one redux
+              const int bits = __float_as_int(sv[t][g]);
+              const int key = bits ^ ((bits >> 31) & 0x7FFFFFFF);
+              const int km = __reduce_max_sync(0xffffffffu, key);
+              if (lane == 0) xmax[((par * MAXBLK + t) * MAXG + g) * 4 + (warp - 4)] = __int_as_float(km ^ ((km >> 31) & 0x7FFFFFFF));
+            }
+          }
+        }
+      }
+      if (warp == 4) DTR(8, j);
+      cx.warp_arrive(B_XCHG);
+      ok = cx.wait_warp(B_XCHG, j & 1);
+      if (!ok) break;
+      if (warp == 4) DTR(9, j);
+      // ---- running maxima of the reverse traversal, then all P_hat of the item
+      {
+        float m[MAXBLK][G], run[G], lsum[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) run[g] = -INFINITY, lsum[g] = 0.0f;
+#pragma unroll
+        for (int t = 0; t < MAXBLK; ++t) {
+          if (t < w.nblk) {
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+              const float4 x = *reinterpret_cast<const float4 *>(&xmax[((par * MAXBLK + t) * MAXG + g) * 4]);
+              run[g] = fmaxf(run[g], fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w)));
+              m[t][g] = run[g];
+            }
+          }
+        }
+        uint8_t *pt = dsm + D_OFF_P + par * MAXBLK * 2048 + (r & 15);
+#pragma unroll
+        for (int t = 0; t < MAXBLK; ++t) {
+          if (t < w.nblk) {
+            float pq[G + 1];
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+              const float pv = ex2_approx(__fmaf_rn(sv[t][g], lam, -__fmul_rn(m[t][g], lam)));   // -inf -> 0
+              float wt = 1.0f;
+              if (m[t][g] != run[g]) wt = ex2_approx(__fmul_rn(m[t][g] - run[g], lam));   // uniform, rare
+              lsum[g] = __fmaf_rn(wt, pv, lsum[g]);
+              pq[g] = __fmul_rn(pv, 448.0f);
+              if (t128 == t * G + g) wtab[(par * MAXBLK + t) * MAXG + g] = wt;
+            }
+            pq[G] = 0.0f;
+#pragma unroll
+            for (int g = 0; g < G; g += 2) {
+              const uint32_t two = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(pq[g], pq[g + 1]), __NV_SATFINITE, __NV_E4M3);
+              pt[t * 2048 + g * 128 + (((r >> 4) ^ g) << 4)] = (uint8_t)two;
+              if (g + 1 < G) pt[t * 2048 + (g + 1) * 128 + (((r >> 4) ^ (g + 1)) << 4)] = (uint8_t)(two >> 8);
+            }
+          }
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          float ls = lsum[g];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+          if (lane == 0) xl[(par * 4 + (warp - 4)) * MAXG + g] = ls;
+          if (t128 == g) mfin[par * MAXG + g] = run[g];
+        }
+      }
+      fence_proxy_async_smem();
+      cx.warp_arrive(B_P_READY + par);
+      if (warp == 4) DTR(10, j);
+      if (j >= 1) {
+        write_out(prev, j - 1);
+        if (!ok) break;
+      }
+      if (warp == 4) DTR(11, j);
+      prev = Prev{w.b, w.hk, w.sp, w.nblk};
+      ++j;
+    }
+    if (ok && j >= 1) {
+      // the tables of the last item were written by other warps: one more exchange round
+      cx.warp_arrive(B_XCHG);
+      ok = cx.wait_warp(B_XCHG, j & 1);
+      if (ok) write_out(prev, j - 1);
     }
   }
 
@@ -674,8 +834,20 @@ extern "C" mpfa_status mpfa_decode(const mpfa_fp4_tensor *q, const mpfa_paged_kv
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t items = (size_t)B * H_kv * n_split;
   const unsigned grid = (unsigned)(items < (size_t)n_sm ? items : (size_t)n_sm);   // one persistent CTA per SM
-  MPFA_CUDA_OK(cudaFuncSetAttribute(decode_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)D_SMEM));
-  decode_split_kernel<<<grid, D_THREADS, D_SMEM, s>>>(p);
+  void (*kern)(const DecodeParams) = nullptr;
+  switch (H_q / H_kv) {
+    case 1: kern = decode_split_kernel<1>; break;
+    case 2: kern = decode_split_kernel<2>; break;
+    case 3: kern = decode_split_kernel<3>; break;
+    case 4: kern = decode_split_kernel<4>; break;
+    case 5: kern = decode_split_kernel<5>; break;
+    case 6: kern = decode_split_kernel<6>; break;
+    case 7: kern = decode_split_kernel<7>; break;
+    case 8: kern = decode_split_kernel<8>; break;
+    default: return MPFA_ERR_UNSUPPORTED;
+  }
+  MPFA_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)D_SMEM));
+  kern<<<grid, D_THREADS, D_SMEM, s>>>(p);
   MPFA_LAUNCH_OK();
   decode_merge_kernel<<<dim3(H_q, B), 128, 0, s>>>(p.parts, seq_lens, st->q_gscale, st->k_gscale, H_q, (int)n_split,
                                                    softmax_scale, v_scale, static_cast<__nv_bfloat16 *>(out_bf16),

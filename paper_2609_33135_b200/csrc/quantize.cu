@@ -219,7 +219,9 @@ __global__ void __launch_bounds__(128) delta_s_kernel(const __nv_bfloat16 *__res
         if ((t >> 6) < (N + PAGE - 1) / PAGE) {   // slots past N inside the last page are zero-filled
           const int page = page_row[t >> 6];
           if (page >= 0 && page < num_pages)
-            delta[((size_t)page * H_q + hk * G + g) * PAGE + (t & 63)] = __float2bfloat16_rn(v);
+            // 16-byte chunks XOR-swizzled by the head's index in its group: the row is read as a
+            // swizzled MN-major tensor-core operand by the decode kernel
+            delta[((size_t)page * H_q + hk * G + g) * PAGE + (((((t & 63) >> 3) ^ g) << 3) | (t & 7))] = __float2bfloat16_rn(v);
         }
       } else {
         delta[((size_t)b * H_q + hk * G + g) * n_pad + t] = __float2bfloat16_rn(v);

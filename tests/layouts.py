@@ -46,3 +46,10 @@ def paged_v_to_logical(slab: np.ndarray) -> np.ndarray:
     """[..., 8192] page slab -> [..., 64 tokens, 128 channels]."""
     t, c = np.meshgrid(np.arange(64), np.arange(128), indexing="ij")
     return slab[..., paged_v_offset(t, c)]
+
+
+def paged_delta_to_logical(page: np.ndarray, G: int) -> np.ndarray:
+    """[H_q, 64] Delta_S page -> [H_q, 64 tokens]."""
+    h = np.arange(page.shape[0])[:, None]
+    t = np.arange(64)[None, :]
+    return np.take_along_axis(page, (((t // 8) ^ (h % G)) * 8 + t % 8), axis=1)

@@ -6,7 +6,7 @@ import torch
 from oracle import mpfa_oracle as orc
 from paper_2609_33135_b200 import workloads as wl
 
-from layouts import paged_k_to_logical, paged_v_to_logical
+from layouts import paged_delta_to_logical, paged_k_to_logical, paged_v_to_logical
 from test_gpu_prefill import MAX_ABS, MEAN_ABS, bf16_neighbours_ok
 
 pytestmark = pytest.mark.gpu
@@ -46,8 +46,9 @@ def check_cache(state, w, caches, smooth=True):
             assert np.array_equal(lv[:, :n], z.v_codes[0, :, 64 * i:64 * i + n])
             assert not lk[:, n:].any() and not lv[:, n:].any()
             if smooth:
-                assert np.array_equal(dl[page][:, :n], z.delta[0, :, 64 * i:64 * i + n])
-                assert not dl[page][:, n:].any()
+                ld = paged_delta_to_logical(dl[page], w.H_q // w.H_kv)
+                assert np.array_equal(ld[:, :n], z.delta[0, :, 64 * i:64 * i + n])
+                assert not ld[:, n:].any()
 
 
 def run(w, smooth=True, v_scale=1.0):
