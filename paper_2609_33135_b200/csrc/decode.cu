@@ -28,7 +28,7 @@
 // sum with the factors multiplied out.  The partition state (m, l, O) goes to the workspace; a
 // second kernel merges partitions by log-sum-exp and writes BF16.
 //
-// Warps: 0 producer, 1 QK issue (+ TMEM allocation), 2 PV issue, 3 rewrites the K scales of
+// Warps: 0, 9 K producers, 8 V producer, 1 QK issue (+ TMEM allocation), 2 PV issue, 3 rewrites the K scales of
 // each block from [token][8] into the 32 x 16-byte tiles tcgen05.cp expects, 4-7 softmax and
 // partition write-out (TMEM lane quadrant = warp % 4).  Every wait is bounded.
 #include <cuda_bf16.h>
@@ -47,7 +47,7 @@ constexpr int MAXBLK = DECODE_SPLIT / TILE;   // 8 blocks per item
 
 constexpr int D_NK = 4;           // K ring stages
 constexpr int D_NV = 8;           // V ring stages
-constexpr int D_THREADS = 256;
+constexpr int D_THREADS = 320;
 
 // one K stage
 constexpr uint32_t KST_K = 0;          // 2 pages x 4096 B of codes: 64-byte rows, 64-byte swizzle
@@ -57,11 +57,11 @@ constexpr uint32_t KST_BYTES = 11264;
 constexpr uint32_t VST_BYTES = 16384;  // 2 pages x 8192 B: 128-byte rows, 128-byte swizzle
 constexpr uint32_t D_OFF_K = 0;
 constexpr uint32_t D_OFF_V = D_OFF_K + D_NK * KST_BYTES;
-constexpr uint32_t D_OFF_P = D_OFF_V + D_NV * VST_BYTES;   // [2 items][8 blocks] x 2048: P_hat^T, 16 rows of 128 keys
-constexpr uint32_t D_OFF_Q = D_OFF_P + 2 * MAXBLK * 2048;  // 2 x 1024: Q codes, 16 rows of 64 B, 64-byte swizzle
+constexpr uint32_t D_OFF_P = D_OFF_V + D_NV * VST_BYTES;   // [2 items][8 blocks] x 1024: P_hat^T, 8 rows of 128 keys (rows 8..15: zero block)
+constexpr uint32_t D_OFF_Q = D_OFF_P + 2 * MAXBLK * 1024;  // 2 x 1024: Q codes, 16 rows of 64 B, 64-byte swizzle
 constexpr uint32_t D_OFF_SFQ = D_OFF_Q + 2048;             // 2 x (2 x 512): Q scales, one tile per 64 channels
 constexpr uint32_t D_OFF_SFK = D_OFF_SFQ + 2048;           // D_NK x (2 x 512): K scales
-constexpr uint32_t D_OFF_ZERO = D_OFF_SFK + D_NK * 1024;    // 2048 B of zeros: the second K group of the Delta_S operand
+constexpr uint32_t D_OFF_ZERO = D_OFF_SFK + D_NK * 1024;    // 2048 B of zeros: second K group of the Delta_S operand, rows 8..15 of P_hat^T
 constexpr uint32_t D_OFF_IDENT = D_OFF_ZERO + 2048;        // 16 x 16 BF16 identity, MN-major, 128-byte swizzle
 constexpr uint32_t D_OFF_BAR = D_OFF_IDENT + 2048;
 constexpr uint32_t D_OFF_XMAX = D_OFF_BAR + 512;           // [2][8 blocks][MAXG][4 warps] floats
@@ -98,6 +98,7 @@ constexpr uint32_t TM_S = 0;       // [2 items][8 blocks] x 16
 constexpr uint32_t TM_O = 256;     // [8 blocks] x 16
 constexpr uint32_t TM_SFQ = 384;   // 2 x 8
 constexpr uint32_t TM_SFK = 400;   // D_NK x 8
+static_assert(TM_SFK + D_NK * 8 <= 512, "tensor memory");
 constexpr uint32_t TM_COLS = 512;
 
 constexpr long long D_WAIT_CYCLES = 4000000000ll;   // about two seconds
@@ -166,24 +167,36 @@ struct DecodeParams {
 // in (partition fastest, kv head, request) order; partitions beyond the sequence are skipped.
 struct WorkIter {
   int idx, stride, total, n_split, H_kv;
+  int ds, dh, db;   // the stride as (partition, kv head, request) digits: no division per step
   int b, hk, sp, L, nblk;
   const int32_t *len_tab;   // shared-memory copy of seq_lens (first D_MAXREQ requests)
   __device__ void init(const DecodeParams &p, const int32_t *tab) {
     len_tab = tab;
     stride = gridDim.x;
-    idx = (int)blockIdx.x - stride;
     n_split = p.n_split;
     H_kv = p.H_kv;
     total = p.B * p.H_kv * p.n_split;
+    ds = stride % n_split;
+    dh = (stride / n_split) % H_kv;
+    db = stride / (n_split * H_kv);
+    // one step before the first item (digits may be negative here; the first step normalises them)
+    idx = (int)blockIdx.x - stride;
+    const int i0 = (int)blockIdx.x;
+    sp = i0 % n_split - ds;
+    hk = (i0 / n_split) % H_kv - dh;
+    b = i0 / (n_split * H_kv) - db;
+    if (sp < 0) sp += n_split, hk -= 1;
+    if (hk < 0) hk += H_kv, b -= 1;
   }
   __device__ bool next(const int32_t *__restrict__ seq_lens) {
     for (;;) {
       idx += stride;
       if (idx >= total) return false;
-      sp = idx % n_split;
-      const int r = idx / n_split;
-      hk = r % H_kv;
-      b = r / H_kv;
+      sp += ds;
+      hk += dh;
+      b += db;
+      if (sp >= n_split) sp -= n_split, hk += 1;
+      if (hk >= H_kv) hk -= H_kv, b += 1;
       L = b < D_MAXREQ ? len_tab[b] : seq_lens[b];
       const int rem = L - sp * DECODE_SPLIT;
       if (rem > 0) {
@@ -226,22 +239,16 @@ struct DCtx {
   }
 };
 
-// Page ids of the blocks of one item, lane l holding block l's two pages (-1 = not there).
+// Page ids of the blocks of one item, lane l holding block l's two table entries (loads only: the values
+// are range-checked where they are used, so that nothing waits for them here).
 __device__ __forceinline__ void lookup_pages(const DecodeParams &p, const WorkIter &w, int lane, int &pid0, int &pid1) {
   pid0 = -1, pid1 = -1;
-  bool bad = false;
   if (lane < w.nblk) {
-    const int first = w.sp * DECODE_SPLIT + lane * TILE;
-    const int pg = first / PAGE;
+    const int pg = (w.sp * DECODE_SPLIT + lane * TILE) / PAGE;
     const int32_t *row = p.page_table + (size_t)w.b * p.max_pages;
     if (pg < p.max_pages) pid0 = row[pg];
-    if (pid0 < 0 || pid0 >= p.num_pages) pid0 = -1, bad = true;
-    if (first + PAGE < w.L) {
-      if (pg + 1 < p.max_pages) pid1 = row[pg + 1];
-      if (pid1 < 0 || pid1 >= p.num_pages) pid1 = -1, bad = true;
-    }
+    if (pg + 1 < p.max_pages) pid1 = row[pg + 1];
   }
-  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(p.status, MPFA_DEV_BAD_PAGE);
 }
 
 template <int G>
@@ -258,11 +265,14 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   DCtx cx{sbase + D_OFF_BAR, abort_flag, p.status};
+#ifdef MPFA_TRACE
+  if (g_dtrace && threadIdx.x == 0) g_dtrace[4096 + 2 * blockIdx.x] = (long long)globaltimer_ns();
+#endif
 
   // ---- set-up: barriers, zeroed operand tiles (rows G..15 stay zero for good), TMEM
   if (threadIdx.x == 0) {
     for (int i = 0; i < D_NK; ++i) {
-      mbar_init(cx.bar(B_K_FULL + i), 1);
+      mbar_init(cx.bar(B_K_FULL + i), 2);
       mbar_init(cx.bar(B_K_EMPTY + i), 1);
       mbar_init(cx.bar(B_SF_READY + i), 1);
     }
@@ -308,112 +318,99 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
   tc_fence_after();
   const uint32_t tm = *tmem_slot;
 
-  if (warp == 0) {
-    // ================= producer: the K walk runs one item ahead of the V walk
-    WorkIter wk, wv;
-    wk.init(p, len_tab);
-    wv.init(p, len_tab);
-    uint32_t kc = 0, vc = 0;
+  if (warp == 0 || warp >= 8) {
+    // ================= producers: warps 0 and 9 stream the K ring (0: codes; 9: block scales and Delta_S,
+    // both arriving on the stage's barrier), warp 8 the V ring.  Issuing a bulk copy costs a warp well over a
+    // hundred cycles, so the ten copies of a block are spread over three warps.
+    // Nothing orders the two streams but the data flow: a K stage is released by its QK MMAs, a V stage
+    // only after the item's softmax, so K runs about one item ahead.  Page ids are loaded one item before
+    // they are used and validated at use, so the loop never waits for the table.
+    const bool is_k = warp != 8, is_codes = warp == 0;
+    WorkIter w, wl;
+    w.init(p, len_tab);
+    wl.init(p, len_tab);
+    uint32_t c = 0;   // block counter of this ring
     bool ok = true;
     const uint32_t d_bytes = p.delta ? (uint32_t)G * PAGE * 2 : 0u;
-    const uint32_t kpage_bytes = 4096u + 512u + d_bytes;
-    int pk0 = -1, pk1 = -1, pv0 = -1, pv1 = -1;
-    auto issue_k = [&](const WorkIter &w, int t) {
-      const uint32_t st = kc % D_NK;
-      if (kc >= (uint32_t)D_NK && !cx.wait_warp(B_K_EMPTY + st, ((kc / D_NK) - 1) & 1)) {
-        ok = false;
-        return;
-      }
-      DTR(0, kc);
-      const int u = w.nblk - 1 - t;
-      const int id0 = __shfl_sync(0xffffffffu, pk0, u), id1 = __shfl_sync(0xffffffffu, pk1, u);
-      if (elect_one()) {
-        const uint32_t full = cx.bar(B_K_FULL + st);
-        const uint32_t sdst = sbase + D_OFF_K + st * KST_BYTES;
-        mbar_expect_tx(full, (id0 >= 0 ? kpage_bytes : 0u) + (id1 >= 0 ? kpage_bytes : 0u));
+    const uint32_t kpage_bytes = is_codes ? 4096u : 512u + d_bytes;
+    const int n_ring = is_k ? D_NK : D_NV;
+    const int b_full = is_k ? B_K_FULL : B_V_FULL, b_empty = is_k ? B_K_EMPTY : B_V_EMPTY;
+    int pc0 = -1, pc1 = -1, pn0 = -1, pn1 = -1;
+    bool vw = w.next(p.seq_lens);
+    bool vl = wl.next(p.seq_lens);
+    if (vw) lookup_pages(p, w, lane, pc0, pc1);
+    uint32_t jtr = 0;
+    while (ok && vw) {
+      if (is_codes) DTR(12, jtr);
+      vl = wl.next(p.seq_lens);
+      if (is_codes) DTR(13, jtr);
+      if (vl) lookup_pages(p, wl, lane, pn0, pn1);   // consumed one item later
+      if (is_codes) DTR(14, jtr);
+      ++jtr;
+      for (int t = 0; ok && t < w.nblk; ++t, ++c) {
+        const uint32_t st = c % n_ring;
+        if (c >= (uint32_t)n_ring && !cx.wait_warp(b_empty + st, ((c / n_ring) - 1) & 1)) {
+          ok = false;
+          break;
+        }
+        if (warp != 9) DTR(is_k ? 0 : 1, c);
+        const int u = w.nblk - 1 - t;
+        int id0 = __shfl_sync(0xffffffffu, pc0, u), id1 = __shfl_sync(0xffffffffu, pc1, u);
+        const bool want1 = w.sp * DECODE_SPLIT + u * TILE + PAGE < w.L;
+        const bool bad = id0 < 0 || id0 >= p.num_pages || (want1 && (id1 < 0 || id1 >= p.num_pages));
+        if (bad && lane == 0 && !is_codes) atomicOr(p.status, MPFA_DEV_BAD_PAGE);
+        if (id0 < 0 || id0 >= p.num_pages) id0 = -1;
+        if (!want1 || id1 < 0 || id1 >= p.num_pages) id1 = -1;
+        const uint32_t full = cx.bar(b_full + st);
+        if (is_k) {
+          if (elect_one()) {
+            const uint32_t sdst = sbase + D_OFF_K + st * KST_BYTES;
+            mbar_expect_tx(full, (id0 >= 0 ? kpage_bytes : 0u) + (id1 >= 0 ? kpage_bytes : 0u));
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const int id = half == 0 ? id0 : id1;
-          if (id < 0) continue;
-          const size_t slab = (size_t)id * p.H_kv + w.hk;
-          bulk_load(sdst + KST_K + half * 4096, p.k_codes + slab * 4096, 4096, full);
-          bulk_load(sdst + KST_SF + half * 512, p.k_sf + slab * 512, 512, full);
-          if (d_bytes)
-            bulk_load(sdst + KST_DELTA + half * 1024, p.delta + ((size_t)id * p.H_q + (size_t)w.hk * G) * PAGE, d_bytes, full);
-        }
-      }
-      __syncwarp();
-      ++kc;
-    };
-    auto issue_v = [&](const WorkIter &w, int t) {
-      const uint32_t st = vc % D_NV;
-      if (vc >= (uint32_t)D_NV && !cx.wait_warp(B_V_EMPTY + st, ((vc / D_NV) - 1) & 1)) {
-        ok = false;
-        return;
-      }
-      DTR(1, vc);
-      const int u = w.nblk - 1 - t;
-      const int id0 = __shfl_sync(0xffffffffu, pv0, u), id1 = __shfl_sync(0xffffffffu, pv1, u);
-      uint8_t *stage = dsm + D_OFF_V + st * VST_BYTES;
-      // a page that is not there contributes P_hat = 0 times V: V must be finite, so zero it
-      if (id0 < 0 || id1 < 0) {
+            for (int half = 0; half < 2; ++half) {
+              const int id = half == 0 ? id0 : id1;
+              if (id < 0) continue;
+              const size_t slab = (size_t)id * p.H_kv + w.hk;
+              if (is_codes) {
+                bulk_load(sdst + KST_K + half * 4096, p.k_codes + slab * 4096, 4096, full);
+              } else {
+                bulk_load(sdst + KST_SF + half * 512, p.k_sf + slab * 512, 512, full);
+                if (d_bytes)
+                  bulk_load(sdst + KST_DELTA + half * 1024, p.delta + ((size_t)id * p.H_q + (size_t)w.hk * G) * PAGE, d_bytes, full);
+              }
+            }
+          }
+        } else {
+          // a page that is not there contributes P_hat = 0 times V: V must be finite, so zero it
+          if (id0 < 0 || id1 < 0) {
+            uint8_t *stage = dsm + D_OFF_V + st * VST_BYTES;
 #pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-          if ((half == 0 ? id0 : id1) >= 0) continue;
-          for (int i = 0; i < 16; ++i)
-            *reinterpret_cast<uint4 *>(stage + half * 8192 + i * 512 + lane * 16) = make_uint4(0u, 0u, 0u, 0u);
+            for (int half = 0; half < 2; ++half) {
+              if ((half == 0 ? id0 : id1) >= 0) continue;
+              for (int i = 0; i < 16; ++i)
+                *reinterpret_cast<uint4 *>(stage + half * 8192 + i * 512 + lane * 16) = make_uint4(0u, 0u, 0u, 0u);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+          }
+          if (elect_one()) {
+            const uint32_t sdst = sbase + D_OFF_V + st * VST_BYTES;
+            mbar_expect_tx(full, (id0 >= 0 ? 8192u : 0u) + (id1 >= 0 ? 8192u : 0u));
+            if (id0 >= 0) bulk_load(sdst, p.v_fp8 + ((size_t)id0 * p.H_kv + w.hk) * 8192, 8192, full);
+            if (id1 >= 0) bulk_load(sdst + 8192, p.v_fp8 + ((size_t)id1 * p.H_kv + w.hk) * 8192, 8192, full);
+          }
         }
-        fence_proxy_async_smem();
         __syncwarp();
       }
-      if (elect_one()) {
-        const uint32_t full = cx.bar(B_V_FULL + st);
-        const uint32_t sdst = sbase + D_OFF_V + st * VST_BYTES;
-        mbar_expect_tx(full, (id0 >= 0 ? 8192u : 0u) + (id1 >= 0 ? 8192u : 0u));
-        if (id0 >= 0) bulk_load(sdst, p.v_fp8 + ((size_t)id0 * p.H_kv + w.hk) * 8192, 8192, full);
-        if (id1 >= 0) bulk_load(sdst + 8192, p.v_fp8 + ((size_t)id1 * p.H_kv + w.hk) * 8192, 8192, full);
-      }
-      __syncwarp();
-      ++vc;
-    };
-    // page ids are looked up one item before the K walk needs them (pn: the item after wk's)
-    WorkIter wl;
-    wl.init(p, len_tab);
-    int pn0 = -1, pn1 = -1;
-    bool vk = wk.next(p.seq_lens);
-    bool vl = wl.next(p.seq_lens);
-    if (vk) {
-      lookup_pages(p, wk, lane, pk0, pk1);
-      vl = wl.next(p.seq_lens);
-      if (vl) lookup_pages(p, wl, lane, pn0, pn1);
-      for (int t = 0; ok && t < wk.nblk; ++t) issue_k(wk, t);
-    }
-    bool vv = wv.next(p.seq_lens);
-    while (ok && vv) {
-      pv0 = pk0, pv1 = pk1;   // wv now stands where wk stood
-      vk = wk.next(p.seq_lens);
-      if (vk) {
-        pk0 = pn0, pk1 = pn1;
-        vl = wl.next(p.seq_lens);
-        if (vl) lookup_pages(p, wl, lane, pn0, pn1);
-      }
-      const int nk = vk ? wk.nblk : 0, nv = wv.nblk;
-      for (int t = 0; ok && t < max(nk, nv); ++t) {
-        if (t < nk) issue_k(wk, t);
-        if (ok && t < nv) issue_v(wv, t);
-      }
-      vv = wv.next(p.seq_lens);
+      if (is_codes) DTR(15, jtr - 1);
+      vw = w.next(p.seq_lens);
+      pc0 = pn0, pc1 = pn1;
     }
     if (!ok) {
       // another role gave up: let the copies already issued land before shared memory goes away
-      for (uint32_t i = kc - min(kc, (uint32_t)D_NK); i < kc; ++i) {
+      for (uint32_t i = c - min(c, (uint32_t)n_ring); i < c; ++i) {
         const long long t0 = clock64();
-        while (!mbar_try_wait(cx.bar(B_K_FULL + i % D_NK), (i / D_NK) & 1) && clock64() - t0 < D_WAIT_CYCLES) {
-        }
-      }
-      for (uint32_t i = vc - min(vc, (uint32_t)D_NV); i < vc; ++i) {
-        const long long t0 = clock64();
-        while (!mbar_try_wait(cx.bar(B_V_FULL + i % D_NV), (i / D_NV) & 1) && clock64() - t0 < D_WAIT_CYCLES) {
+        while (!mbar_try_wait(cx.bar(b_full + i % n_ring), (i / n_ring) & 1) && clock64() - t0 < D_WAIT_CYCLES) {
         }
       }
     }
@@ -489,7 +486,9 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
         tc_fence_after();
         if (elect_one()) {
           const uint64_t d_v = smem_desc(sbase + D_OFF_V + st * VST_BYTES, 16, 1024, SWZ_128B);
-          const uint64_t d_p = smem_desc(sbase + D_OFF_P + (par * MAXBLK + t) * 2048, 16, 1024, SWZ_128B);
+          // rows 0..7 of P_hat^T in the block's tile, rows 8..15 (the next 8-row group) from the zero block
+          const uint32_t a_p = sbase + D_OFF_P + (par * MAXBLK + t) * 1024;
+          const uint64_t d_p = smem_desc(a_p, 16, sbase + D_OFF_ZERO - a_p, SWZ_128B);
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)   // 32 keys per MMA
             mma_e4m3_ss(tm + TM_O + t * 16, d_v + (uint64_t)((4096 * k4) >> 4), d_p + (uint64_t)((32 * k4) >> 4), id_pv,
@@ -678,7 +677,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
             }
           }
         }
-        uint8_t *pt = dsm + D_OFF_P + par * MAXBLK * 2048 + (r & 15);
+        uint8_t *pt = dsm + D_OFF_P + par * MAXBLK * 1024 + (r & 15);
 #pragma unroll
         for (int t = 0; t < MAXBLK; ++t) {
           if (t < w.nblk) {
@@ -696,8 +695,8 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
 #pragma unroll
             for (int g = 0; g < G; g += 2) {
               const uint32_t two = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(pq[g], pq[g + 1]), __NV_SATFINITE, __NV_E4M3);
-              pt[t * 2048 + g * 128 + (((r >> 4) ^ g) << 4)] = (uint8_t)two;
-              if (g + 1 < G) pt[t * 2048 + (g + 1) * 128 + (((r >> 4) ^ (g + 1)) << 4)] = (uint8_t)(two >> 8);
+              pt[t * 1024 + g * 128 + (((r >> 4) ^ g) << 4)] = (uint8_t)two;
+              if (g + 1 < G) pt[t * 1024 + (g + 1) * 128 + (((r >> 4) ^ (g + 1)) << 4)] = (uint8_t)(two >> 8);
             }
           }
         }
@@ -732,6 +731,9 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tm, TM_COLS);
+#ifdef MPFA_TRACE
+  if (g_dtrace && threadIdx.x == 0) g_dtrace[4096 + 2 * blockIdx.x + 1] = (long long)globaltimer_ns();
+#endif
 }
 
 // Merge of the partition states (Section 5.3): M = max m_s, w_s = 2^(lam (m_s - M)),
