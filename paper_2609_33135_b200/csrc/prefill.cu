@@ -102,6 +102,29 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// Packed FP32 pairs (one issue slot for two IEEE operations; each half rounds like the scalar form).
+__device__ __forceinline__ void fma2(float &d0, float &d1, float a0, float a1, float b, float c) {
+  asm("{.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+__device__ __forceinline__ void mul2(float &d0, float &d1, float a0, float a1, float b) {
+  asm("{.reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\t"
+      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b));
+}
+__device__ __forceinline__ void acc2(float &d0, float &d1, float a0, float a1) {
+  asm("{.reg .b64 ra, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rd, {%0, %1};\n\t"
+      "add.rn.f32x2 rd, rd, ra;\n\tmov.b64 {%0, %1}, rd;}"
+      : "+f"(d0), "+f"(d1)
+      : "f"(a0), "f"(a1));
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -404,12 +427,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       {
         uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
         uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
-        uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
-        uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
         tmem_ld32(tS, s0);
         tmem_ld32(tS + 32, s1);
-        tmem_ld32(tS + 64, s2);
-        tmem_ld32(tS + 96, s3);
       }
       // While the scores are on their way, test (without blocking) the two other conditions this
       // block needs; the answers are consumed later, so their latency overlaps the TMEM load:
@@ -423,19 +442,40 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #ifdef MPFA_ABLATE_NO_MHAND
       have_prev = true;
 #endif
+      const bool ragged = key0 + TILE - 1 > limit;   // diagonal / ragged block only
       tmem_ld_wait();
-      tc_fence_before();
-      warp_arrive(cx.bar(BAR_S_EMPTY), lane);   // the row is in registers: Q K^T of block t+1 may overwrite it
-      TR(2 + grp, t, 2);
-      if (key0 + TILE - 1 > limit) {   // diagonal / ragged block only
+      {
+        // second half of the row in flight while the maximum of the first half is taken
+        uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
+        uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
+        tmem_ld32(tS + 64, s2);
+        tmem_ld32(tS + 96, s3);
+      }
+      if (ragged) {
 #pragma unroll
-        for (int i = 0; i < 128; ++i)
+        for (int i = 0; i < 64; ++i)
           if (key0 + i > limit) s[i] = 0xFF800000u;   // -inf
       }
       // row maximum (Eq. 3)
       float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-      for (int i = 0; i < 128; i += 8) {
+      for (int i = 0; i < 64; i += 8) {
+        mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+        mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+        mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+      }
+      tmem_ld_wait();
+      tc_fence_before();
+      warp_arrive(cx.bar(BAR_S_EMPTY), lane);   // the row is in registers: Q K^T of block t+1 may overwrite it
+      TR(2 + grp, t, 2);
+      if (ragged) {
+#pragma unroll
+        for (int i = 64; i < 128; ++i)
+          if (key0 + i > limit) s[i] = 0xFF800000u;   // -inf
+      }
+#pragma unroll
+      for (int i = 64; i < 128; i += 8) {
         mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
         mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
         mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
@@ -482,14 +522,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #endif
           // q = 448 P is the E4M3 operand (Section 4.1); the row sum is taken over q and the
           // factor 448 is divided out once in the epilogue
-          const float q0 = __fmul_rn(EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i]), lam, c)), 448.0f);
-          const float q1 = __fmul_rn(EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 1]), lam, c)), 448.0f);
-          const float q2 = __fmul_rn(EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 2]), lam, c)), 448.0f);
-          const float q3 = __fmul_rn(EX2_(__fmaf_rn(__uint_as_float(s[c0 + 4 * i + 3]), lam, c)), 448.0f);
-          sum0 += q0;
-          sum1 += q1;
-          sum2 += q2;
-          sum3 += q3;
+          float x0, x1, x2, x3, q0, q1, q2, q3;
+          fma2(x0, x1, __uint_as_float(s[c0 + 4 * i]), __uint_as_float(s[c0 + 4 * i + 1]), lam, c);
+          fma2(x2, x3, __uint_as_float(s[c0 + 4 * i + 2]), __uint_as_float(s[c0 + 4 * i + 3]), lam, c);
+          mul2(q0, q1, EX2_(x0), EX2_(x1), 448.0f);
+          mul2(q2, q3, EX2_(x2), EX2_(x3), 448.0f);
+          acc2(sum0, sum1, q0, q1);
+          acc2(sum2, sum3, q2, q3);
           const uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q0, q1), __NV_SATFINITE, __NV_E4M3);
           const uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q2, q3), __NV_SATFINITE, __NV_E4M3);
           packed[i] = (lo & 0xFFFFu) | (hi << 16);
