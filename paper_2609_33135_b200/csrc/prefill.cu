@@ -177,8 +177,7 @@ struct Ctx {
     for (;;) {
 #pragma unroll 1
       for (int k = 0; k < 32; ++k) {
-        if (mbar_try_wait(a, parity)) return true;
-        __nanosleep(20);
+        if (mbar_try_wait_hint(a, parity, 1000u)) return true;   // the hardware may park the thread meanwhile
       }
       if (*abort_flag) return false;
       if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
@@ -510,34 +509,49 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       sum0 = __uint_as_float(s[5]);
       if (false)
 #endif
-#pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t packed[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
+      {
 #ifdef MPFA_ABLATE_NO_EXP
 #define EX2_(x) (x)
 #else
 #define EX2_(x) ex2_approx(x)
 #endif
-          // q = 448 P is the E4M3 operand (Section 4.1); the row sum is taken over q and the
-          // factor 448 is divided out once in the epilogue
-          float x0, x1, x2, x3, q0, q1, q2, q3;
-          fma2(x0, x1, __uint_as_float(s[c0 + 4 * i]), __uint_as_float(s[c0 + 4 * i + 1]), lam, c);
-          fma2(x2, x3, __uint_as_float(s[c0 + 4 * i + 2]), __uint_as_float(s[c0 + 4 * i + 3]), lam, c);
-          mul2(q0, q1, EX2_(x0), EX2_(x1), 448.0f);
-          mul2(q2, q3, EX2_(x2), EX2_(x3), 448.0f);
-          acc2(sum0, sum1, q0, q1);
-          acc2(sum2, sum3, q2, q3);
-          const uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q0, q1), __NV_SATFINITE, __NV_E4M3);
-          const uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q2, q3), __NV_SATFINITE, __NV_E4M3);
-          packed[i] = (lo & 0xFFFFu) | (hi << 16);
-        }
+        // Software pipeline at 32-column granularity, in place: the exponentials of chunk k+1 are
+        // issued between the instructions that consume chunk k (scale by 448, row sum, E4M3 pack),
+        // so a result is needed a few hundred cycles after its MUFU instruction was issued.
+        // q = 448 P is the E4M3 operand (Section 4.1); the row sum is taken over q and the factor
+        // 448 is divided out once in the epilogue.
+        auto exp_pair = [&](int i) {   // s[i], s[i+1] <- 2^(lam s - lam m)
+          float x0, x1;
+          fma2(x0, x1, __uint_as_float(s[i]), __uint_as_float(s[i + 1]), lam, c);
+          s[i] = __float_as_uint(EX2_(x0));
+          s[i + 1] = __float_as_uint(EX2_(x1));
+        };
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) exp_pair(i);
+#pragma unroll
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t packed[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if (c0 + 32 < 128) {
+              exp_pair(c0 + 32 + 4 * i);
+              exp_pair(c0 + 32 + 4 * i + 2);
+            }
+            float q0, q1, q2, q3;
+            mul2(q0, q1, __uint_as_float(s[c0 + 4 * i]), __uint_as_float(s[c0 + 4 * i + 1]), 448.0f);
+            mul2(q2, q3, __uint_as_float(s[c0 + 4 * i + 2]), __uint_as_float(s[c0 + 4 * i + 3]), 448.0f);
+            acc2(sum0, sum1, q0, q1);
+            acc2(sum2, sum3, q2, q3);
+            const uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q0, q1), __NV_SATFINITE, __NV_E4M3);
+            const uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q2, q3), __NV_SATFINITE, __NV_E4M3);
+            packed[i] = (lo & 0xFFFFu) | (hi << 16);
+          }
 #ifndef MPFA_ABLATE_NO_PST
-        tmem_st8(tP + (c0 >> 2), packed);
+          tmem_st8(tP + (c0 >> 2), packed);
 #else
-        if (packed[0] == 0x12345u && packed[7] == 77u) tmem_st8(tP + (c0 >> 2), packed);
+          if (packed[0] == 0x12345u && packed[7] == 77u) tmem_st8(tP + (c0 >> 2), packed);
 #endif
+        }
       }
       l_own = __fadd_rn(__fmul_rn(a_own, l_own), (sum0 + sum1) + (sum2 + sum3));
       m_own = m_t;
