@@ -145,7 +145,7 @@ mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, int B, int 
  * The column sums and maxima live in a fixed MPFA_STATIC_SCRATCH_BYTES buffer that is
  * part of the library image: every GPU that loads the library carries it until the
  * process exits.  Shapes whose statistics need more (mpfa_quantize_workspace_bytes(B, H_q,
- * H_kv) > MPFA_STATIC_SCRATCH_BYTES, i.e. roughly B * (H_q + H_kv) > 500) are rejected
+ * H_kv) > MPFA_STATIC_SCRATCH_BYTES, i.e. roughly B * (H_q + H_kv) > 250) are rejected
  * with MPFA_ERR_WORKSPACE and nothing is launched.  The call allocates nothing and frees
  * nothing.  The first call on each device looks up the buffer's device address (with that
  * device current); make that first call before starting any stream capture.  All calls on

@@ -28,8 +28,6 @@ mpfa_status check_arch() {
 
 namespace {
 
-constexpr int COLS_PER_BLOCK = 2048;  // 256 threads x 8 columns
-constexpr int TOK_PER_BLOCK = 128;
 
 __device__ __forceinline__ void unpack8(const uint4 &u, float (&f)[8]) {
   const uint32_t w[4] = {u.x, u.y, u.z, u.w};
@@ -40,52 +38,96 @@ __device__ __forceinline__ void unpack8(const uint4 &u, float (&f)[8]) {
   }
 }
 
-// Column sums in FP64.  For BF16 inputs whose nonzero magnitudes are >= 2^-14 every
-// partial sum of up to 2^17 tokens is exactly representable, so the atomic accumulation
-// order cannot change the result.
-__global__ void __launch_bounds__(256) colsum_kernel(const __nv_bfloat16 *__restrict__ x, int N, int cols,
-                                                     double *__restrict__ sums) {
-  const int b = blockIdx.z;
-  const int col = blockIdx.y * COLS_PER_BLOCK + threadIdx.x * 8;
-  if (col >= cols) return;
-  const int t0 = blockIdx.x * TOK_PER_BLOCK;
-  const int t1 = min(N, t0 + TOK_PER_BLOCK);
-  double acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  const __nv_bfloat16 *p = x + ((size_t)b * N + t0) * cols + col;
-  for (int t = t0; t < t1; ++t, p += cols) {
-    float f[8];
-    unpack8(*reinterpret_cast<const uint4 *>(p), f);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] += (double)f[i];
-  }
-#pragma unroll
-  for (int i = 0; i < 8; ++i) atomicAdd(&sums[(size_t)b * cols + col + i], acc[i]);
+// One pass over a tensor [B, N, cols] gives, per column, everything the statistics need:
+//   the sum in FP64 (Eq. 7) - for BF16 inputs whose nonzero magnitudes are >= 2^-14 every partial sum
+//   of up to 2^17 tokens is exactly representable, so the accumulation order cannot change the result;
+//   max x and max (-x) - rounding is monotonic and symmetric, so
+//   max_t |fl(x_t - mu)| = max(fl(max x - mu), fl(mu - min x)) and no second pass over the tensor is
+//   needed for the per-tensor scale.
+// A CTA covers 256 columns x COLSTAT_TOKENS tokens: thread = (token lane 0..7, 8 columns), a warp
+// reads 512 contiguous bytes of one token row, four independent 16-byte loads in flight per thread;
+// the eight token lanes are folded in shared memory, then one atomic per column and statistic.
+// Maxima are stored as order-preserving unsigned keys so that a zeroed workspace is the identity.
+constexpr int COLSTAT_COLS = 256;
+constexpr int COLSTAT_TOKENS = 256;
+
+__device__ __forceinline__ unsigned int ordered_key(float f) {   // monotonic float -> unsigned, key(-inf) > 0
+  const unsigned int b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_key(unsigned int k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
-__global__ void finalize_mean_kernel(const double *__restrict__ sums, int n, int N, float *__restrict__ mean) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) mean[i] = __double2float_rn(__ddiv_rn(sums[i], (double)N));
-}
-
-// max |x - mean| per batch element; non-negative floats order like their bit patterns.
-__global__ void __launch_bounds__(256) amax_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ mean,
-                                                   int N, int cols, unsigned int *__restrict__ amax) {
+__global__ void __launch_bounds__(256) colstat_kernel(const __nv_bfloat16 *__restrict__ x, int N, int cols,
+                                                      double *__restrict__ sums, unsigned int *__restrict__ kmax,
+                                                      unsigned int *__restrict__ knegmax) {
+  __shared__ double s_sum[8][COLSTAT_COLS];
+  __shared__ float s_max[8][COLSTAT_COLS], s_neg[8][COLSTAT_COLS];
   const int b = blockIdx.z;
-  const int col = blockIdx.y * COLS_PER_BLOCK + threadIdx.x * 8;
-  float m = 0.0f;
+  const int tl = threadIdx.x >> 5, cg = threadIdx.x & 31;
+  const int col = blockIdx.y * COLSTAT_COLS + cg * 8;
+  const int t0 = blockIdx.x * COLSTAT_TOKENS;
+  const int t1 = min(N, t0 + COLSTAT_TOKENS);
+  double acc[8];
+  float mx[8], ng[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0.0, mx[i] = -INFINITY, ng[i] = -INFINITY;
   if (col < cols) {
-    float mu[8];
+    const __nv_bfloat16 *p = x + ((size_t)b * N + t0 + tl) * cols + col;
+    const size_t step = (size_t)8 * cols;
+    int t = t0 + tl;
+    for (; t + 24 < t1; t += 32, p += 4 * step) {
+      uint4 u[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) mu[i] = mean[(size_t)b * cols + col + i];
-    const int t0 = blockIdx.x * TOK_PER_BLOCK;
-    const int t1 = min(N, t0 + TOK_PER_BLOCK);
-    const __nv_bfloat16 *p = x + ((size_t)b * N + t0) * cols + col;
-    for (int t = t0; t < t1; ++t, p += cols) {
+      for (int j = 0; j < 4; ++j) u[j] = *reinterpret_cast<const uint4 *>(p + j * step);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float f[8];
+        unpack8(u[j], f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] += (double)f[i], mx[i] = fmaxf(mx[i], f[i]), ng[i] = fmaxf(ng[i], -f[i]);
+      }
+    }
+    for (; t < t1; t += 8, p += step) {
       float f[8];
       unpack8(*reinterpret_cast<const uint4 *>(p), f);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(__fsub_rn(f[i], mu[i])));
+      for (int i = 0; i < 8; ++i) acc[i] += (double)f[i], mx[i] = fmaxf(mx[i], f[i]), ng[i] = fmaxf(ng[i], -f[i]);
     }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) s_sum[tl][cg * 8 + i] = acc[i], s_max[tl][cg * 8 + i] = mx[i], s_neg[tl][cg * 8 + i] = ng[i];
+  __syncthreads();
+  const int c = blockIdx.y * COLSTAT_COLS + threadIdx.x;
+  if (c < cols) {
+    double a = 0.0;
+    float m = -INFINITY, g = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) a += s_sum[j][threadIdx.x], m = fmaxf(m, s_max[j][threadIdx.x]), g = fmaxf(g, s_neg[j][threadIdx.x]);
+    const size_t o = (size_t)b * cols + c;
+    atomicAdd(&sums[o], a);
+    atomicMax(&kmax[o], ordered_key(m));
+    atomicMax(&knegmax[o], ordered_key(g));
+  }
+}
+
+// Per column: mean = fl(sum / N) (0 without smoothing); per batch element: max |x - mean| from the
+// column extremes.  grid (ceil(cols / 256), B).
+__global__ void __launch_bounds__(256) finalize_stats_kernel(const double *__restrict__ sums,
+                                                             const unsigned int *__restrict__ kmax,
+                                                             const unsigned int *__restrict__ knegmax, int cols, int N,
+                                                             int smooth, float *__restrict__ mean,
+                                                             unsigned int *__restrict__ amax) {
+  const int b = blockIdx.y, c = blockIdx.x * 256 + threadIdx.x;
+  float m = 0.0f;
+  if (c < cols) {
+    const size_t o = (size_t)b * cols + c;
+    const float mu = smooth ? __double2float_rn(__ddiv_rn(sums[o], (double)N)) : 0.0f;
+    mean[o] = mu;
+    const float hi = from_ordered_key(kmax[o]), lo = -from_ordered_key(knegmax[o]);
+    m = fmaxf(__fsub_rn(hi, mu), __fsub_rn(mu, lo));   // non-negative: lo <= mu <= hi (or mu = 0 and the larger side wins)
+    m = fmaxf(m, 0.0f);
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
@@ -95,7 +137,7 @@ __global__ void __launch_bounds__(256) amax_kernel(const __nv_bfloat16 *__restri
   if (threadIdx.x == 0) {
 #pragma unroll
     for (int i = 1; i < 8; ++i) m = fmaxf(m, wmax[i]);
-    atomicMax(&amax[b], __float_as_uint(m));
+    atomicMax(&amax[b], __float_as_uint(m));   // non-negative floats order like their bit patterns
   }
 }
 
@@ -323,6 +365,7 @@ size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 struct StatsWorkspace {
   double *sums_q, *sums_k;
+  unsigned int *max_q, *neg_q, *max_k, *neg_k;   // per-column extremes as ordered keys
   unsigned int *amax_q, *amax_k;
   size_t bytes;
 };
@@ -335,6 +378,14 @@ StatsWorkspace carve(void *ws, int B, int H_q, int H_kv) {
   o += align256((size_t)B * H_q * HEAD_DIM * sizeof(double));
   w.sums_k = reinterpret_cast<double *>(base + o);
   o += align256((size_t)B * H_kv * HEAD_DIM * sizeof(double));
+  w.max_q = reinterpret_cast<unsigned int *>(base + o);
+  o += align256((size_t)B * H_q * HEAD_DIM * sizeof(unsigned int));
+  w.neg_q = reinterpret_cast<unsigned int *>(base + o);
+  o += align256((size_t)B * H_q * HEAD_DIM * sizeof(unsigned int));
+  w.max_k = reinterpret_cast<unsigned int *>(base + o);
+  o += align256((size_t)B * H_kv * HEAD_DIM * sizeof(unsigned int));
+  w.neg_k = reinterpret_cast<unsigned int *>(base + o);
+  o += align256((size_t)B * H_kv * HEAD_DIM * sizeof(unsigned int));
   w.amax_q = reinterpret_cast<unsigned int *>(base + o);
   o += align256((size_t)B * sizeof(unsigned int));
   w.amax_k = reinterpret_cast<unsigned int *>(base + o);
@@ -343,20 +394,15 @@ StatsWorkspace carve(void *ws, int B, int H_q, int H_kv) {
   return w;
 }
 
-// Means and per-tensor scale of one tensor [B, N, H, 128].
-mpfa_status tensor_stats(const __nv_bfloat16 *x, int B, int N, int H, bool smooth, double *sums, unsigned int *amax,
-                         float *mean, float *gscale, cudaStream_t st) {
+// Means and per-tensor scale of one tensor [B, N, H, 128]: one pass over the data.
+mpfa_status tensor_stats(const __nv_bfloat16 *x, int B, int N, int H, bool smooth, double *sums, unsigned int *kmax,
+                         unsigned int *knegmax, unsigned int *amax, float *mean, float *gscale, cudaStream_t st) {
   const int cols = H * HEAD_DIM;
-  dim3 grid((N + TOK_PER_BLOCK - 1) / TOK_PER_BLOCK, (cols + COLS_PER_BLOCK - 1) / COLS_PER_BLOCK, B);
-  if (smooth) {
-    colsum_kernel<<<grid, 256, 0, st>>>(x, N, cols, sums);
-    MPFA_LAUNCH_OK();
-    finalize_mean_kernel<<<(B * cols + 255) / 256, 256, 0, st>>>(sums, B * cols, N, mean);
-    MPFA_LAUNCH_OK();
-  } else {
-    MPFA_CUDA_OK(cudaMemsetAsync(mean, 0, (size_t)B * cols * sizeof(float), st));
-  }
-  amax_kernel<<<grid, 256, 0, st>>>(x, mean, N, cols, amax);
+  dim3 grid((N + COLSTAT_TOKENS - 1) / COLSTAT_TOKENS, (cols + COLSTAT_COLS - 1) / COLSTAT_COLS, B);
+  colstat_kernel<<<grid, 256, 0, st>>>(x, N, cols, sums, kmax, knegmax);
+  MPFA_LAUNCH_OK();
+  finalize_stats_kernel<<<dim3((cols + 255) / 256, B), 256, 0, st>>>(sums, kmax, knegmax, cols, N, smooth ? 1 : 0, mean,
+                                                                    amax);
   MPFA_LAUNCH_OK();
   finalize_scale_kernel<<<(B + 127) / 128, 128, 0, st>>>(amax, B, gscale);
   MPFA_LAUNCH_OK();
@@ -407,11 +453,11 @@ extern "C" mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, 
   if (!frozen) {
     MPFA_CUDA_OK(cudaMemsetAsync(workspace, 0, w.bytes, s));
     if (q) {
-      rc = tensor_stats(q, B, N_q, H_q, smooth, w.sums_q, w.amax_q, st->q_mean, st->q_gscale, s);
+      rc = tensor_stats(q, B, N_q, H_q, smooth, w.sums_q, w.max_q, w.neg_q, w.amax_q, st->q_mean, st->q_gscale, s);
       if (rc != MPFA_OK) return rc;
     }
     if (k) {
-      rc = tensor_stats(k, B, N_kv, H_kv, smooth, w.sums_k, w.amax_k, st->k_mean, st->k_gscale, s);
+      rc = tensor_stats(k, B, N_kv, H_kv, smooth, w.sums_k, w.max_k, w.neg_k, w.amax_k, st->k_mean, st->k_gscale, s);
       if (rc != MPFA_OK) return rc;
     }
   }
@@ -478,7 +524,7 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
   const __nv_bfloat16 *v = static_cast<const __nv_bfloat16 *>(v_bf16);
   if (!frozen) {
     MPFA_CUDA_OK(cudaMemsetAsync(workspace, 0, w.bytes, s));
-    rc = tensor_stats(k, 1, N_tokens, H_kv, smooth, w.sums_k, w.amax_k, st->k_mean, st->k_gscale, s);
+    rc = tensor_stats(k, 1, N_tokens, H_kv, smooth, w.sums_k, w.max_k, w.neg_k, w.amax_k, st->k_mean, st->k_gscale, s);
     if (rc != MPFA_OK) return rc;
   }
   const int n_pages = (N_tokens + PAGE - 1) / PAGE;
