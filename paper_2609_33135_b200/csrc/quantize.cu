@@ -227,28 +227,41 @@ __global__ void __launch_bounds__(128) delta_s_kernel(const __nv_bfloat16 *__res
                                                       const int32_t *__restrict__ page_row, int num_pages) {
   constexpr int MAXG = 8;
   __shared__ float kmu[HEAD_DIM];
-  __shared__ float qmu[MAXG][HEAD_DIM];
+  __shared__ double qmu[MAXG][HEAD_DIM];   // converted once: the conversion is as costly as the FMA
   const int tile = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int G = H_q / H_kv;
   const int n_pad = gridDim.x * TILE;
   kmu[threadIdx.x] = k_mean[((size_t)b * H_kv + hk) * HEAD_DIM + threadIdx.x];
-  for (int g = 0; g < G; ++g) qmu[g][threadIdx.x] = q_mean[((size_t)b * H_q + hk * G + g) * HEAD_DIM + threadIdx.x];
+  for (int g = 0; g < G; ++g) qmu[g][threadIdx.x] = (double)q_mean[((size_t)b * H_q + hk * G + g) * HEAD_DIM + threadIdx.x];
+  __syncthreads();
+  // The tile's K rows are staged in shared memory with coalesced 16-byte loads (a row is 256 contiguous
+  // bytes, rows of one head are H_kv * 256 bytes apart); each thread then walks its own row.  Row pitch
+  // 272 bytes: the 16-byte reads of 8 consecutive threads fall into 8 different bank groups.
+  constexpr int PITCH = 272;
+  __shared__ __align__(16) uint8_t rows[TILE * PITCH];
+  for (int i = threadIdx.x; i < TILE * 16; i += 128) {
+    const int r = i >> 4, ch = i & 15;
+    const int tt = tile * TILE + r;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (tt < N) v = *reinterpret_cast<const uint4 *>(k + (((size_t)b * N + tt) * H_kv + hk) * HEAD_DIM + ch * 8);
+    *reinterpret_cast<uint4 *>(rows + r * PITCH + ch * 16) = v;
+  }
   __syncthreads();
   const int t = tile * TILE + threadIdx.x;
   double acc[MAXG];
 #pragma unroll
   for (int g = 0; g < MAXG; ++g) acc[g] = 0.0;
   if (t < N) {
-    const __nv_bfloat16 *row = k + (((size_t)b * N + t) * H_kv + hk) * HEAD_DIM;
+    const uint8_t *row = rows + threadIdx.x * PITCH;
     for (int c0 = 0; c0 < HEAD_DIM; c0 += 8) {
       float f[8];
-      unpack8(*reinterpret_cast<const uint4 *>(row + c0), f);
+      unpack8(*reinterpret_cast<const uint4 *>(row + c0 * 2), f);
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const double kc = (double)__fsub_rn(f[i], kmu[c0 + i]);
 #pragma unroll
         for (int g = 0; g < MAXG; ++g)
-          if (g < G) acc[g] = fma((double)qmu[g][c0 + i], kc, acc[g]);
+          if (g < G) acc[g] = fma(qmu[g][c0 + i], kc, acc[g]);
       }
     }
   }
