@@ -96,13 +96,24 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def dist_setup(n):
+_DIST_DEVICE = "cuda"   # where the rank-to-rank reductions live: "cuda" under NCCL, "cpu" under gloo
+
+
+def dist_setup(n, backend="nccl"):
+    """One process per GPU, rendezvous from the torchrun environment.  `backend="gloo"` runs the same
+    rank plumbing on CPU (used by the multi-rank tests; the data path itself has no collective)."""
+    global _DIST_DEVICE
     if n <= 1:
         return 0, 1, 0
     import torch.distributed as dist
     rank, world, local = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"]), int(os.environ.get("LOCAL_RANK", 0))
-    torch.cuda.set_device(local)
-    dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if backend == "nccl":
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        _DIST_DEVICE = "cuda"
+    else:
+        dist.init_process_group(backend)
+        _DIST_DEVICE = "cpu"
     return rank, world, local
 
 
@@ -110,16 +121,28 @@ def barrier(world):
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    torch.cuda.synchronize()
+    if _DIST_DEVICE == "cuda" and torch.cuda.is_available():
+        torch.cuda.synchronize()
 
 
 def max_over_ranks(x: float, world) -> float:
     if world <= 1:
         return x
     import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    t = torch.tensor([x], dtype=torch.float64, device=_DIST_DEVICE)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def whole_job_value(world: int, flops_per_rank: float, ms_per_step: float) -> float:
+    """Weak scaling: every rank runs its own batch element; the job's TFLOPS is the work of all ranks over
+    the slowest rank's time."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Batch element of a rank: rank r takes element r of a global batch (distinct seeds, same shape)."""
+    return base_seed + 100 * rank
 
 
 # ------------------------------------------------------------------------------------------
@@ -200,7 +223,7 @@ def run_ours(args, rank, world, local):
     peaks = load_peaks()
     dev = torch.device("cuda", local)
     N = args.seq_len
-    w = wl.config2_llama(N)
+    w = wl.config2_llama(N, seed=rank_seed(1002, rank))   # rank r: batch element r
     hq, hk, hv = w.q.pin_memory(), w.k.pin_memory(), w.v.pin_memory()
     q, k, v = hq.to(dev), hk.to(dev), hv.to(dev)
     s1 = binding.stage1(q, k, v)           # allocates outputs once; steps reuse them
@@ -263,7 +286,7 @@ def run_ours(args, rank, world, local):
     _ = float(host_out[0, 0, 0, 0])  # the host reads the result
 
     flops = w.flops
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    value = whole_job_value(world, flops, ms_step)
     long_run = total_ms > 2000.0
     bf16_peak = peaks["bf16_sustained"] if long_run else peaks["bf16"]
     peak = bf16_peak * MIXED_OVER_BF16
@@ -277,7 +300,7 @@ def run_ours(args, rank, world, local):
                    "l2": "inputs_exceed_l2 (Q+K+V 201 MB, output 134 MB per step vs 126 MB L2)",
                    "step": "quantize_qk + quantize_v + prefill"},
         "clocks": clocks,
-        "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOPS", "ms_per_step": e2e_ms,
+        "e2e": {"value": whole_job_value(world, flops, e2e_ms), "unit": "TFLOPS", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": (q.numel() + k.numel() + v.numel()) * 2, "d2h_bytes_per_step": out.numel() * 2},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": {"kernel": "prefill_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,

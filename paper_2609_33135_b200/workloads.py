@@ -117,8 +117,9 @@ def config1b_tiny_qbias() -> PrefillWorkload:
     return prefill_workload("cfg1b_tiny_qbias_256", 1011, 1, 256, 1, 1, False, n_outlier=4, q_bias=True)
 
 
-def config2_llama(N: int = 16384) -> PrefillWorkload:
-    return prefill_workload(f"cfg2_llama8b_causal_{N}", 1002, 1, N, 32, 8, True)
+def config2_llama(N: int = 16384, seed: int = 1002) -> PrefillWorkload:
+    """`seed` selects the batch element (data-parallel ranks take different elements of the same shape)."""
+    return prefill_workload(f"cfg2_llama8b_causal_{N}", seed, 1, N, 32, 8, True)
 
 
 def config3_qwen(N: int = 32768) -> PrefillWorkload:

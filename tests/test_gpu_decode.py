@@ -70,14 +70,47 @@ def compare(st, ref32):
     assert bf16_neighbours_ok(g16, ref32).all()
 
 
-@pytest.mark.parametrize("hq,hkv", [(8, 2), (10, 2), (4, 4)])
-def test_decode_matches_oracle(hq, hkv):
+@pytest.mark.parametrize("hq,hkv", [(8, 2), (10, 2), (4, 4), (4, 2), (6, 2), (12, 2), (14, 2), (16, 2)])
+def test_decode_matches_oracle(hq, hkv):   # every GQA group size 1..8 (the kernel is specialised on it)
     # lengths that hit the edges: one key, one page, one block + 1, one partition + 1, ragged multi-partition
     w = wl.decode_workload("dec_small", 61 + hq, 5, hq, hkv, 1, 2600, seq_lens=[1, 64, 129, 1025, 2600])
     ref32, ref16, caches = oracle_decode(w)
     st = run(w)
     check_cache(st, w, caches)
     compare(st, ref32)
+
+
+def oracle_decode_one(w, b):
+    k, v = w.kv_for_request(b)
+    z = orc.stage1(orc.bf16_bits(w.q_sample[b:b + 1].contiguous()), orc.bf16_bits(k), orc.bf16_bits(v))
+    zq = orc.stage1(orc.bf16_bits(w.q_new[b:b + 1].contiguous()), orc.bf16_bits(k), orc.bf16_bits(v), frozen=z)
+    o32, _ = orc.decode(zq.q_codes[:, :, 0], zq.q_sf[:, :, 0], z.k_codes, z.k_sf, z.v_codes, z.delta, z.dq, z.dk, 1.0,
+                        w.softmax_scale, np.array([int(w.seq_lens[b])], np.int32))
+    return o32[0]
+
+
+def test_decode_many_short_requests():
+    """More requests than the kernel caches lengths for (768), far more work items than CTAs, most of them
+    a single partial block: the persistent work walk, the item-boundary hand-offs and the table fallback."""
+    B = 800
+    w = wl.decode_workload("dec_many", 75, B, 4, 2, 1, 200, n_stat_tokens=64)
+    st = run(w)
+    got = st.out_f32.cpu().numpy()
+    assert np.isfinite(got).all()
+    for b in list(range(0, B, 37)) + [767, 768, 769, B - 1]:
+        d = np.abs(got[b] - oracle_decode_one(w, b))
+        assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (b, float(d.max()), float(d.mean()))
+
+
+def test_decode_long_request_many_partitions():
+    """One request of 20 partitions next to a one-token request: many items per (request, head), merge kernel
+    over many partition states."""
+    w = wl.decode_workload("dec_long", 76, 2, 8, 2, 1, 20000, seq_lens=[19999, 1])
+    st = run(w)
+    got = st.out_f32.cpu().numpy()
+    for b in range(2):
+        d = np.abs(got[b] - oracle_decode_one(w, b))
+        assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (b, float(d.max()), float(d.mean()))
 
 
 def test_decode_direct_variant_and_v_scale():
