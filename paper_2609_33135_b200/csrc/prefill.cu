@@ -47,20 +47,21 @@ constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM clock
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;       // drain path only
 constexpr int NTHREADS = 512;
 
-constexpr uint32_t OFF_Q = 0;
-constexpr uint32_t OFF_K = OFF_Q + 8192;
+constexpr uint32_t OFF_Q = 0;                               // 2 tiles (the next tile's queries are prefetched)
+constexpr uint32_t OFF_K = OFF_Q + 2 * 8192;
 constexpr uint32_t OFF_V = OFF_K + KSTAGES * 8192;
 constexpr uint32_t OFF_DELTA = OFF_V + VSTAGES * 16384;
 constexpr uint32_t OFF_ONES = OFF_DELTA + KSTAGES * 4096;
 constexpr uint32_t OFF_SFQ = OFF_ONES + 4096;
-constexpr uint32_t OFF_SFK = OFF_SFQ + 1024;
+constexpr uint32_t OFF_SFK = OFF_SFQ + 2 * 1024;
 constexpr uint32_t OFF_ALPHA = OFF_SFK + KSTAGES * 1024;   // alpha[2][128]
 constexpr uint32_t OFF_M = OFF_ALPHA + 2 * 128 * 4;        // running maximum after block t, [t & 1][128]
-constexpr uint32_t OFF_L = OFF_M + 2 * 128 * 4;            // final (l, m) of the two softmax groups, [2][2][128]
-constexpr uint32_t OFF_BAR = OFF_L + 4 * 128 * 4;
+constexpr uint32_t OFF_L = OFF_M + 2 * 128 * 4;            // final (l, m) of the two softmax groups, [item & 3][2][2][128]
+constexpr uint32_t OFF_BAR = OFF_L + 4 * 4 * 128 * 4;
 enum {
-  BAR_Q_FULL = 0,
-  BAR_K_FULL = 1,
+  BAR_Q_FULL = 0,                       // [2] query tile of work item i in buffer i & 1
+  BAR_Q_EMPTY = 2,                      // [2] every Q K^T MMA of that work item has completed
+  BAR_K_FULL = 4,
   BAR_K_EMPTY = BAR_K_FULL + KSTAGES,
   BAR_V_FULL = BAR_K_EMPTY + KSTAGES,
   BAR_V_EMPTY = BAR_V_FULL + VSTAGES,
@@ -72,14 +73,18 @@ enum {
   BAR_M_FULL = BAR_P_EMPTY + 2,         // [2] running maximum and alpha of block t published
   BAR_O_FULL = BAR_M_FULL + 2,          // [2] P V of block t accumulated into O[t & 1]
   BAR_O_READY = BAR_O_FULL + 2,         // [2] O[t & 1] rescaled for block t
-  BAR_L_FULL = BAR_O_READY + 2,
-  NUM_BARS = BAR_L_FULL + 1
+  BAR_L_FULL = BAR_O_READY + 2,         // [4] row sums of work item i published, slot i & 3.  The softmax warps can
+                                        //     be at most three (one-block) items ahead of the epilogue - P_hat of
+                                        //     block c needs P V of block c-2, which needs the correction warps - so
+                                        //     a slot is never two phases ahead of its reader
+  BAR_O_FREE = BAR_L_FULL + 4,          // the epilogue has read both accumulators (phase = items with T > 0)
+  NUM_BARS = BAR_O_FREE + 1
 };
 constexpr uint32_t OFF_MISC = OFF_BAR + NUM_BARS * 8;   // tmem base, abort flag
 constexpr uint32_t SMEM_BYTES = OFF_MISC + 16 + 1024;   // + slack for the 1024-byte alignment
 
-constexpr uint32_t TM_S = 0, TM_O0 = 128, TM_O1 = 256, TM_P0 = 384, TM_P1 = 416, TM_SFQ = 448, TM_SFK0 = 456,
-                   TM_SFK1 = 464;
+constexpr uint32_t TM_S = 0, TM_O0 = 128, TM_O1 = 256, TM_P0 = 384, TM_P1 = 416, TM_SFQ = 448 /* 2 x 8 */,
+                   TM_SFK0 = 464, TM_SFK1 = 472;
 constexpr uint32_t TMEM_COLS = 512;
 
 struct PrefillParams {
@@ -91,7 +96,7 @@ struct PrefillParams {
   __nv_bfloat16 *out;
   float *out_f32;  // may be null
   int32_t *status;
-  int B, N_q, N_kv, H_q, H_kv, nq_tiles, nk_tiles;
+  int B, N_q, N_kv, H_q, H_kv, nq_tiles, nk_tiles, n_items;
   int causal;
   float softmax_scale, v_scale;
 };
@@ -188,6 +193,37 @@ struct Ctx {
   }
 };
 
+// One work item: a 128-row query tile of one q head.
+struct Tile {
+  int b, hq, hk, qt, row0, T;   // T: KV blocks to visit
+};
+
+// The list of work items of this CTA.  Items are ordered by length (latest query tile first; all heads of a
+// tile adjacent, so the G heads of a kv head stream the same K/V through L2 together) and dealt to the CTAs
+// boustrophedon: round r goes 0..n-1, round r+1 goes n-1..0.  For a causal 16K problem on 148 CTAs the
+// heaviest CTA gets 0.15 % more blocks than the mean (plain round-robin: 7 %).
+struct TileWalk {
+  int round;   // everything else is read from the kernel parameters (constant bank), not kept in registers
+  __device__ __forceinline__ void init() { round = 0; }
+  __device__ __forceinline__ bool next(const PrefillParams &pp, Tile &t) {
+    const int c = (round & 1) ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
+    const int i = round * (int)gridDim.x + c;
+    ++round;
+    if (i >= pp.n_items) return false;
+    const int n_heads = pp.B * pp.H_q;
+    t.qt = pp.nq_tiles - 1 - i / n_heads;
+    const int h = i % n_heads;
+    t.b = h / pp.H_q;
+    t.hq = h % pp.H_q;
+    t.hk = t.hq / (pp.H_q / pp.H_kv);
+    t.row0 = t.qt * TILE;
+    const int last_row = min(pp.N_q - 1, t.row0 + TILE - 1);
+    const int last_key = pp.causal ? min(pp.N_kv - 1, last_row + (pp.N_kv - pp.N_q)) : pp.N_kv - 1;   // bottom-right aligned
+    t.T = last_key < 0 ? 0 : last_key / TILE + 1;
+    return true;
+  }
+};
+
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const PrefillParams p) {
@@ -195,24 +231,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-  // ---- work item: kv head outermost so co-resident CTAs share K/V through L2; within a
-  // head the longest (latest) query tiles first, the GQA group innermost.
-  const int G = p.H_q / p.H_kv;
-  int w = blockIdx.x;
-  const int g = w % G;
-  w /= G;
-  const int qt = p.nq_tiles - 1 - (w % p.nq_tiles);
-  w /= p.nq_tiles;
-  const int hk = w % p.H_kv;
-  const int b = w / p.H_kv;
-  const int hq = hk * G + g;
-
-  const int off = p.N_kv - p.N_q;   // causal masks are bottom-right aligned
-  const int row0 = qt * TILE;
-  const int last_row = min(p.N_q - 1, row0 + TILE - 1);
-  const int last_key = p.causal ? min(p.N_kv - 1, last_row + off) : p.N_kv - 1;
-  const int T = last_key < 0 ? 0 : last_key / TILE + 1;   // KV blocks to visit
 
 #ifdef MPFA_TRACE
   if ((int)blockIdx.x == g_trace_cta && tid == 12 * 32 && g_trace) g_trace[((0) * 256 + 255) * 8 + 1] = clock64();   // kernel entry
@@ -226,7 +244,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   // ---- one-time setup
   if (tid == 0) {
     *cx.abort_flag = 0;
-    mbar_init(cx.bar(BAR_Q_FULL), 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(cx.bar(BAR_Q_FULL + i), 1); mbar_init(cx.bar(BAR_Q_EMPTY + i), 1); }
     for (int i = 0; i < KSTAGES; ++i) { mbar_init(cx.bar(BAR_K_FULL + i), 1); mbar_init(cx.bar(BAR_K_EMPTY + i), 1); }
     for (int i = 0; i < VSTAGES; ++i) { mbar_init(cx.bar(BAR_V_FULL + i), 1); mbar_init(cx.bar(BAR_V_EMPTY + i), 1); }
     mbar_init(cx.bar(BAR_S_FULL), 1);
@@ -239,7 +257,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_init(cx.bar(BAR_O_FULL + i), 1);
       mbar_init(cx.bar(BAR_O_READY + i), 4);
     }
-    mbar_init(cx.bar(BAR_L_FULL), 8);
+    for (int i = 0; i < 4; ++i) mbar_init(cx.bar(BAR_L_FULL + i), 8);
+    mbar_init(cx.bar(BAR_O_FREE), 4);
     mbar_init_fence();
     prefetch_tmap(&tm_q);
     prefetch_tmap(&tm_k);
@@ -264,128 +283,157 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const bool has_delta = p.delta != nullptr;
   TR_INIT();
   if (warp == 12) TR(0, 255, 2);   // roles start (after setup)
-  const size_t q_row = ((size_t)b * p.H_q + hq) * (size_t)(p.nq_tiles * TILE) + row0;
-  const size_t k_row = ((size_t)b * p.H_kv + hk) * (size_t)(p.nk_tiles * TILE);
+
+  // Every role walks the same list of work items (q tile x q head) and keeps the same running count of
+  // KV blocks; ring slots and barrier phases are functions of those two counters, so the pipeline runs
+  // straight through item boundaries: the next item's Q/K/V arrive and its first scores are computed while
+  // the correction warps write the previous item's output.
+  TileWalk walk;
+  walk.init();
+  Tile tl;
+  uint32_t gb = 0;   // KV blocks of the items already walked
+  uint32_t ti = 0;   // index of the current item in this CTA's list
 
   if (warp < 4) setmaxnreg_dec<88>();
   if (warp == 0) {
     // =========================== TMA producer ===========================
     // The whole warp runs the loop (uniform control flow keeps addresses and barrier handles in
     // uniform registers); a single elected lane issues each copy.
-    if (T > 0) {
-      int armed = 0;
+    bool ok = true;
+    uint32_t nk_armed = 0, nv_armed = 0, nq_armed = 0;
+    for (; ok && walk.next(p, tl); gb += tl.T, ++ti) {
+      const uint32_t qb = ti & 1;
+      if (ti >= 2) ok = cx.wait(BAR_Q_EMPTY + qb, ((ti >> 1) - 1) & 1u);
+      if (!ok) break;
+      const size_t q_row = ((size_t)tl.b * p.H_q + tl.hq) * (size_t)(p.nq_tiles * TILE) + tl.row0;
+      const size_t k_row = ((size_t)tl.b * p.H_kv + tl.hk) * (size_t)(p.nk_tiles * TILE);
       if (elect_one()) {
-        mbar_expect_tx(cx.bar(BAR_Q_FULL), 8192 + 1024);
-        tma_load_2d(sbase + OFF_Q, &tm_q, 0, (int)q_row, cx.bar(BAR_Q_FULL));
-        bulk_load(sbase + OFF_SFQ, p.q_sf + (((size_t)b * p.H_q + hq) * p.nq_tiles + qt) * 1024, 1024,
-                  cx.bar(BAR_Q_FULL));
+        mbar_expect_tx(cx.bar(BAR_Q_FULL + qb), 8192 + 1024);
+        tma_load_2d(sbase + OFF_Q + qb * 8192, &tm_q, 0, (int)q_row, cx.bar(BAR_Q_FULL + qb));
+        bulk_load(sbase + OFF_SFQ + qb * 1024, p.q_sf + (((size_t)tl.b * p.H_q + tl.hq) * p.nq_tiles + tl.qt) * 1024, 1024,
+                  cx.bar(BAR_Q_FULL + qb));
       }
-      bool ok = true;
-      for (int t = 0; t < T && ok; ++t) {
-        const int jb = T - 1 - t;
-        const int ks = t % KSTAGES, vs = t % VSTAGES;
-        if (t >= KSTAGES) ok = cx.wait(BAR_K_EMPTY + ks, (uint32_t)(t / KSTAGES - 1) & 1u);
+      nq_armed = ti + 1;
+      for (int t = 0; t < tl.T && ok; ++t) {
+        const uint32_t c = gb + t;
+        const int jb = tl.T - 1 - t;
+        const uint32_t ks = c % KSTAGES, vs = c % VSTAGES;
+        if (c >= (uint32_t)KSTAGES) ok = cx.wait(BAR_K_EMPTY + ks, (c / KSTAGES - 1) & 1u);
         if (!ok) break;
-        TR(0, t, 0);
+        TR(0, c, 0);
         if (elect_one()) {
           mbar_expect_tx(cx.bar(BAR_K_FULL + ks), 8192 + 1024 + (has_delta ? 256 : 0));
           tma_load_2d(sbase + OFF_K + ks * 8192, &tm_k, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_K_FULL + ks));
-          bulk_load(sbase + OFF_SFK + ks * 1024, p.k_sf + (((size_t)b * p.H_kv + hk) * p.nk_tiles + jb) * 1024, 1024,
+          bulk_load(sbase + OFF_SFK + ks * 1024, p.k_sf + (((size_t)tl.b * p.H_kv + tl.hk) * p.nk_tiles + jb) * 1024, 1024,
                     cx.bar(BAR_K_FULL + ks));
           if (has_delta) {
-            const __nv_bfloat16 *d = p.delta + ((size_t)b * p.H_q + hq) * (size_t)(p.nk_tiles * TILE) + (size_t)jb * TILE;
+            const __nv_bfloat16 *d = p.delta + ((size_t)tl.b * p.H_q + tl.hq) * (size_t)(p.nk_tiles * TILE) + (size_t)jb * TILE;
             bulk_load(sbase + OFF_DELTA + ks * 4096, d, 128, cx.bar(BAR_K_FULL + ks));
             bulk_load(sbase + OFF_DELTA + ks * 4096 + 2048, d + 64, 128, cx.bar(BAR_K_FULL + ks));
           }
         }
-        if (t >= VSTAGES) ok = cx.wait(BAR_V_EMPTY + vs, (uint32_t)(t / VSTAGES - 1) & 1u);
-        if (!ok) { armed = -(t + 1); break; }   // K of block t armed, V not
-        TR(0, t, 1);
+        nk_armed = c + 1;
+        if (c >= (uint32_t)VSTAGES) ok = cx.wait(BAR_V_EMPTY + vs, (c / VSTAGES - 1) & 1u);
+        if (!ok) break;
+        TR(0, c, 1);
         if (elect_one()) {
           mbar_expect_tx(cx.bar(BAR_V_FULL + vs), 16384);
           tma_load_2d(sbase + OFF_V + vs * 16384, &tm_v, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
         }
-        armed = t + 1;
+        nv_armed = c + 1;
       }
-      if (*cx.abort_flag) {
-        // Drain: copies still in flight must land before the CTA's shared memory is released.
-        const int nk = armed < 0 ? -armed : armed, nv = armed < 0 ? -armed - 1 : armed;
-        for (int t = max(0, nk - KSTAGES); t < nk; ++t)
-          mbar_wait_ns(cx.bar(BAR_K_FULL + t % KSTAGES), (uint32_t)(t / KSTAGES) & 1u, WAIT_LIMIT_NS);
-        for (int t = max(0, nv - VSTAGES); t < nv; ++t)
-          mbar_wait_ns(cx.bar(BAR_V_FULL + t % VSTAGES), (uint32_t)(t / VSTAGES) & 1u, WAIT_LIMIT_NS);
-        mbar_wait_ns(cx.bar(BAR_Q_FULL), 0, WAIT_LIMIT_NS);
-      }
+    }
+    if (*cx.abort_flag) {
+      // Drain: copies still in flight must land before the CTA's shared memory is released.
+      for (uint32_t c = nk_armed - min(nk_armed, (uint32_t)KSTAGES); c < nk_armed; ++c)
+        mbar_wait_ns(cx.bar(BAR_K_FULL + c % KSTAGES), (c / KSTAGES) & 1u, WAIT_LIMIT_NS);
+      for (uint32_t c = nv_armed - min(nv_armed, (uint32_t)VSTAGES); c < nv_armed; ++c)
+        mbar_wait_ns(cx.bar(BAR_V_FULL + c % VSTAGES), (c / VSTAGES) & 1u, WAIT_LIMIT_NS);
+      for (uint32_t i = nq_armed - min(nq_armed, 2u); i < nq_armed; ++i)
+        mbar_wait_ns(cx.bar(BAR_Q_FULL + (i & 1)), (i >> 1) & 1u, WAIT_LIMIT_NS);
     }
   } else if (warp == 1) {
     // =========================== Q K^T issuer ===========================
     // Whole warp in uniform control flow; lane 0 (always the elected lane of a full warp) issues
     // every tcgen05 instruction, so the commits track the MMAs of the same thread.  This warp
     // only waits for operands (K block in shared memory, score buffer handed back by its
-    // softmax group), so it runs up to two blocks ahead of the P V issuer (warp 3).
-    if (T > 0) {
-      const uint32_t id_fp4 = idesc_nvfp4(128, 128);
-      const uint32_t id_bf16 = idesc_bf16(128, 128, 1, 1);
-      // All shared-memory descriptors are built once; a ring stage or K step only adds a
-      // constant to the 14-bit start-address field (shared addresses stay below 256 KB).
-      const uint64_t d_ones = smem_desc(sbase + OFF_ONES, 2048, 1024, SWZ_128B);
-      const uint64_t d_delta0 = smem_desc(sbase + OFF_DELTA, 2048, 1024, SWZ_128B);
-      const uint64_t d_q0 = smem_desc(sbase + OFF_Q, 16, 512, SWZ_64B);
-      const uint64_t d_k0 = smem_desc(sbase + OFF_K, 16, 512, SWZ_64B);
-      const uint64_t d_sfq0 = smem_desc(sbase + OFF_SFQ, 0, 128, SWZ_NONE);
-      const uint64_t d_sfk0 = smem_desc(sbase + OFF_SFK, 0, 128, SWZ_NONE);
-      bool ok = cx.wait(BAR_Q_FULL, 0);
-      if (ok) {
-        tc_fence_after();
-        if (elect_one()) {
-          tmem_cp_32x128b_warpx4(tm + TM_SFQ, d_sfq0);
-          tmem_cp_32x128b_warpx4(tm + TM_SFQ + 4, d_sfq0 + (512 >> 4));
-        }
+    // softmax group), so it runs ahead of the P V issuer (warp 3), also into the next work item.
+    const uint32_t id_fp4 = idesc_nvfp4(128, 128);
+    const uint32_t id_bf16 = idesc_bf16(128, 128, 1, 1);
+    // All shared-memory descriptors are built once; a ring stage or K step only adds a
+    // constant to the 14-bit start-address field (shared addresses stay below 256 KB).
+    const uint64_t d_ones = smem_desc(sbase + OFF_ONES, 2048, 1024, SWZ_128B);
+    const uint64_t d_delta0 = smem_desc(sbase + OFF_DELTA, 2048, 1024, SWZ_128B);
+    const uint64_t d_q00 = smem_desc(sbase + OFF_Q, 16, 512, SWZ_64B);
+    const uint64_t d_k0 = smem_desc(sbase + OFF_K, 16, 512, SWZ_64B);
+    const uint64_t d_sfq00 = smem_desc(sbase + OFF_SFQ, 0, 128, SWZ_NONE);
+    const uint64_t d_sfk0 = smem_desc(sbase + OFF_SFK, 0, 128, SWZ_NONE);
+    bool ok = true;
+    for (; ok && walk.next(p, tl); gb += tl.T, ++ti) {
+      const uint32_t qb = ti & 1;
+      ok = cx.wait(BAR_Q_FULL + qb, (ti >> 1) & 1u);
+      if (!ok) break;
+      const uint64_t d_q0 = d_q00 + (uint64_t)((qb * 8192) >> 4);
+      const uint32_t tSFQ = tm + TM_SFQ + qb * 8;
+      tc_fence_after();
+      if (elect_one()) {
+        const uint64_t d_sfq0 = d_sfq00 + (uint64_t)((qb * 1024) >> 4);
+        tmem_cp_32x128b_warpx4(tSFQ, d_sfq0);
+        tmem_cp_32x128b_warpx4(tSFQ + 4, d_sfq0 + (512 >> 4));
       }
-      for (int t = 0; t < T && ok; ++t) {
-        const int ks = t % KSTAGES, sb = t & 1;
-        TR(5, t, 0);
-        ok = cx.wait(BAR_K_FULL + ks, (uint32_t)(t / KSTAGES) & 1u);
+      for (int t = 0; t < tl.T && ok; ++t) {
+        const uint32_t c = gb + t;
+        const uint32_t ks = c % KSTAGES, sb = c & 1;
+        TR(5, c, 0);
+        ok = cx.wait(BAR_K_FULL + ks, (c / KSTAGES) & 1u);
         if (!ok) break;
         const uint32_t tSFK = tm + (sb ? TM_SFK1 : TM_SFK0);
         const uint64_t d_sfk = d_sfk0 + (uint64_t)((ks * 1024) >> 4);
         const uint64_t d_k = d_k0 + (uint64_t)((ks * 8192) >> 4);
         const uint64_t d_delta = d_delta0 + (uint64_t)((ks * 4096) >> 4);
         tc_fence_after();
-        if (elect_one()) {   // scale factors first: their TMEM columns were last used by block t-2
+        if (elect_one()) {   // scale factors first: their TMEM columns were last used by block c-2
           tmem_cp_32x128b_warpx4(tSFK, d_sfk);
           tmem_cp_32x128b_warpx4(tSFK + 4, d_sfk + (512 >> 4));
         }
-        // the softmax group of block t-1 has read its scores out of the buffer
-        if (t >= 1) ok = cx.wait(BAR_S_EMPTY, (uint32_t)(t - 1) & 1u);
+        // the softmax group of block c-1 has read its scores out of the buffer
+        if (c >= 1) ok = cx.wait(BAR_S_EMPTY, (c - 1) & 1u);
         if (!ok) break;
-        TR(5, t, 1);
+        TR(5, c, 1);
         tc_fence_after();
         if (elect_one()) {
           if (has_delta) mma_bf16_ss(tm + TM_S, d_ones, d_delta, id_bf16, 0);
-          mma_nvfp4_ss(tm + TM_S, d_q0, d_k, id_fp4, tm + TM_SFQ, tSFK, has_delta ? 1u : 0u);
-          mma_nvfp4_ss(tm + TM_S, d_q0 + (32 >> 4), d_k + (32 >> 4), id_fp4, tm + TM_SFQ + 4, tSFK + 4, 1u);
+          mma_nvfp4_ss(tm + TM_S, d_q0, d_k, id_fp4, tSFQ, tSFK, has_delta ? 1u : 0u);
+          mma_nvfp4_ss(tm + TM_S, d_q0 + (32 >> 4), d_k + (32 >> 4), id_fp4, tSFQ + 4, tSFK + 4, 1u);
           mma_commit(cx.bar(BAR_S_FULL + sb));
           mma_commit(cx.bar(BAR_K_EMPTY + ks));
         }
-        TR(5, t, 5);
+        TR(5, c, 5);
       }
+      if (ok && elect_one()) mma_commit(cx.bar(BAR_Q_EMPTY + qb));   // after every MMA that reads this query tile
+      __syncwarp();
     }
   } else if (warp == 3) {
     // =========================== P V issuer ===========================
-    if (T > 0) {
-      const uint32_t id_fp8 = idesc_e4m3(128, 128, 0, 1);
-      const uint64_t d_v0 = smem_desc(sbase + OFF_V, 16, 1024, SWZ_128B);
-      bool ok = true;
-      for (int t = 0; t < T && ok; ++t) {
-        TR(1, t, 0);
-        const int sb = t & 1, vs = t % VSTAGES;
-        ok = cx.wait(BAR_V_FULL + vs, (uint32_t)(t / VSTAGES) & 1u);
-        TR(1, t, 1);
-        ok = ok && cx.wait(BAR_O_READY + sb, (uint32_t)(t >> 1) & 1u);
-        TR(1, t, 2);
-        ok = ok && cx.wait(BAR_P_FULL + sb, (uint32_t)(t >> 1) & 1u);
-        TR(1, t, 3);
+    const uint32_t id_fp8 = idesc_e4m3(128, 128, 0, 1);
+    const uint64_t d_v0 = smem_desc(sbase + OFF_V, 16, 1024, SWZ_128B);
+    bool ok = true;
+    uint32_t n_used = 0;   // items so far that used the accumulators (T > 0)
+    for (; ok && walk.next(p, tl); gb += tl.T, ++ti) {
+      if (tl.T == 0) continue;
+      // the previous such item's epilogue has read both accumulators
+      if (n_used >= 1) ok = cx.wait(BAR_O_FREE, (n_used - 1) & 1u);
+      ++n_used;
+      for (int t = 0; t < tl.T && ok; ++t) {
+        const uint32_t c = gb + t;
+        TR(1, c, 0);
+        const uint32_t sb = c & 1, vs = c % VSTAGES;
+        ok = cx.wait(BAR_V_FULL + vs, (c / VSTAGES) & 1u);
+        TR(1, c, 1);
+        ok = ok && cx.wait(BAR_O_READY + sb, (c >> 1) & 1u);
+        TR(1, c, 2);
+        ok = ok && cx.wait(BAR_P_FULL + sb, (c >> 1) & 1u);
+        TR(1, c, 3);
         if (!ok) break;
         tc_fence_after();
         const uint32_t tP = tm + (sb ? TM_P1 : TM_P0);
@@ -399,285 +447,289 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           mma_commit(cx.bar(BAR_P_EMPTY + sb));
           mma_commit(cx.bar(BAR_V_EMPTY + vs));
         }
-        TR(1, t, 5);
+        TR(1, c, 5);
       }
     }
   } else if (warp >= 4 && warp < 12) {
-    // =========================== softmax (two groups alternating over KV blocks) ===========
+    // =========================== softmax groups ===========================
     setmaxnreg_inc<168>();
-    const int grp = (warp - 4) >> 2;                 // 0: even blocks / S0, 1: odd blocks / S1
+    const int grp = (warp - 4) >> 2;                 // takes the KV blocks whose running count has this parity
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const int r_abs = row0 + row;
-    const int limit = p.causal ? min(p.N_kv - 1, r_abs + off) : p.N_kv - 1;   // last visible key
-    const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[b]), p.k_gscale[b]);
-    float m_own = -INFINITY;   // running maximum after this group's previous block
-    float l_own = 0.0f;        // sum of 448 P over this group's blocks, relative to m_own
+    const float *gq = p.q_gscale, *gk = p.k_gscale;
     float *s_m = reinterpret_cast<float *>(smem + OFF_M);
     const uint32_t tS = tm + TM_S + lane_off;
     const uint32_t tP = tm + (grp ? TM_P1 : TM_P0) + lane_off;
-    for (int t = grp; t < T; t += 2) {
-      const int key0 = (T - 1 - t) * TILE;
-      TR(2 + grp, t, 0);
-      if (!__all_sync(0xffffffffu, cx.wait(BAR_S_FULL + grp, (uint32_t)(t >> 1) & 1u))) break;
-      TR(2 + grp, t, 1);
-      tc_fence_after();
-      uint32_t s[128];
-      {
-        uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
-        uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
-        tmem_ld32(tS, s0);
-        tmem_ld32(tS + 32, s1);
-      }
-      // While the scores are on their way, test (without blocking) the two other conditions this
-      // block needs; the answers are consumed later, so their latency overlaps the TMEM load:
-      //  - P V of block t-2 has consumed this group's P_hat columns (this also means the
-      //    correction warps have read the maximum this group published two blocks ago);
-      //  - the other group's running maximum of block t-1 is published.
-      const uint32_t par_pe = (uint32_t)((t >> 1) - 1) & 1u, par_m = (uint32_t)((t - 1) >> 1) & 1u;
-      const bool pe_early = (t < 2) || cx.probe(BAR_P_EMPTY + grp, par_pe);
-      bool have_prev = (t == 0) || cx.probe(BAR_M_FULL + (grp ^ 1), par_m);
-      float m_prev = -INFINITY;
+    bool ok = true;
+    for (; ok && walk.next(p, tl); gb += tl.T, ++ti) {
+      const int T = tl.T;
+      const int r_abs = tl.row0 + row;
+      const int limit = p.causal ? min(p.N_kv - 1, r_abs + (p.N_kv - p.N_q)) : p.N_kv - 1;   // last visible key
+      const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), gq[tl.b]), gk[tl.b]);
+      float m_own = -INFINITY;   // running maximum after this group's previous block
+      float l_own = 0.0f;        // sum of 448 P over this group's blocks, relative to m_own
+      for (int t = (grp ^ (int)gb) & 1; t < T; t += 2) {
+        const uint32_t c = gb + t;
+        const int key0 = (T - 1 - t) * TILE;
+        TR(2 + grp, c, 0);
+        if (!__all_sync(0xffffffffu, cx.wait(BAR_S_FULL + grp, (c >> 1) & 1u))) { ok = false; break; }
+        TR(2 + grp, c, 1);
+        tc_fence_after();
+        uint32_t s[128];
+        {
+          uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
+          uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
+          tmem_ld32(tS, s0);
+          tmem_ld32(tS + 32, s1);
+        }
+        // While the scores are on their way, test (without blocking) the two other conditions this
+        // block needs; the answers are consumed later, so their latency overlaps the TMEM load:
+        //  - P V of block c-2 has consumed this group's P_hat columns (this also means the
+        //    correction warps have read the maximum this group published two blocks ago);
+        //  - the other group's running maximum of block c-1 (same item) is published.
+        const uint32_t par_pe = ((c >> 1) - 1) & 1u, par_m = ((c - 1) >> 1) & 1u;
+        const bool pe_early = (c < 2) || cx.probe(BAR_P_EMPTY + grp, par_pe);
+        bool have_prev = (t == 0) || cx.probe(BAR_M_FULL + (grp ^ 1), par_m);
+        float m_prev = -INFINITY;
 #ifdef MPFA_ABLATE_NO_MHAND
-      have_prev = true;
+        have_prev = true;
 #endif
-      const bool ragged = key0 + TILE - 1 > limit;   // diagonal / ragged block only
-      tmem_ld_wait();
-      {
-        // second half of the row in flight while the maximum of the first half is taken
-        uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
-        uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
-        tmem_ld32(tS + 64, s2);
-        tmem_ld32(tS + 96, s3);
-      }
-      if (ragged) {
+        const bool ragged = key0 + TILE - 1 > limit;   // diagonal / ragged block only
+        tmem_ld_wait();
+        {
+          // second half of the row in flight while the maximum of the first half is taken
+          uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
+          uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
+          tmem_ld32(tS + 64, s2);
+          tmem_ld32(tS + 96, s3);
+        }
+        if (ragged) {
 #pragma unroll
-        for (int i = 0; i < 64; ++i)
-          if (key0 + i > limit) s[i] = 0xFF800000u;   // -inf
-      }
-      // row maximum (Eq. 3)
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+          for (int i = 0; i < 64; ++i)
+            if (key0 + i > limit) s[i] = 0xFF800000u;   // -inf
+        }
+        // row maximum (Eq. 3)
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-      for (int i = 0; i < 64; i += 8) {
-        mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
-        mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
-        mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
-        mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
-      }
-      tmem_ld_wait();
-      tc_fence_before();
-      warp_arrive(cx.bar(BAR_S_EMPTY), lane);   // the row is in registers: Q K^T of block t+1 may overwrite it
-      TR(2 + grp, t, 2);
-      if (ragged) {
+        for (int i = 0; i < 64; i += 8) {
+          mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+          mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+          mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+          mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+        }
+        tmem_ld_wait();
+        tc_fence_before();
+        warp_arrive(cx.bar(BAR_S_EMPTY), lane);   // the row is in registers: Q K^T of block c+1 may overwrite it
+        TR(2 + grp, c, 2);
+        if (ragged) {
 #pragma unroll
-        for (int i = 64; i < 128; ++i)
-          if (key0 + i > limit) s[i] = 0xFF800000u;   // -inf
-      }
+          for (int i = 64; i < 128; ++i)
+            if (key0 + i > limit) s[i] = 0xFF800000u;   // -inf
+        }
 #pragma unroll
-      for (int i = 64; i < 128; i += 8) {
-        mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
-        mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
-        mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
-        mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
-      }
+        for (int i = 64; i < 128; i += 8) {
+          mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+          mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+          mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+          mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+        }
 #ifdef MPFA_ABLATE_NO_MAX
-      const float mx = fmaxf(__uint_as_float(s[0]), __uint_as_float(s[127])) + 30.0f;
+        const float mx = fmaxf(__uint_as_float(s[0]), __uint_as_float(s[127])) + 30.0f;
 #else
-      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
 #endif
-      // running maximum: the other group owns block t-1
-      if (!__all_sync(0xffffffffu, have_prev)) {
-        if (!__all_sync(0xffffffffu, cx.wait(BAR_M_FULL + (grp ^ 1), par_m))) break;
-      }
-      if (t > 0) m_prev = s_m[(grp ^ 1) * 128 + row];
+        // running maximum: the other group owns block c-1
+        if (!__all_sync(0xffffffffu, have_prev)) {
+          if (!__all_sync(0xffffffffu, cx.wait(BAR_M_FULL + (grp ^ 1), par_m))) { ok = false; break; }
+        }
+        if (t > 0) m_prev = s_m[(grp ^ 1) * 128 + row];
 #ifdef MPFA_ABLATE_NO_MHAND
-      m_prev = m_own;
+        m_prev = m_own;
 #endif
-      if (!__all_sync(0xffffffffu, pe_early)) {
-        if (!__all_sync(0xffffffffu, cx.wait(BAR_P_EMPTY + grp, par_pe))) break;
-      }
-      TR(2 + grp, t, 3);
-      const float m_t = fmaxf(m_prev, mx);
-      s_m[grp * 128 + row] = m_t;
-      warp_arrive(cx.bar(BAR_M_FULL + grp), lane);
-      TR(2 + grp, t, 4);
-      const float a_own = (m_t == m_own) ? 1.0f : ex2_approx(__fmul_rn(m_own - m_t, lam));
-      // P = 2^(lam S - lam m) (Eq. 4)
-      const float c = (m_t == -INFINITY) ? 0.0f : -__fmul_rn(m_t, lam);
-      float sum0 = 0.0f, sum1 = 0.0f, sum2 = 0.0f, sum3 = 0.0f;
+        if (!__all_sync(0xffffffffu, pe_early)) {
+          if (!__all_sync(0xffffffffu, cx.wait(BAR_P_EMPTY + grp, par_pe))) { ok = false; break; }
+        }
+        TR(2 + grp, c, 3);
+        const float m_t = fmaxf(m_prev, mx);
+        s_m[grp * 128 + row] = m_t;
+        warp_arrive(cx.bar(BAR_M_FULL + grp), lane);
+        TR(2 + grp, c, 4);
+        const float a_own = (m_t == m_own) ? 1.0f : ex2_approx(__fmul_rn(m_own - m_t, lam));
+        // P = 2^(lam S - lam m) (Eq. 4)
+        const float cc = (m_t == -INFINITY) ? 0.0f : -__fmul_rn(m_t, lam);
+        float sum0 = 0.0f, sum1 = 0.0f, sum2 = 0.0f, sum3 = 0.0f;
 #ifdef MPFA_ABLATE_NO_SOFTMAX
-      sum0 = __uint_as_float(s[5]);
-      if (false)
+        sum0 = __uint_as_float(s[5]);
+        if (false)
 #endif
-      {
+        {
 #ifdef MPFA_ABLATE_NO_EXP
 #define EX2_(x) (x)
 #else
 #define EX2_(x) ex2_approx(x)
 #endif
-        // Software pipeline at 32-column granularity, in place: the exponentials of chunk k+1 are
-        // issued between the instructions that consume chunk k (scale by 448, row sum, E4M3 pack),
-        // so a result is needed a few hundred cycles after its MUFU instruction was issued.
-        // q = 448 P is the E4M3 operand (Section 4.1); the row sum is taken over q and the factor
-        // 448 is divided out once in the epilogue.
-        auto exp_pair = [&](int i) {   // s[i], s[i+1] <- 2^(lam s - lam m)
-          float x0, x1;
-          fma2(x0, x1, __uint_as_float(s[i]), __uint_as_float(s[i + 1]), lam, c);
-          s[i] = __float_as_uint(EX2_(x0));
-          s[i + 1] = __float_as_uint(EX2_(x1));
-        };
+          // q = 448 P is the E4M3 operand (Section 4.1); the row sum is taken over q and the factor
+          // 448 is divided out once in the epilogue.
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) exp_pair(i);
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t packed[8];
 #pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t packed[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            if (c0 + 32 < 128) {
-              exp_pair(c0 + 32 + 4 * i);
-              exp_pair(c0 + 32 + 4 * i + 2);
+            for (int i = 0; i < 8; ++i) {
+              float x0, x1, x2, x3, q0, q1, q2, q3;
+              fma2(x0, x1, __uint_as_float(s[c0 + 4 * i]), __uint_as_float(s[c0 + 4 * i + 1]), lam, cc);
+              fma2(x2, x3, __uint_as_float(s[c0 + 4 * i + 2]), __uint_as_float(s[c0 + 4 * i + 3]), lam, cc);
+              mul2(q0, q1, EX2_(x0), EX2_(x1), 448.0f);
+              mul2(q2, q3, EX2_(x2), EX2_(x3), 448.0f);
+              acc2(sum0, sum1, q0, q1);
+              acc2(sum2, sum3, q2, q3);
+              const uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q0, q1), __NV_SATFINITE, __NV_E4M3);
+              const uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q2, q3), __NV_SATFINITE, __NV_E4M3);
+              packed[i] = (lo & 0xFFFFu) | (hi << 16);
             }
-            float q0, q1, q2, q3;
-            mul2(q0, q1, __uint_as_float(s[c0 + 4 * i]), __uint_as_float(s[c0 + 4 * i + 1]), 448.0f);
-            mul2(q2, q3, __uint_as_float(s[c0 + 4 * i + 2]), __uint_as_float(s[c0 + 4 * i + 3]), 448.0f);
-            acc2(sum0, sum1, q0, q1);
-            acc2(sum2, sum3, q2, q3);
-            const uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q0, q1), __NV_SATFINITE, __NV_E4M3);
-            const uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q2, q3), __NV_SATFINITE, __NV_E4M3);
-            packed[i] = (lo & 0xFFFFu) | (hi << 16);
-          }
 #ifndef MPFA_ABLATE_NO_PST
-          tmem_st8(tP + (c0 >> 2), packed);
+            tmem_st8(tP + (c0 >> 2), packed);
 #else
-          if (packed[0] == 0x12345u && packed[7] == 77u) tmem_st8(tP + (c0 >> 2), packed);
+            if (packed[0] == 0x12345u && packed[7] == 77u) tmem_st8(tP + (c0 >> 2), packed);
 #endif
+          }
         }
+        l_own = __fadd_rn(__fmul_rn(a_own, l_own), (sum0 + sum1) + (sum2 + sum3));
+        m_own = m_t;
+        TR(2 + grp, c, 5);
+        tmem_st_wait();
+        tc_fence_before();
+        warp_arrive(cx.bar(BAR_P_FULL + grp), lane);
+        TR(2 + grp, c, 6);
       }
-      l_own = __fadd_rn(__fmul_rn(a_own, l_own), (sum0 + sum1) + (sum2 + sum3));
-      m_own = m_t;
-      TR(2 + grp, t, 5);
-      tmem_st_wait();
-      tc_fence_before();
-      warp_arrive(cx.bar(BAR_P_FULL + grp), lane);
-      TR(2 + grp, t, 6);
+      if (!ok) break;
+      // which group took the item's last block decides how the epilogue combines the two accumulators
+      float *s_fin = reinterpret_cast<float *>(smem + OFF_L) + (ti & 3) * 512;
+      s_fin[(grp * 2 + 0) * 128 + row] = l_own;
+      s_fin[(grp * 2 + 1) * 128 + row] = m_own;
+      warp_arrive(cx.bar(BAR_L_FULL + (ti & 3)), lane);
     }
-    float *s_fin = reinterpret_cast<float *>(smem + OFF_L);
-    s_fin[(grp * 2 + 0) * 128 + row] = l_own;
-    s_fin[(grp * 2 + 1) * 128 + row] = m_own;
-    warp_arrive(cx.bar(BAR_L_FULL), lane);
   } else if (warp >= 12) {
     // =========================== correction + epilogue ===========================
     setmaxnreg_dec<88>();
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const int r_abs = row0 + row;
     const float *s_m = reinterpret_cast<const float *>(smem + OFF_M);
     const uint32_t tO0 = tm + TM_O0 + lane_off, tO1 = tm + TM_O1 + lane_off;
-    const float lam_c = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[b]), p.k_gscale[b]);
     bool ok = true;
-    float alpha_prev = 1.0f, alpha = 1.0f, m_before = -INFINITY;
-    for (int t = 0; t < T; ++t) {
-      const int sb = t & 1;
-      TR(4, t, 0);
-      ok = __all_sync(0xffffffffu, cx.wait(BAR_M_FULL + sb, (uint32_t)(t >> 1) & 1u));
-      if (!ok) break;
-      TR(4, t, 1);
-      // alpha_t = 2^(lam (m_{t-1} - m_t)) (Eq. 5/6), from the running maxima the softmax groups publish
-      const float m_now = s_m[sb * 128 + row];
-      alpha = (m_now == m_before) ? 1.0f : ex2_approx(__fmul_rn(m_before - m_now, lam_c));
-      m_before = m_now;
-      if (t >= 2) {
-        // O[sb] holds blocks t-2, t-4, ... relative to the maximum after block t-2
-        const float scale = __fmul_rn(alpha, alpha_prev);
-        ok = __all_sync(0xffffffffu, cx.wait(BAR_O_FULL + sb, (uint32_t)((t >> 1) - 1) & 1u));
+    for (; walk.next(p, tl); gb += tl.T, ++ti) {
+      const int T = tl.T;
+      const int r_abs = tl.row0 + row;
+      const float lam_c = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[tl.b]), p.k_gscale[tl.b]);
+      float alpha_prev = 1.0f, alpha = 1.0f, m_before = -INFINITY;
+      for (int t = 0; ok && t < T; ++t) {
+        const uint32_t c = gb + t;
+        const uint32_t sb = c & 1;
+        TR(4, c, 0);
+        ok = __all_sync(0xffffffffu, cx.wait(BAR_M_FULL + sb, (c >> 1) & 1u));
         if (!ok) break;
-        TR(4, t, 2);
-        tc_fence_after();
+        TR(4, c, 1);
+        // alpha_t = 2^(lam (m_{t-1} - m_t)) (Eq. 5/6), from the running maxima the softmax groups publish
+        const float m_now = s_m[sb * 128 + row];
+        alpha = (m_now == m_before) ? 1.0f : ex2_approx(__fmul_rn(m_before - m_now, lam_c));
+        m_before = m_now;
+        if (t >= 2) {
+          // O[sb] holds blocks t-2, t-4, ... relative to the maximum after block t-2
+          const float scale = __fmul_rn(alpha, alpha_prev);
+          ok = __all_sync(0xffffffffu, cx.wait(BAR_O_FULL + sb, ((c >> 1) - 1) & 1u));
+          if (!ok) break;
+          TR(4, c, 2);
+          tc_fence_after();
 #ifdef MPFA_ABLATE_NO_CORR
-        if (false) {
+          if (false) {
 #else
-        if (__any_sync(0xffffffffu, scale != 1.0f)) {   // identical result when every factor is exactly 1
+          if (__any_sync(0xffffffffu, scale != 1.0f)) {   // identical result when every factor is exactly 1
 #endif
-          const uint32_t tO = sb ? tO1 : tO0;
+            const uint32_t tO = sb ? tO1 : tO0;
 #pragma unroll
-          for (int c0 = 0; c0 < HEAD_DIM; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld32(tO + c0, r);
-            tmem_ld_wait();
+            for (int c0 = 0; c0 < HEAD_DIM; c0 += 32) {
+              uint32_t r[32];
+              tmem_ld32(tO + c0, r);
+              tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__fmul_rn(__uint_as_float(r[i]), scale));
-            tmem_st32(tO + c0, r);
+              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__fmul_rn(__uint_as_float(r[i]), scale));
+              tmem_st32(tO + c0, r);
+            }
+            tmem_st_wait();
           }
-          tmem_st_wait();
+          tc_fence_before();
         }
-        tc_fence_before();
+        alpha_prev = alpha;
+        TR(4, c, 3);
+        warp_arrive(cx.bar(BAR_O_READY + sb), lane);
       }
-      alpha_prev = alpha;
-      TR(4, t, 3);
-      warp_arrive(cx.bar(BAR_O_READY + sb), lane);
-    }
-    // final normalisation (Algorithm 1 line 17): O / (448 l) * v_scale -> BF16.  The two softmax
-    // groups hold partial sums relative to their own last maximum; bring both to the final one.
-    // The accumulator of the last block is current; the other one is one alpha behind.
-    const int last = (T - 1) & 1;
-    float l = 0.0f, a_other = 0.0f;
-    if (T > 0 && ok) {
-      ok = cx.wait(BAR_O_FULL + last, (uint32_t)((T - 1) >> 1) & 1u);
-      if (ok && T > 1) ok = cx.wait(BAR_O_FULL + (last ^ 1), (uint32_t)((T - 2) >> 1) & 1u);
-      ok = ok && cx.wait(BAR_L_FULL, 0);
-      tc_fence_after();
+      // final normalisation (Algorithm 1 line 17): O / (448 l) * v_scale -> BF16.  The two softmax
+      // groups hold partial sums relative to their own last maximum; bring both to the final one.
+      // The accumulator of the last block is current; the other one is one alpha behind.
+      const int last = (int)((gb + T - 1) & 1);
+      float l = 0.0f, a_other = 0.0f;
       if (ok) {
-        const float lam = lam_c;
-        const float *s_fin = reinterpret_cast<const float *>(smem + OFF_L);
-        const float l0 = s_fin[0 * 128 + row], m0 = s_fin[1 * 128 + row];
-        const float l1 = s_fin[2 * 128 + row], m1 = s_fin[3 * 128 + row];
-        const float mf = fmaxf(m0, m1);
-        if (mf != -INFINITY) {
-          const float w0 = (m0 == mf) ? 1.0f : ex2_approx(__fmul_rn(m0 - mf, lam));
-          const float w1 = (m1 == mf) ? 1.0f : ex2_approx(__fmul_rn(m1 - mf, lam));
-          l = __fadd_rn(__fmul_rn(w0, l0), __fmul_rn(w1, l1));
-        }
-        if (T > 1) a_other = alpha;   // alpha of the last block
-      }
-    }
-    // tcgen05.ld is warp-collective: every lane loads, only the stores are predicated.
-    const bool warp_ok = __all_sync(0xffffffffu, ok);
-    const bool store = r_abs < p.N_q && (warp_ok || T == 0);
-    const size_t o_off = (((size_t)b * p.N_q + (store ? r_abs : 0)) * p.H_q + hq) * HEAD_DIM;
-    // one IEEE reciprocal per row; 128 divisions per thread would cost more than ten KV blocks
-    const float inv_denom = (l > 0.0f) ? __frcp_rn(l) : 0.0f;   // l already carries the factor 448
-    const uint32_t tOl = last ? tO1 : tO0, tOo = last ? tO0 : tO1;
-#pragma unroll 1
-    for (int c0 = 0; c0 < HEAD_DIM; c0 += 16) {
-      uint32_t r[16], ro[16];
-      if (T > 0 && warp_ok) {
-        tmem_ld16(tOl + c0, r);
-        if (T > 1) tmem_ld16(tOo + c0, ro);
-        tmem_ld_wait();
-      }
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        float acc = __uint_as_float(r[i]);
-        if (T > 1) acc = __fadd_rn(acc, __fmul_rn(a_other, __uint_as_float(ro[i])));
-        r[i] = (l > 0.0f) ? __float_as_uint(__fmul_rn(__fmul_rn(acc, inv_denom), p.v_scale)) : 0u;
-      }
-      if (store) {
-        if (p.out_f32) {
-#pragma unroll
-          for (int i = 0; i < 16; i += 4)
-            *reinterpret_cast<uint4 *>(p.out_f32 + o_off + c0 + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
-        }
-#pragma unroll
-        for (int i = 0; i < 16; i += 8) {
-          uint32_t h[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[i + 2 * j]), __uint_as_float(r[i + 2 * j + 1]));
-            h[j] = *reinterpret_cast<uint32_t *>(&v);
+        if (T > 0) ok = cx.wait(BAR_O_FULL + last, ((gb + T - 1) >> 1) & 1u);
+        if (ok && T > 1) ok = cx.wait(BAR_O_FULL + (last ^ 1), ((gb + T - 2) >> 1) & 1u);
+        ok = ok && cx.wait(BAR_L_FULL + (ti & 3), (ti >> 2) & 1u);
+        tc_fence_after();
+        if (ok && T > 0) {
+          const float lam = lam_c;
+          const float *s_fin = reinterpret_cast<const float *>(smem + OFF_L) + (ti & 3) * 512;
+          const float l0 = s_fin[0 * 128 + row], m0 = s_fin[1 * 128 + row];
+          const float l1 = s_fin[2 * 128 + row], m1 = s_fin[3 * 128 + row];
+          const float mf = fmaxf(m0, m1);
+          if (mf != -INFINITY) {
+            const float w0 = (m0 == mf) ? 1.0f : ex2_approx(__fmul_rn(m0 - mf, lam));
+            const float w1 = (m1 == mf) ? 1.0f : ex2_approx(__fmul_rn(m1 - mf, lam));
+            l = __fadd_rn(__fmul_rn(w0, l0), __fmul_rn(w1, l1));
           }
-          *reinterpret_cast<uint4 *>(p.out + o_off + c0 + i) = make_uint4(h[0], h[1], h[2], h[3]);
+          if (T > 1) a_other = alpha;   // alpha of the last block
         }
       }
+      // tcgen05.ld is warp-collective: every lane loads, only the stores are predicated.
+      const bool warp_ok = __all_sync(0xffffffffu, ok);
+      const bool store = r_abs < p.N_q && (warp_ok || T == 0);
+      const size_t o_off = (((size_t)tl.b * p.N_q + (store ? r_abs : 0)) * p.H_q + tl.hq) * HEAD_DIM;
+      // one IEEE reciprocal per row; 128 divisions per thread would cost more than ten KV blocks
+      const float inv_denom = (l > 0.0f) ? __frcp_rn(l) : 0.0f;   // l already carries the factor 448
+      const uint32_t tOl = last ? tO1 : tO0, tOo = last ? tO0 : tO1;
+#pragma unroll 1
+      for (int c0 = 0; c0 < HEAD_DIM; c0 += 16) {
+        uint32_t r[16], ro[16];
+        if (T > 0 && warp_ok) {
+          tmem_ld16(tOl + c0, r);
+          if (T > 1) tmem_ld16(tOo + c0, ro);
+          tmem_ld_wait();
+        }
+        if (c0 == HEAD_DIM - 16 && T > 0) {   // both accumulators are in registers: the next item's P V may overwrite them
+          tc_fence_before();
+          warp_arrive(cx.bar(BAR_O_FREE), lane);
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float acc = __uint_as_float(r[i]);
+          if (T > 1) acc = __fadd_rn(acc, __fmul_rn(a_other, __uint_as_float(ro[i])));
+          r[i] = (l > 0.0f) ? __float_as_uint(__fmul_rn(__fmul_rn(acc, inv_denom), p.v_scale)) : 0u;
+        }
+        if (store) {
+          if (p.out_f32) {
+#pragma unroll
+            for (int i = 0; i < 16; i += 4)
+              *reinterpret_cast<uint4 *>(p.out_f32 + o_off + c0 + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+          }
+#pragma unroll
+          for (int i = 0; i < 16; i += 8) {
+            uint32_t h[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[i + 2 * j]), __uint_as_float(r[i + 2 * j + 1]));
+              h[j] = *reinterpret_cast<uint32_t *>(&v);
+            }
+            *reinterpret_cast<uint4 *>(p.out + o_off + c0 + i) = make_uint4(h[0], h[1], h[2], h[3]);
+          }
+        }
+      }
+      if (!ok) break;
     }
   }
   if (warp == 12) TR(0, 255, 3);   // epilogue stores issued
@@ -779,8 +831,13 @@ extern "C" mpfa_status mpfa_prefill(const mpfa_fp4_tensor *q, const mpfa_fp4_ten
   p.causal = causal ? 1 : 0;
   p.softmax_scale = softmax_scale;
   p.v_scale = v_scale;
+  p.n_items = (int)n_cta;
+  int dev = 0, n_sm = 0;
+  MPFA_CUDA_OK(cudaGetDevice(&dev));
+  MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  const unsigned grid = (unsigned)(n_cta < (uint64_t)n_sm ? n_cta : (uint64_t)n_sm);   // one persistent CTA per SM
   MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-  prefill_kernel<<<(unsigned)n_cta, NTHREADS, SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p);
+  prefill_kernel<<<grid, NTHREADS, SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p);
   MPFA_LAUNCH_OK();
   return MPFA_OK;
 }
