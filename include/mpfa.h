@@ -198,7 +198,9 @@ mpfa_status mpfa_prefill(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tensor *h_k,
  * page_table [B, max_pages_per_req].  Each (request, kv head, 1024-token partition) keeps a
  * local (m, l, O) state for its GQA group in `workspace`; a second kernel merges the
  * partitions by log-sum-exp.  The number of partitions is fixed by max_seq_len, so the call
- * sequence does not depend on seq_lens.  out_bf16 [B, H_q, 128]; out_f32 optional. */
+ * sequence (one 4-byte memory set of the work counter at the end of `workspace`, two kernels)
+ * does not depend on seq_lens.  Work items are drawn from that counter by the running CTAs, so
+ * two calls that overlap on the GPU need separate workspaces.  out_bf16 [B, H_q, 128]; out_f32 optional. */
 mpfa_status mpfa_decode(const mpfa_fp4_tensor *h_q, const mpfa_paged_kv *h_kv, const int32_t *page_table,
                         int max_pages_per_req, const int32_t *seq_lens, const mpfa_stats *h_stats,
                         float v_scale, float softmax_scale, void *out_bf16, float *out_f32, void *workspace,

@@ -28,7 +28,7 @@
 // sum with the factors multiplied out.  The partition state (m, l, O) goes to the workspace; a
 // second kernel merges partitions by log-sum-exp and writes BF16.
 //
-// Warps: 0, 9 K producers, 8 V producer, 1 QK issue (+ TMEM allocation), 2 PV issue, 3 rewrites the K scales of
+// Warps: 10 draws work items, 0, 9 K producers, 8 V producer, 1 QK issue (+ TMEM allocation), 2 PV issue, 3 rewrites the K scales of
 // each block from [token][8] into the 32 x 16-byte tiles tcgen05.cp expects, 4-7 softmax and
 // partition write-out (TMEM lane quadrant = warp % 4).  Every wait is bounded.
 #include <cuda_bf16.h>
@@ -47,7 +47,8 @@ constexpr int MAXBLK = DECODE_SPLIT / TILE;   // 8 blocks per item
 
 constexpr int D_NK = 4;           // K ring stages
 constexpr int D_NV = 8;           // V ring stages
-constexpr int D_THREADS = 320;
+constexpr int D_THREADS = 352;
+constexpr int D_NITEM = 8;        // work items published ahead of their use
 
 // one K stage
 constexpr uint32_t KST_K = 0;          // 2 pages x 4096 B of codes: 64-byte rows, 64-byte swizzle
@@ -64,15 +65,17 @@ constexpr uint32_t D_OFF_SFK = D_OFF_SFQ + 2048;           // D_NK x (2 x 512): 
 constexpr uint32_t D_OFF_ZERO = D_OFF_SFK + D_NK * 1024;    // 2048 B of zeros: second K group of the Delta_S operand, rows 8..15 of P_hat^T
 constexpr uint32_t D_OFF_IDENT = D_OFF_ZERO + 2048;        // 16 x 16 BF16 identity, MN-major, 128-byte swizzle
 constexpr uint32_t D_OFF_BAR = D_OFF_IDENT + 2048;
-constexpr uint32_t D_OFF_XMAX = D_OFF_BAR + 512;           // [2][8 blocks][MAXG][4 warps] floats
+constexpr uint32_t D_OFF_XMAX = D_OFF_BAR + 1024;           // [2][8 blocks][MAXG][4 warps] floats
 constexpr uint32_t D_OFF_WTAB = D_OFF_XMAX + 2 * MAXBLK * MAXG * 16;   // [2][8 blocks][MAXG] floats
 constexpr uint32_t D_OFF_MFIN = D_OFF_WTAB + 2 * MAXBLK * MAXG * 4;    // [2][MAXG]
 constexpr uint32_t D_OFF_XL = D_OFF_MFIN + 2 * MAXG * 4;               // [2][4 warps][MAXG]
 constexpr uint32_t D_OFF_MISC = D_OFF_XL + 2 * 4 * MAXG * 4;           // TMEM address, abort flag
 constexpr int D_MAXREQ = 768;                                          // requests whose length / lambda are cached
-constexpr uint32_t D_OFF_LEN = D_OFF_MISC + 64;                        // [D_MAXREQ] int32
+constexpr uint32_t D_OFF_LEN = D_OFF_MISC + 64;                        // [D_MAXREQ] int32 lengths
 constexpr uint32_t D_OFF_LAM = D_OFF_LEN + D_MAXREQ * 4;               // [D_MAXREQ] float
-constexpr uint32_t D_SMEM_USED = D_OFF_LAM + D_MAXREQ * 4;
+constexpr uint32_t D_OFF_RING = D_OFF_LAM + D_MAXREQ * 4;              // [D_NITEM] int4 work items {b, hk, sp, L}
+constexpr uint32_t D_OFF_PRE = D_OFF_RING + D_NITEM * 16;              // [D_MAXREQ + 1] items of the requests before b
+constexpr uint32_t D_SMEM_USED = D_OFF_PRE + (D_MAXREQ + 4) * 4;
 constexpr uint32_t D_SMEM = D_SMEM_USED + 1024;     // slack for the 1024-byte alignment of the base
 
 // barriers (8 bytes each)
@@ -88,8 +91,10 @@ constexpr int B_Q_READY = B_P_READY + 2;         // [2] scale warp
 constexpr int B_O_FULL = B_Q_READY + 2;          // [1] PV commit after the item's last block
 constexpr int B_O_FREE = B_O_FULL + 1;           // [1] 4 warps
 constexpr int B_XCHG = B_O_FREE + 1;             // [1] 4 warps
-constexpr int B_COUNT = B_XCHG + 1;
-static_assert(B_COUNT * 8 <= 512, "barrier block");
+constexpr int B_ITEM_FULL = B_XCHG + 1;          // [D_NITEM] work item published
+constexpr int B_ITEM_EMPTY = B_ITEM_FULL + D_NITEM;   // [D_NITEM] read by all ten consumer warps
+constexpr int B_COUNT = B_ITEM_EMPTY + D_NITEM;
+static_assert(B_COUNT * 8 <= 1024, "barrier block");
 static_assert(D_SMEM <= 232448, "shared memory");
 static_assert(KST_BYTES % 1024 == 0 && D_OFF_V % 1024 == 0 && D_OFF_P % 1024 == 0, "swizzle atoms");
 
@@ -159,53 +164,16 @@ struct DecodeParams {
   const float *q_gscale, *k_gscale;
   float *parts;  // [B, H_q, n_split, 130]
   int32_t *status;
+  unsigned int *ticket;   // global work counter, zeroed before the launch
   int B, H_q, H_kv, max_pages, num_pages, n_split;
   float softmax_scale;
 };
 
-// The work list, walked identically by every role: items blockIdx.x, blockIdx.x + gridDim.x, ...
-// in (partition fastest, kv head, request) order; partitions beyond the sequence are skipped.
-struct WorkIter {
-  int idx, stride, total, n_split, H_kv;
-  int ds, dh, db;   // the stride as (partition, kv head, request) digits: no division per step
-  int b, hk, sp, L, nblk;
-  const int32_t *len_tab;   // shared-memory copy of seq_lens (first D_MAXREQ requests)
-  __device__ void init(const DecodeParams &p, const int32_t *tab) {
-    len_tab = tab;
-    stride = gridDim.x;
-    n_split = p.n_split;
-    H_kv = p.H_kv;
-    total = p.B * p.H_kv * p.n_split;
-    ds = stride % n_split;
-    dh = (stride / n_split) % H_kv;
-    db = stride / (n_split * H_kv);
-    // one step before the first item (digits may be negative here; the first step normalises them)
-    idx = (int)blockIdx.x - stride;
-    const int i0 = (int)blockIdx.x;
-    sp = i0 % n_split - ds;
-    hk = (i0 / n_split) % H_kv - dh;
-    b = i0 / (n_split * H_kv) - db;
-    if (sp < 0) sp += n_split, hk -= 1;
-    if (hk < 0) hk += H_kv, b -= 1;
-  }
-  __device__ bool next(const int32_t *__restrict__ seq_lens) {
-    for (;;) {
-      idx += stride;
-      if (idx >= total) return false;
-      sp += ds;
-      hk += dh;
-      b += db;
-      if (sp >= n_split) sp -= n_split, hk += 1;
-      if (hk >= H_kv) hk -= H_kv, b += 1;
-      L = b < D_MAXREQ ? len_tab[b] : seq_lens[b];
-      const int rem = L - sp * DECODE_SPLIT;
-      if (rem > 0) {
-        nblk = (min(rem, DECODE_SPLIT) + TILE - 1) / TILE;
-        return true;
-      }
-    }
-  }
-};
+// Work items (request, kv head, 1024-token partition) are handed out dynamically: one warp per CTA draws
+// tickets from a global counter and publishes the decoded items in a small shared-memory ring; every other
+// warp walks that ring.  SMs do not stream at the same rate (those far from the memory they read are up to
+// 8 % slower), so a static split leaves the fast ones idle at the end.
+struct WorkIter;
 
 struct DCtx {
   uint32_t bar0;
@@ -236,6 +204,28 @@ struct DCtx {
   __device__ __forceinline__ void warp_arrive(int i) const {
     __syncwarp();
     if ((threadIdx.x & 31) == 0) mbar_arrive(bar(i));
+  }
+};
+
+struct WorkIter {
+  uint32_t n;          // items taken so far
+  bool release;        // the warp's main walk hands the ring slot back; look-ahead walks only read
+  int b, hk, sp, L, nblk;
+  __device__ void init(bool main_walk) {
+    n = 0;
+    release = main_walk;
+  }
+  // Whole warp.  false: no more items (or the CTA is giving up).
+  __device__ bool next(const DCtx &cx, const int4 *ring) {
+    const uint32_t slot = n % D_NITEM;
+    if (!cx.wait_warp(B_ITEM_FULL + slot, (n / D_NITEM) & 1)) return false;
+    const int4 it = ring[slot];
+    if (it.x < 0) return false;   // end marker: stays in its slot, nobody moves past it
+    if (release) cx.warp_arrive(B_ITEM_EMPTY + slot);
+    ++n;
+    b = it.x, hk = it.y, sp = it.z, L = it.w;
+    nblk = (min(L - sp * DECODE_SPLIT, DECODE_SPLIT) + TILE - 1) / TILE;
+    return true;
   }
 };
 
@@ -289,6 +279,10 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
     mbar_init(cx.bar(B_O_FULL), 1);
     mbar_init(cx.bar(B_O_FREE), 4);
     mbar_init(cx.bar(B_XCHG), 4);
+    for (int i = 0; i < D_NITEM; ++i) {
+      mbar_init(cx.bar(B_ITEM_FULL + i), 1);
+      mbar_init(cx.bar(B_ITEM_EMPTY + i), 10);
+    }
     mbar_init_fence();
     *abort_flag = 0;
   }
@@ -317,8 +311,74 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
   __syncthreads();
   tc_fence_after();
   const uint32_t tm = *tmem_slot;
+  const int4 *ring = reinterpret_cast<const int4 *>(dsm + D_OFF_RING);
 
-  if (warp == 0 || warp >= 8) {
+  if (warp == 10) {
+    // ================= work distribution: tickets from the global counter, decoded, published D_NITEM ahead.
+    // With at most D_MAXREQ requests the tickets number only the partitions that exist (prefix sums of
+    // ceil(L / 1024) * H_kv per request, request found by bisection); otherwise they number every
+    // (request, kv head, partition slot) and the empty ones are drawn again.
+    int4 *ring_w = reinterpret_cast<int4 *>(dsm + D_OFF_RING);
+    int32_t *pre = reinterpret_cast<int32_t *>(dsm + D_OFF_PRE);
+    const bool compact = p.B <= D_MAXREQ;
+    uint32_t total;
+    if (compact) {
+      // pre[b] = items of requests 0..b-1: every lane sums a contiguous run of requests, the warp scans the runs
+      const int per = (p.B + 31) / 32, lo = min(p.B, lane * per), hi = min(p.B, lo + per);
+      int run = 0;
+      for (int i = lo; i < hi; ++i) run += min((max(len_tab[i], 0) + DECODE_SPLIT - 1) / DECODE_SPLIT, p.n_split) * p.H_kv;
+      int incl = run;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      int acc = incl - run;
+      for (int i = lo; i < hi; ++i) {
+        pre[i] = acc;
+        acc += min((max(len_tab[i], 0) + DECODE_SPLIT - 1) / DECODE_SPLIT, p.n_split) * p.H_kv;
+      }
+      total = (uint32_t)__shfl_sync(0xffffffffu, incl, 31);
+      if (lane == 31) pre[p.B] = (int)total;
+      __syncwarp();
+    } else {
+      total = (uint32_t)p.B * p.H_kv * p.n_split;
+    }
+    bool ok = true;
+    for (uint32_t k = 0; ok; ++k) {
+      const uint32_t slot = k % D_NITEM;
+      if (k >= (uint32_t)D_NITEM) ok = cx.wait_warp(B_ITEM_EMPTY + slot, ((k / D_NITEM) - 1) & 1);
+      if (!ok) break;
+      int4 item = make_int4(-1, 0, 0, 0);
+      if (lane == 0) {
+        for (;;) {
+          const uint32_t tkt = atomicAdd(p.ticket, 1u);
+          if (tkt >= total) break;
+          if (compact) {
+            int lo = 0, hi = p.B;   // largest b with pre[b] <= tkt
+            while (hi - lo > 1) {
+              const int mid = (lo + hi) >> 1;
+              if ((uint32_t)pre[mid] <= tkt) lo = mid; else hi = mid;
+            }
+            const int L = len_tab[lo], nsp = min((L + DECODE_SPLIT - 1) / DECODE_SPLIT, p.n_split);
+            const int r = (int)tkt - pre[lo];
+            item = make_int4(lo, r / nsp, r % nsp, L);
+            break;
+          }
+          const int sp = (int)(tkt % (uint32_t)p.n_split), r = (int)(tkt / (uint32_t)p.n_split);
+          const int b = r / p.H_kv, L = p.seq_lens[b];
+          if (L - sp * DECODE_SPLIT > 0) {
+            item = make_int4(b, r % p.H_kv, sp, L);
+            break;
+          }
+        }
+        ring_w[slot] = item;
+        mbar_arrive(cx.bar(B_ITEM_FULL + slot));
+      }
+      item.x = __shfl_sync(0xffffffffu, item.x, 0);
+      if (item.x < 0) break;   // the end marker is in the ring; this CTA draws no more
+    }
+  } else if (warp == 0 || warp >= 8) {
     // ================= producers: warps 0 and 9 stream the K ring (0: codes; 9: block scales and Delta_S,
     // both arriving on the stage's barrier), warp 8 the V ring.  Issuing a bulk copy costs a warp well over a
     // hundred cycles, so the ten copies of a block are spread over three warps.
@@ -327,8 +387,8 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
     // they are used and validated at use, so the loop never waits for the table.
     const bool is_k = warp != 8, is_codes = warp == 0;
     WorkIter w, wl;
-    w.init(p, len_tab);
-    wl.init(p, len_tab);
+    w.init(true);
+    wl.init(false);
     uint32_t c = 0;   // block counter of this ring
     bool ok = true;
     const uint32_t d_bytes = p.delta ? (uint32_t)G * PAGE * 2 : 0u;
@@ -336,13 +396,13 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
     const int n_ring = is_k ? D_NK : D_NV;
     const int b_full = is_k ? B_K_FULL : B_V_FULL, b_empty = is_k ? B_K_EMPTY : B_V_EMPTY;
     int pc0 = -1, pc1 = -1, pn0 = -1, pn1 = -1;
-    bool vw = w.next(p.seq_lens);
-    bool vl = wl.next(p.seq_lens);
+    bool vw = w.next(cx, ring);
+    bool vl = wl.next(cx, ring);
     if (vw) lookup_pages(p, w, lane, pc0, pc1);
     uint32_t jtr = 0;
     while (ok && vw) {
       if (is_codes) DTR(12, jtr);
-      vl = wl.next(p.seq_lens);
+      vl = wl.next(cx, ring);
       if (is_codes) DTR(13, jtr);
       if (vl) lookup_pages(p, wl, lane, pn0, pn1);   // consumed one item later
       if (is_codes) DTR(14, jtr);
@@ -403,7 +463,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
         __syncwarp();
       }
       if (is_codes) DTR(15, jtr - 1);
-      vw = w.next(p.seq_lens);
+      vw = w.next(cx, ring);
       pc0 = pn0, pc1 = pn1;
     }
     if (!ok) {
@@ -421,10 +481,10 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
     const uint64_t d_ident = smem_desc(sbase + D_OFF_IDENT, 2048, 1024, SWZ_128B);
     const bool has_delta = p.delta != nullptr;
     WorkIter w;
-    w.init(p, len_tab);
+    w.init(true);
     uint32_t kc = 0, j = 0;
     bool ok = true;
-    while (ok && w.next(p.seq_lens)) {
+    while (ok && w.next(cx, ring)) {
       const uint32_t par = j & 1;
       ok = cx.wait_warp(B_Q_READY + par, (j >> 1) & 1);
       if (ok && j >= 2) ok = cx.wait_warp(B_S_FREE + par, ((j >> 1) - 1) & 1);   // scores of item j-2 have been read
@@ -471,10 +531,10 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
     // ================= PV issue: O_u^T = V_u^T P_hat_u^T as V stages land
     const uint32_t id_pv = idesc_e4m3(128, NCOL, 1, 0);
     WorkIter w;
-    w.init(p, len_tab);
+    w.init(true);
     uint32_t vc = 0, j = 0;
     bool ok = true;
-    while (ok && w.next(p.seq_lens)) {
+    while (ok && w.next(cx, ring)) {
       const uint32_t par = j & 1;
       ok = cx.wait_warp(B_P_READY + par, (j >> 1) & 1);
       if (ok && j >= 1) ok = cx.wait_warp(B_O_FREE, (j - 1) & 1);   // the previous item's O has been read
@@ -508,15 +568,15 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
     // The same warp stages the query tile (codes and scales of the group's G heads) of item j+1 while
     // item j is scored: that slot was last read by the MMAs of item j-1.
     WorkIter w, wq;
-    w.init(p, len_tab);
-    wq.init(p, len_tab);
+    w.init(true);
+    wq.init(false);
     uint32_t kc = 0, j = 0, n_staged = 0;
     bool ok = true;
     uint4 qv = make_uint4(0u, 0u, 0u, 0u);
     uint32_t qs0 = 0, qs1 = 0;
     bool have_q = false;
     auto load_q = [&]() {   // global loads of the next item's tile, consumed one item later
-      have_q = wq.next(p.seq_lens);
+      have_q = wq.next(cx, ring);
       if (!have_q) return;
       if (lane < G * 4)
         qv = *reinterpret_cast<const uint4 *>(p.q_codes + ((size_t)wq.b * p.H_q + wq.hk * G + (lane >> 2)) * (TILE * 64) + (lane & 3) * 16);
@@ -547,7 +607,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
     load_q();
     store_q();
     load_q();
-    while (ok && w.next(p.seq_lens)) {
+    while (ok && w.next(cx, ring)) {
       if (j >= 1) {
         // all QK MMAs of item j-1 are complete once its last block's scores are
         const uint32_t pj = j - 1;
@@ -618,10 +678,10 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
     };
 
     WorkIter w;
-    w.init(p, len_tab);
+    w.init(true);
     uint32_t j = 0;
     Prev prev{0, 0, 0, 0};
-    while (ok && w.next(p.seq_lens)) {
+    while (ok && w.next(cx, ring)) {
       const uint32_t par = j & 1;
       const float lam = w.b < D_MAXREQ ? lam_tab[w.b]
                                        : __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[w.b]), p.k_gscale[w.b]);
@@ -780,10 +840,15 @@ extern "C" int mpfa_debug_set_decode_trace(long long *buf, int cta) {
 }
 #endif
 
+// partition states, then (256-byte aligned) the work counter of the split kernel
+static size_t decode_parts_bytes(int B, int H_q, size_t n_split) {
+  return ((size_t)B * H_q * n_split * PART_FLOATS * sizeof(float) + 255) / 256 * 256;
+}
+
 extern "C" size_t mpfa_decode_workspace_bytes(int B, int H_q, int H_kv, int max_pages_per_req) {
   if (B <= 0 || H_q <= 0 || H_kv <= 0 || max_pages_per_req <= 0) return 0;
   const size_t n_split = ((size_t)max_pages_per_req * PAGE + DECODE_SPLIT - 1) / DECODE_SPLIT;
-  return (size_t)B * H_q * n_split * PART_FLOATS * sizeof(float);
+  return decode_parts_bytes(B, H_q, n_split) + 256;
 }
 
 extern "C" mpfa_status mpfa_decode(const mpfa_fp4_tensor *q, const mpfa_paged_kv *kv, const int32_t *page_table,
@@ -802,7 +867,7 @@ extern "C" mpfa_status mpfa_decode(const mpfa_fp4_tensor *q, const mpfa_paged_kv
   if (H_kv <= 0 || kv->H_q != H_q) return MPFA_ERR_INVALID_ARG;
   if (H_q % H_kv != 0 || H_q / H_kv > MAXG) return MPFA_ERR_UNSUPPORTED;
   const size_t n_split = ((size_t)max_pages_per_req * PAGE + DECODE_SPLIT - 1) / DECODE_SPLIT;
-  const size_t need = (size_t)B * H_q * n_split * PART_FLOATS * sizeof(float);
+  const size_t need = decode_parts_bytes(B, H_q, n_split) + 256;
   if (workspace_bytes < need) return MPFA_ERR_WORKSPACE;
   if ((size_t)B * H_kv * n_split > 0x7FFFFFFFull || B > 65535) return MPFA_ERR_UNSUPPORTED;
   if (!aligned(q->codes, 16) || !aligned(q->sf, 16) || !aligned(kv->k_codes, 256) || !aligned(kv->k_sf, 256) ||
@@ -825,6 +890,7 @@ extern "C" mpfa_status mpfa_decode(const mpfa_fp4_tensor *q, const mpfa_paged_kv
   p.q_gscale = st->q_gscale;
   p.k_gscale = st->k_gscale;
   p.parts = static_cast<float *>(workspace);
+  p.ticket = reinterpret_cast<unsigned int *>(static_cast<uint8_t *>(workspace) + decode_parts_bytes(B, H_q, n_split));
   p.status = device_status;
   p.B = B;
   p.H_q = H_q;
@@ -849,6 +915,7 @@ extern "C" mpfa_status mpfa_decode(const mpfa_fp4_tensor *q, const mpfa_paged_kv
     default: return MPFA_ERR_UNSUPPORTED;
   }
   MPFA_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)D_SMEM));
+  MPFA_CUDA_OK(cudaMemsetAsync(p.ticket, 0, sizeof(unsigned int), s));   // a memory-set node, no allocation
   kern<<<grid, D_THREADS, D_SMEM, s>>>(p);
   MPFA_LAUNCH_OK();
   decode_merge_kernel<<<dim3(H_q, B), 128, 0, s>>>(p.parts, seq_lens, st->q_gscale, st->k_gscale, H_q, (int)n_split,
