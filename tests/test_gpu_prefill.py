@@ -59,6 +59,13 @@ CASES = {
     "ragged_causal": lambda: wl.prefill_workload("rag", 53, 2, 333, 4, 2, True, q_bias=True),
     "ragged_noncausal_nq_lt_nkv": lambda: wl.prefill_workload("rag2", 54, 1, 517, 2, 1, False, N_q=200),
     "causal_offset": lambda: wl.prefill_workload("coff", 55, 1, 640, 2, 2, True, N_q=130, q_bias=True),
+    # more queries than keys under a bottom-right aligned causal mask: the first 300 rows see no key (output 0),
+    # two whole query tiles have no KV block to visit
+    "causal_nq_gt_nkv": lambda: wl.prefill_workload("cgt", 56, 1, 200, 2, 1, True, N_q=500, q_bias=True),
+    # 320 one-block work items on 148 persistent CTAs: item boundaries back to back
+    "many_one_block_items": lambda: wl.prefill_workload("one", 57, 1, 128, 8, 2, False, N_q=5120, q_bias=True),
+    # 2- and 3-block items only
+    "many_short_items": lambda: wl.prefill_workload("short", 58, 2, 300, 8, 4, False, N_q=1500),
 }
 
 
