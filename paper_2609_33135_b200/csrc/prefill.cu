@@ -402,9 +402,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         TR(5, c, 1);
         tc_fence_after();
         if (elect_one()) {
+#ifdef MPFA_ABLATE_NO_QK
+          if (t > 100000)
+#endif
+          {
           if (has_delta) mma_bf16_ss(tm + TM_S, d_ones, d_delta, id_bf16, 0);
           mma_nvfp4_ss(tm + TM_S, d_q0, d_k, id_fp4, tSFQ, tSFK, has_delta ? 1u : 0u);
           mma_nvfp4_ss(tm + TM_S, d_q0 + (32 >> 4), d_k + (32 >> 4), id_fp4, tSFQ + 4, tSFK + 4, 1u);
+          }
           mma_commit(cx.bar(BAR_S_FULL + sb));
           mma_commit(cx.bar(BAR_K_EMPTY + ks));
         }
@@ -442,6 +447,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (elect_one()) {
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
+#ifdef MPFA_ABLATE_NO_PV
+            if (k4 > 100)
+#endif
             mma_e4m3_ts(tOacc, tP + 8 * k4, d_v + (uint64_t)((4096 * k4) >> 4), id_fp8, (t >= 2 || k4 > 0) ? 1u : 0u);
           mma_commit(cx.bar(BAR_O_FULL + sb));
           mma_commit(cx.bar(BAR_P_EMPTY + sb));
