@@ -172,7 +172,11 @@ mpfa_status mpfa_quantize_v(const void *v_bf16, int B, int N_kv, int H_kv, float
  * page of tokens [64 i, 64 i + 64).  h_stats points at this request's statistics
  * (B = 1 slices).  Without MPFA_STATS_FROZEN (allowed only when first_token == 0) k_mean and
  * k_gscale are computed from these tokens; q_mean and q_gscale are always read.
- * Slots of the last page beyond the written tokens are zero-filled. */
+ * With MPFA_STATS_FROZEN first_token may be any position (decode-time append, Section 6: a
+ * new token is centered with the frozen means and quantized with the frozen tensor scale):
+ * the tokens land in their slots of partly filled pages without touching their neighbours.
+ * Slots beyond the written tokens are zero-filled in every page that this call starts
+ * (position 0 of the page is among the written tokens); decode relies on that. */
 mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_bf16, int N_tokens, int first_token,
                                    int H_q, int H_kv, int flags, mpfa_stats *h_stats, float v_scale,
                                    const mpfa_paged_kv *h_kv, const int32_t *page_table_row,

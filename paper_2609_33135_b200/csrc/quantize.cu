@@ -374,6 +374,71 @@ __global__ void __launch_bounds__(256) quantize_kv_page_kernel(const __nv_bfloat
   reinterpret_cast<uint4 *>(v_fp8 + slab * 8192)[threadIdx.x + 256] = reinterpret_cast<const uint4 *>(sv)[threadIdx.x + 256];
 }
 
+// Decode-time append (Section 6: new tokens are centered with the frozen means and quantized with the
+// frozen tensor scale): tokens first_token .. first_token + N - 1 of one request go to their slots of the
+// paged cache, wherever in a page they fall.  Thread = (token slot, 16-channel block); a block covers 32
+// slots of one kv head.  The grid runs to the end of the last page touched: slots past the last new token
+// are zero-filled if this call started their page (a recycled page may hold anything, and decode needs
+// finite bytes there); slots of a page that was started earlier are left alone.
+__global__ void __launch_bounds__(256) append_kv_kernel(const __nv_bfloat16 *__restrict__ k,
+                                                        const __nv_bfloat16 *__restrict__ v,
+                                                        const float *__restrict__ q_mean,
+                                                        const float *__restrict__ k_mean,
+                                                        const float *__restrict__ q_gscale,
+                                                        const float *__restrict__ k_gscale, int N, int first_token,
+                                                        int H_q, int H_kv, float inv_vscale, int smooth,
+                                                        const int32_t *__restrict__ page_row, int num_pages,
+                                                        uint8_t *__restrict__ k_codes, uint8_t *__restrict__ k_sf,
+                                                        uint8_t *__restrict__ v_fp8, __nv_bfloat16 *__restrict__ delta) {
+  constexpr int MAXG = 8;
+  __shared__ float kmu[HEAD_DIM];
+  __shared__ double qmu[MAXG][HEAD_DIM];
+  __shared__ float kc[32][HEAD_DIM + 4];   // centered K rows of the block's tokens (for Delta_S)
+  const int h = blockIdx.y, G = H_q / H_kv;
+  const int slot = threadIdx.x >> 3, g = threadIdx.x & 7;
+  const int i = blockIdx.x * 32 + slot;          // index among the slots this call covers
+  const int tok = first_token + i;               // absolute token position
+  const bool is_new = i < N;
+  const bool in_range = tok < ((first_token + N + PAGE - 1) / PAGE) * PAGE;   // the grid is rounded up to 32 slots
+  if (threadIdx.x < HEAD_DIM) kmu[threadIdx.x] = k_mean[(size_t)h * HEAD_DIM + threadIdx.x];
+  if (smooth)
+    for (int j = threadIdx.x; j < G * HEAD_DIM; j += 256)
+      qmu[j >> 7][j & 127] = (double)q_mean[((size_t)h * G + (j >> 7)) * HEAD_DIM + (j & 127)];
+  __syncthreads();
+  const int page = in_range ? page_row[tok >> 6] : -1;
+  const bool page_ok = page >= 0 && page < num_pages;
+  const bool fresh_pad = !is_new && (tok & ~63) >= first_token;   // padding slot of a page this call started
+  const int t = tok & 63;
+  uint2 c = make_uint2(0u, 0u);
+  uint8_t sc = 0;
+  uint4 vc = make_uint4(0u, 0u, 0u, 0u);
+  if (is_new) {
+    float xc[16];
+    load_center16(k + ((size_t)i * H_kv + h) * HEAD_DIM + g * 16, kmu + g * 16, xc);
+    quantize_block16(xc, k_gscale[0], sc, c);
+    vc = quantize_v16(v + ((size_t)i * H_kv + h) * HEAD_DIM + g * 16, inv_vscale);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) kc[slot][g * 16 + j] = xc[j];
+  }
+  if (page_ok && (is_new || fresh_pad)) {
+    const size_t slab = (size_t)page * H_kv + h;
+    *reinterpret_cast<uint2 *>(k_codes + slab * 4096 + (t >> 3) * 512 + (t & 7) * 64 + (((g >> 1) ^ ((t & 7) >> 1)) << 4) + (g & 1) * 8) = c;
+    k_sf[slab * 512 + t * 8 + g] = sc;
+    *reinterpret_cast<uint4 *>(v_fp8 + slab * 8192 + (t >> 3) * 1024 + (t & 7) * 128 + ((g ^ (t & 7)) << 4)) = vc;
+  }
+  __syncthreads();
+  // Delta_S (Eq. 9) of the new tokens: thread (slot, g) takes head g of the group, FP64, channels ascending
+  if (smooth && g < G && page_ok && (is_new || fresh_pad)) {
+    float val = 0.0f;
+    if (is_new) {
+      double acc = 0.0;
+      for (int ch = 0; ch < HEAD_DIM; ++ch) acc = fma(qmu[g][ch], (double)kc[slot][ch], acc);
+      val = __double2float_rn(__ddiv_rn(acc, (double)q_gscale[0] * (double)k_gscale[0]));
+    }
+    delta[((size_t)page * H_q + h * G + g) * PAGE + ((((t >> 3) ^ g) << 3) | (t & 7))] = __float2bfloat16_rn(val);
+  }
+}
+
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 struct StatsWorkspace {
@@ -518,7 +583,6 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
   if (smooth && !kv->delta_s_bf16) return MPFA_ERR_INVALID_ARG;
   if (kv->page_size != PAGE || H_q % H_kv != 0 || H_q / H_kv > 8) return MPFA_ERR_UNSUPPORTED;
   if (kv->H_q != H_q || kv->H_kv != H_kv) return MPFA_ERR_INVALID_ARG;
-  if (first_token % PAGE != 0) return MPFA_ERR_UNSUPPORTED;  // appends inside a partly filled page: not built yet
   if (!frozen && first_token != 0) return MPFA_ERR_INVALID_ARG;
   if (!aligned(k_bf16, 16) || !aligned(v_bf16, 16) || !aligned(kv->k_codes, 256) || !aligned(kv->k_sf, 256) ||
       !aligned(kv->v_fp8, 256) || !aligned(kv->delta_s_bf16, 256))
@@ -539,6 +603,17 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
     MPFA_CUDA_OK(cudaMemsetAsync(workspace, 0, w.bytes, s));
     rc = tensor_stats(k, 1, N_tokens, H_kv, smooth, w.sums_k, w.max_k, w.neg_k, w.amax_k, st->k_mean, st->k_gscale, s);
     if (rc != MPFA_OK) return rc;
+  }
+  if (first_token % PAGE != 0) {
+    // append into a partly filled page (frozen statistics; checked above): slot-granular kernel
+    const int last_page_end = (first_token + N_tokens + PAGE - 1) / PAGE * PAGE;
+    const int n_slots = last_page_end - first_token;
+    append_kv_kernel<<<dim3((n_slots + 31) / 32, H_kv), 256, 0, s>>>(
+        k, v, st->q_mean, st->k_mean, st->q_gscale, st->k_gscale, N_tokens, first_token, H_q, H_kv, 1.0f / v_scale,
+        smooth ? 1 : 0, page_table_row, kv->num_pages, kv->k_codes, kv->k_sf, kv->v_fp8,
+        static_cast<__nv_bfloat16 *>(kv->delta_s_bf16));
+    MPFA_LAUNCH_OK();
+    return MPFA_OK;
   }
   const int n_pages = (N_tokens + PAGE - 1) / PAGE;
   quantize_kv_page_kernel<<<dim3(n_pages, H_kv), 256, 0, s>>>(k, v, st->k_mean, st->k_gscale, N_tokens, H_kv,

@@ -144,3 +144,57 @@ def test_decode_bad_page_is_reported_not_followed():
     torch.cuda.synchronize()
     assert int(st.status.item()) & 2
     assert torch.isfinite(st.out_f32).all()
+
+
+def test_append_into_partly_filled_pages_then_decode():
+    """Decode-time appends: a cache built from the first L0 tokens (statistics frozen there) grows token by token
+    and in ragged chunks, across page boundaries and into fresh pages; every slab must equal what the oracle
+    quantizes for the full sequence with the same frozen statistics (bit-exact), pad slots stay zero, and the
+    decode over the grown cache matches the oracle's."""
+    from paper_2609_33135_b200 import binding as B_, decode_cache
+    L0, L1 = [100, 64, 1], [391, 200, 131]
+    w_full = wl.decode_workload("dec_append", 77, 3, 8, 2, 1, 400, seq_lens=L1)
+    w0 = wl.decode_workload("dec_append", 77, 3, 8, 2, 1, 400, seq_lens=L0)
+    # same page pool and table for both: allocate for the final lengths, fill only the first L0 tokens
+    w0.page_table, w0.num_pages = w_full.page_table, w_full.num_pages
+    kv_full = [w_full.kv_for_request(b) for b in range(3)]
+    w0.kv_for_request = lambda b, device="cpu": (kv_full[b][0][:, :L0[b]].contiguous(), kv_full[b][1][:, :L0[b]].contiguous())
+    st = decode_cache.build_cache(w0)
+    # poison the pages that the appends will start, so that missing zero-fill shows
+    for b in range(3):
+        for i in range((L0[b] + 63) // 64, (L1[b] + 63) // 64):
+            pg = int(w_full.page_table[b, i])
+            st.kv.k_codes[pg].fill_(0x7F)
+            st.kv.k_sf[pg].fill_(0x7F)
+            st.kv.v_fp8[pg].fill_(0x7F)
+            st.kv.delta[pg].fill_(float("nan"))
+    flags = B_.MPFA_SMOOTH | B_.MPFA_STATS_FROZEN
+    for b in range(3):
+        k, v = kv_full[b][0][0].cuda(), kv_full[b][1][0].cuda()
+        pos, step = L0[b], 1
+        while pos < L1[b]:
+            n = min(step, L1[b] - pos)
+            B_.mpfa_quantize_kv_paged(k[pos:pos + n].contiguous(), v[pos:pos + n].contiguous(), pos, w_full.H_q, flags,
+                                      st.stats.request(b), 1.0, st.kv, st.page_table[b], None)
+            pos += n
+            step = step % 37 + 5 if pos > L0[b] + 3 else 1   # a few single tokens, then ragged chunks
+    torch.cuda.synchronize()
+    # oracle: statistics from the first L0 tokens, then everything quantized with them
+    caches, refs = [], []
+    for b in range(3):
+        kb, vb = kv_full[b]
+        z0 = orc.stage1(orc.bf16_bits(w_full.q_sample[b:b + 1].contiguous()), orc.bf16_bits(kb[:, :L0[b]].contiguous()),
+                        orc.bf16_bits(vb[:, :L0[b]].contiguous()))
+        z = orc.stage1(orc.bf16_bits(w_full.q_sample[b:b + 1].contiguous()), orc.bf16_bits(kb), orc.bf16_bits(vb), frozen=z0)
+        zq = orc.stage1(orc.bf16_bits(w_full.q_new[b:b + 1].contiguous()), orc.bf16_bits(kb), orc.bf16_bits(vb), frozen=z0)
+        o32, _ = orc.decode(zq.q_codes[:, :, 0], zq.q_sf[:, :, 0], z.k_codes, z.k_sf, z.v_codes, z.delta, z.dq, z.dk, 1.0,
+                            w_full.softmax_scale, np.array([L1[b]], np.int32))
+        caches.append(z)
+        refs.append(o32[0])
+    st.w = w_full
+    check_cache(st, w_full, caches)
+    st.seq_lens.copy_(w_full.seq_lens.to(st.seq_lens.device))
+    decode_cache.decode_step(st)
+    torch.cuda.synchronize()
+    assert int(st.status.item()) == 0
+    compare(st, np.stack(refs))
