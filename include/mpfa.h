@@ -197,6 +197,22 @@ mpfa_status mpfa_prefill(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tensor *h_k,
                          float softmax_scale, void *out_bf16, float *out_f32, int32_t *device_status,
                          void *stream);
 
+/* QK4PV8 prefill of a chunk of queries against the paged cache (Section 6: the serving path keeps
+ * K/V only in low-bit pages; a later chunk of the prompt, or a prompt with a cached prefix,
+ * attends to them there).  q: [B, H_q, N_q] tile-layout tensor holding, for every request, the
+ * LAST N_q tokens of its context, quantized with the request's frozen statistics; seq_lens[b]
+ * (device) is the request's context length including those tokens, whose K/V must already be in
+ * the cache (mpfa_quantize_kv_paged).  Causal, bottom-right aligned: query i of the chunk sees
+ * keys 0 .. seq_lens[b] - N_q + i.  Same arithmetic and block order as mpfa_prefill (128-key
+ * blocks counted from key 0, visited last to first); lambda uses q_gscale[b] * k_gscale[b].
+ * Delta_S is applied when the cache has a delta_s pool.  A page-table entry outside
+ * [0, num_pages) raises MPFA_DEV_BAD_PAGE in *device_status (output of that request undefined,
+ * no out-of-pool access).  out_bf16 [B, N_q, H_q, 128]; out_f32 optional. */
+mpfa_status mpfa_prefill_paged(const mpfa_fp4_tensor *h_q, const mpfa_paged_kv *h_kv, const int32_t *page_table,
+                               int max_pages_per_req, const int32_t *seq_lens, const mpfa_stats *h_stats,
+                               float v_scale, float softmax_scale, void *out_bf16, float *out_f32,
+                               int32_t *device_status, void *stream);
+
 /* QK4PV8 decode (Section 5.3): one query token per request (q: tile-layout tensor with
  * N = 1, centered with the frozen means), its first seq_lens[b] keys found through
  * page_table [B, max_pages_per_req].  Each (request, kv head, 1024-token partition) keeps a

@@ -90,6 +90,9 @@ def lib() -> ctypes.CDLL:
         L.mpfa_decode.restype = i
         L.mpfa_decode.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_PagedKV), vp, i, vp, ctypes.POINTER(_Stats),
                                   f, f, vp, vp, vp, sz, vp, vp]
+        L.mpfa_prefill_paged.restype = i
+        L.mpfa_prefill_paged.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_PagedKV), vp, i, vp,
+                                         ctypes.POINTER(_Stats), f, f, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -281,6 +284,17 @@ def mpfa_decode(q: Fp4Tensor, kv: PagedKV, page_table: torch.Tensor, seq_lens: t
                            ctypes.byref(sc), v_scale, softmax_scale, _ptr(out), _ptr(out_f32), _ptr(workspace),
                            workspace.numel(), _ptr(device_status), _stream())
     _check(rc, "mpfa_decode")
+
+
+def mpfa_prefill_paged(q: Fp4Tensor, kv: PagedKV, page_table: torch.Tensor, seq_lens: torch.Tensor, stats: Stats,
+                       v_scale: float, softmax_scale: float, out: torch.Tensor, out_f32: Optional[torch.Tensor],
+                       device_status: torch.Tensor) -> None:
+    assert page_table.dtype == torch.int32 and page_table.is_contiguous() and seq_lens.dtype == torch.int32
+    sc, qc, kc = stats.c(), q.c(), kv.c()
+    rc = lib().mpfa_prefill_paged(ctypes.byref(qc), ctypes.byref(kc), _ptr(page_table), page_table.shape[1],
+                                  _ptr(seq_lens), ctypes.byref(sc), v_scale, softmax_scale, _ptr(out), _ptr(out_f32),
+                                  _ptr(device_status), _stream())
+    _check(rc, "mpfa_prefill_paged")
 
 
 # ---------------------------------------------------------------------------------------

@@ -78,10 +78,15 @@ enum {
                                         //     block c needs P V of block c-2, which needs the correction warps - so
                                         //     a slot is never two phases ahead of its reader
   BAR_O_FREE = BAR_L_FULL + 4,          // the epilogue has read both accumulators (phase = items with T > 0)
-  NUM_BARS = BAR_O_FREE + 1
+  BAR_SF_READY = BAR_O_FREE + 1,        // [KSTAGES] paged source only: scales and Delta_S of the stage re-tiled
+  NUM_BARS = BAR_SF_READY + KSTAGES
 };
 constexpr uint32_t OFF_MISC = OFF_BAR + NUM_BARS * 8;   // tmem base, abort flag
-constexpr uint32_t SMEM_BYTES = OFF_MISC + 16 + 1024;   // + slack for the 1024-byte alignment
+// paged source only: per K stage the two pages' scale bytes (2 x 512) and Delta_S rows (2 x 128) as stored
+constexpr uint32_t RAW_STAGE = 1280;
+constexpr uint32_t OFF_RAW = (OFF_MISC + 16 + 127) & ~127u;
+constexpr uint32_t SMEM_BYTES = OFF_MISC + 16 + 1024;                          // + slack for the 1024-byte alignment
+constexpr uint32_t SMEM_BYTES_PAGED = OFF_RAW + KSTAGES * RAW_STAGE + 1024;
 
 constexpr uint32_t TM_S = 0, TM_O0 = 128, TM_O1 = 256, TM_P0 = 384, TM_P1 = 416, TM_SFQ = 448 /* 2 x 8 */,
                    TM_SFK0 = 464, TM_SFK1 = 472;
@@ -99,6 +104,17 @@ struct PrefillParams {
   int B, N_q, N_kv, H_q, H_kv, nq_tiles, nk_tiles, n_items;
   int causal;
   float softmax_scale, v_scale;
+};
+
+// K, V and Delta_S read from the paged cache instead of contiguous tensors: 64-token pages whose
+// (page, kv head) slabs are stored as halves of this kernel's operand tiles (same swizzles), K scales
+// row-major [token][8] and Delta_S [page][q head][64] with its 16-byte groups XOR-ed by (q head mod G).
+struct PagedSrc {
+  const uint8_t *k_codes, *k_sf, *v_fp8;
+  const __nv_bfloat16 *delta;   // may be null
+  const int32_t *page_table;    // [B, max_pages]
+  const int32_t *seq_lens;      // [B] keys of each request (the last N_q of them are the queries' own)
+  int max_pages, num_pages;
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -193,9 +209,39 @@ struct Ctx {
   }
 };
 
+// Paged source: the two physical pages of KV block jb (t-th block of the traversal) of an item.  Every 16 blocks
+// the warp reads 32 page ids with one coalesced load (lane l: page index 2 jb + 1 - l); in between the ids come
+// from the lanes' registers.  A page past the end of the context (all its keys are masked) or with an id outside
+// the pool (reported in *status) is replaced by the block's other page, so operand tiles always hold finite bytes.
+struct PageLookup {
+  int ids;
+  __device__ __forceinline__ void get(const PagedSrc &pg, int32_t *status, int b, int nkv, int t, int jb, int lane,
+                                      int &page_lo, int &page_hi) {
+    if ((t & 15) == 0) {
+      const int n_pg = (nkv + 63) >> 6;
+      const int pi = 2 * jb + 1 - lane;
+      int id = -1;
+      if (pi >= 0 && pi < n_pg) {
+        id = pg.page_table[(size_t)b * pg.max_pages + pi];
+        if (id < 0 || id >= pg.num_pages) {
+          atomicOr(status, MPFA_DEV_BAD_PAGE);
+          id = -1;
+        }
+      }
+      ids = id;
+    }
+    page_hi = __shfl_sync(0xffffffffu, ids, (t & 15) * 2);
+    page_lo = __shfl_sync(0xffffffffu, ids, (t & 15) * 2 + 1);
+    if (page_hi < 0) page_hi = page_lo;
+    if (page_lo < 0) page_lo = page_hi < 0 ? 0 : page_hi;
+    if (page_hi < 0) page_hi = 0;
+  }
+};
+
 // One work item: a 128-row query tile of one q head.
 struct Tile {
   int b, hq, hk, qt, row0, T;   // T: KV blocks to visit
+  int nkv;                      // keys of this item's request
 };
 
 // The list of work items of this CTA.  Items are ordered by length (latest query tile first; all heads of a
@@ -205,7 +251,8 @@ struct Tile {
 struct TileWalk {
   int round;   // everything else is read from the kernel parameters (constant bank), not kept in registers
   __device__ __forceinline__ void init() { round = 0; }
-  __device__ __forceinline__ bool next(const PrefillParams &pp, Tile &t) {
+  template <bool PAGED>
+  __device__ __forceinline__ bool next(const PrefillParams &pp, const PagedSrc &pg, Tile &t) {
     const int c = (round & 1) ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
     const int i = round * (int)gridDim.x + c;
     ++round;
@@ -218,15 +265,18 @@ struct TileWalk {
     t.hk = t.hq / (pp.H_q / pp.H_kv);
     t.row0 = t.qt * TILE;
     const int last_row = min(pp.N_q - 1, t.row0 + TILE - 1);
-    const int last_key = pp.causal ? min(pp.N_kv - 1, last_row + (pp.N_kv - pp.N_q)) : pp.N_kv - 1;   // bottom-right aligned
+    const int n_kv = PAGED ? pg.seq_lens[t.b] : pp.N_kv;
+    t.nkv = n_kv;
+    const int last_key = pp.causal ? min(n_kv - 1, last_row + (n_kv - pp.N_q)) : n_kv - 1;   // bottom-right aligned
     t.T = last_key < 0 ? 0 : last_key / TILE + 1;
     return true;
   }
 };
 
+template <bool PAGED>
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-               const __grid_constant__ CUtensorMap tm_v, const PrefillParams p) {
+               const __grid_constant__ CUtensorMap tm_v, const PrefillParams p, const PagedSrc pg) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -259,10 +309,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
     for (int i = 0; i < 4; ++i) mbar_init(cx.bar(BAR_L_FULL + i), 8);
     mbar_init(cx.bar(BAR_O_FREE), 4);
+    for (int i = 0; i < KSTAGES; ++i) mbar_init(cx.bar(BAR_SF_READY + i), 1);
     mbar_init_fence();
     prefetch_tmap(&tm_q);
-    prefetch_tmap(&tm_k);
-    prefetch_tmap(&tm_v);
+    if (!PAGED) {
+      prefetch_tmap(&tm_k);
+      prefetch_tmap(&tm_v);
+    }
   }
   // rank-one operands: MN-major, 128B swizzle, K = 16.  Row k = 0 of each 64-element half
   // holds the data (ones / Delta_S), every other row stays zero for the CTA's lifetime.
@@ -301,7 +354,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // uniform registers); a single elected lane issues each copy.
     bool ok = true;
     uint32_t nk_armed = 0, nv_armed = 0, nq_armed = 0;
-    for (; ok && walk.next(p, tl); gb += tl.T, ++ti) {
+    for (; ok && walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
       const uint32_t qb = ti & 1;
       if (ti >= 2) ok = cx.wait(BAR_Q_EMPTY + qb, ((ti >> 1) - 1) & 1u);
       if (!ok) break;
@@ -314,14 +367,31 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                   cx.bar(BAR_Q_FULL + qb));
       }
       nq_armed = ti + 1;
+      PageLookup look;
       for (int t = 0; t < tl.T && ok; ++t) {
         const uint32_t c = gb + t;
         const int jb = tl.T - 1 - t;
         const uint32_t ks = c % KSTAGES, vs = c % VSTAGES;
+        int page_lo = 0, page_hi = 0;
+        if (PAGED) look.get(pg, p.status, tl.b, tl.nkv, t, jb, lane, page_lo, page_hi);
         if (c >= (uint32_t)KSTAGES) ok = cx.wait(BAR_K_EMPTY + ks, (c / KSTAGES - 1) & 1u);
         if (!ok) break;
         TR(0, c, 0);
-        if (elect_one()) {
+        if (PAGED) {
+          if (elect_one()) {
+            const uint32_t bar = cx.bar(BAR_K_FULL + ks);
+            mbar_expect_tx(bar, 8192 + 1024 + (has_delta ? 256 : 0));
+            const size_t s_lo = (size_t)page_lo * p.H_kv + tl.hk, s_hi = (size_t)page_hi * p.H_kv + tl.hk;
+            bulk_load(sbase + OFF_K + ks * 8192, pg.k_codes + s_lo * 4096, 4096, bar);
+            bulk_load(sbase + OFF_K + ks * 8192 + 4096, pg.k_codes + s_hi * 4096, 4096, bar);
+            bulk_load(sbase + OFF_RAW + ks * RAW_STAGE, pg.k_sf + s_lo * 512, 512, bar);
+            bulk_load(sbase + OFF_RAW + ks * RAW_STAGE + 512, pg.k_sf + s_hi * 512, 512, bar);
+            if (has_delta) {
+              bulk_load(sbase + OFF_RAW + ks * RAW_STAGE + 1024, pg.delta + ((size_t)page_lo * p.H_q + tl.hq) * 64, 128, bar);
+              bulk_load(sbase + OFF_RAW + ks * RAW_STAGE + 1152, pg.delta + ((size_t)page_hi * p.H_q + tl.hq) * 64, 128, bar);
+            }
+          }
+        } else if (elect_one()) {
           mbar_expect_tx(cx.bar(BAR_K_FULL + ks), 8192 + 1024 + (has_delta ? 256 : 0));
           tma_load_2d(sbase + OFF_K + ks * 8192, &tm_k, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_K_FULL + ks));
           bulk_load(sbase + OFF_SFK + ks * 1024, p.k_sf + (((size_t)tl.b * p.H_kv + tl.hk) * p.nk_tiles + jb) * 1024, 1024,
@@ -336,7 +406,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (c >= (uint32_t)VSTAGES) ok = cx.wait(BAR_V_EMPTY + vs, (c / VSTAGES - 1) & 1u);
         if (!ok) break;
         TR(0, c, 1);
-        if (elect_one()) {
+        if (PAGED) {
+          if (elect_one()) {
+            const uint32_t bar = cx.bar(BAR_V_FULL + vs);
+            mbar_expect_tx(bar, 16384);
+            bulk_load(sbase + OFF_V + vs * 16384, pg.v_fp8 + ((size_t)page_lo * p.H_kv + tl.hk) * 8192, 8192, bar);
+            bulk_load(sbase + OFF_V + vs * 16384 + 8192, pg.v_fp8 + ((size_t)page_hi * p.H_kv + tl.hk) * 8192, 8192, bar);
+          }
+        } else if (elect_one()) {
           mbar_expect_tx(cx.bar(BAR_V_FULL + vs), 16384);
           tma_load_2d(sbase + OFF_V + vs * 16384, &tm_v, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
         }
@@ -369,7 +446,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint64_t d_sfq00 = smem_desc(sbase + OFF_SFQ, 0, 128, SWZ_NONE);
     const uint64_t d_sfk0 = smem_desc(sbase + OFF_SFK, 0, 128, SWZ_NONE);
     bool ok = true;
-    for (; ok && walk.next(p, tl); gb += tl.T, ++ti) {
+    for (; ok && walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
       const uint32_t qb = ti & 1;
       ok = cx.wait(BAR_Q_FULL + qb, (ti >> 1) & 1u);
       if (!ok) break;
@@ -386,6 +463,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const uint32_t ks = c % KSTAGES, sb = c & 1;
         TR(5, c, 0);
         ok = cx.wait(BAR_K_FULL + ks, (c / KSTAGES) & 1u);
+        if (PAGED) ok = ok && cx.wait(BAR_SF_READY + ks, (c / KSTAGES) & 1u);
         if (!ok) break;
         const uint32_t tSFK = tm + (sb ? TM_SFK1 : TM_SFK0);
         const uint64_t d_sfk = d_sfk0 + (uint64_t)((ks * 1024) >> 4);
@@ -418,13 +496,42 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (ok && elect_one()) mma_commit(cx.bar(BAR_Q_EMPTY + qb));   // after every MMA that reads this query tile
       __syncwarp();
     }
+  } else if (PAGED && warp == 2) {
+    // ==== paged source: re-tile the K scales and un-swizzle Delta_S of every stage ====
+    const int G = p.H_q / p.H_kv;
+    bool ok = true;
+    for (; ok && walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
+      const int rsw = tl.hq % G;
+      for (int t = 0; t < tl.T && ok; ++t) {
+        const uint32_t c = gb + t;
+        const uint32_t ks = c % KSTAGES;
+        ok = cx.wait(BAR_K_FULL + ks, (c / KSTAGES) & 1u);
+        if (!ok) break;
+        const uint8_t *raw = smem + OFF_RAW + ks * RAW_STAGE;
+        // scales: row-major [key][8] -> the 32x128b tile layout tcgen05.cp expects (lane = key mod 32)
+        uint2 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) v[q] = *reinterpret_cast<const uint2 *>(raw + (q >> 1) * 512 + ((q & 1) * 32 + lane) * 8);
+        uint8_t *dst = smem + OFF_SFK + ks * 1024 + lane * 16;
+        *reinterpret_cast<uint4 *>(dst) = make_uint4(v[0].x, v[1].x, v[2].x, v[3].x);
+        *reinterpret_cast<uint4 *>(dst + 512) = make_uint4(v[0].y, v[1].y, v[2].y, v[3].y);
+        // Delta_S: 16-byte group c of a page is stored at c ^ (q head mod G); row 0 of the operand wants them in order
+        if (has_delta && lane < 16) {
+          const int half = lane >> 3, cg = lane & 7;
+          const uint4 d = *reinterpret_cast<const uint4 *>(raw + 1024 + half * 128 + ((cg ^ rsw) << 4));
+          *reinterpret_cast<uint4 *>(smem + OFF_DELTA + ks * 4096 + half * 2048 + (cg << 4)) = d;
+        }
+        fence_proxy_async_smem();
+        warp_arrive(cx.bar(BAR_SF_READY + ks), lane);
+      }
+    }
   } else if (warp == 3) {
     // =========================== P V issuer ===========================
     const uint32_t id_fp8 = idesc_e4m3(128, 128, 0, 1);
     const uint64_t d_v0 = smem_desc(sbase + OFF_V, 16, 1024, SWZ_128B);
     bool ok = true;
     uint32_t n_used = 0;   // items so far that used the accumulators (T > 0)
-    for (; ok && walk.next(p, tl); gb += tl.T, ++ti) {
+    for (; ok && walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
       if (tl.T == 0) continue;
       // the previous such item's epilogue has read both accumulators
       if (n_used >= 1) ok = cx.wait(BAR_O_FREE, (n_used - 1) & 1u);
@@ -469,10 +576,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t tS = tm + TM_S + lane_off;
     const uint32_t tP = tm + (grp ? TM_P1 : TM_P0) + lane_off;
     bool ok = true;
-    for (; ok && walk.next(p, tl); gb += tl.T, ++ti) {
+    for (; ok && walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
       const int T = tl.T;
       const int r_abs = tl.row0 + row;
-      const int limit = p.causal ? min(p.N_kv - 1, r_abs + (p.N_kv - p.N_q)) : p.N_kv - 1;   // last visible key
+      const int n_kv = PAGED ? tl.nkv : p.N_kv;
+      const int limit = p.causal ? min(n_kv - 1, r_abs + (n_kv - p.N_q)) : n_kv - 1;   // last visible key
       const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), gq[tl.b]), gk[tl.b]);
       float m_own = -INFINITY;   // running maximum after this group's previous block
       float l_own = 0.0f;        // sum of 448 P over this group's blocks, relative to m_own
@@ -624,7 +732,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const float *s_m = reinterpret_cast<const float *>(smem + OFF_M);
     const uint32_t tO0 = tm + TM_O0 + lane_off, tO1 = tm + TM_O1 + lane_off;
     bool ok = true;
-    for (; walk.next(p, tl); gb += tl.T, ++ti) {
+    for (; walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
       const int T = tl.T;
       const int r_abs = tl.row0 + row;
       const float lam_c = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[tl.b]), p.k_gscale[tl.b]);
@@ -844,8 +952,72 @@ extern "C" mpfa_status mpfa_prefill(const mpfa_fp4_tensor *q, const mpfa_fp4_ten
   MPFA_CUDA_OK(cudaGetDevice(&dev));
   MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
   const unsigned grid = (unsigned)(n_cta < (uint64_t)n_sm ? n_cta : (uint64_t)n_sm);   // one persistent CTA per SM
-  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-  prefill_kernel<<<grid, NTHREADS, SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p);
+  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+  prefill_kernel<false><<<grid, NTHREADS, SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+  MPFA_LAUNCH_OK();
+  return MPFA_OK;
+}
+
+extern "C" mpfa_status mpfa_prefill_paged(const mpfa_fp4_tensor *q, const mpfa_paged_kv *kv, const int32_t *page_table,
+                                          int max_pages_per_req, const int32_t *seq_lens, const mpfa_stats *st,
+                                          float v_scale, float softmax_scale, void *out_bf16, float *out_f32,
+                                          int32_t *device_status, void *stream) {
+  if (!q || !kv || !page_table || !seq_lens || !st || !out_bf16 || !device_status) return MPFA_ERR_INVALID_ARG;
+  if (!q->codes || !q->sf || !kv->k_codes || !kv->k_sf || !kv->v_fp8 || !st->q_gscale || !st->k_gscale)
+    return MPFA_ERR_INVALID_ARG;
+  if (q->B <= 0 || q->H <= 0 || q->N <= 0 || kv->num_pages <= 0 || max_pages_per_req <= 0) return MPFA_ERR_INVALID_ARG;
+  if (q->H != kv->H_q || kv->H_kv <= 0) return MPFA_ERR_INVALID_ARG;
+  if (!(softmax_scale > 0.0f) || !(v_scale > 0.0f)) return MPFA_ERR_INVALID_ARG;
+  if (kv->page_size != 64 || q->H % kv->H_kv != 0 || q->H / kv->H_kv > 8) return MPFA_ERR_UNSUPPORTED;
+  if (!aligned(q->codes, 1024) || !aligned(q->sf, 1024) || !aligned(kv->k_codes, 256) || !aligned(kv->k_sf, 256) ||
+      !aligned(kv->v_fp8, 256) || !aligned(kv->delta_s_bf16, 256) || !aligned(out_bf16, 16) || !aligned(out_f32, 16))
+    return MPFA_ERR_ALIGNMENT;
+  const int nq_tiles = pad128(q->N) / TILE;
+  const uint64_t q_rows = (uint64_t)q->B * q->H * nq_tiles * TILE;
+  if (q_rows >= (1ull << 31)) return MPFA_ERR_UNSUPPORTED;
+  const uint64_t n_cta = (uint64_t)q->B * q->H * nq_tiles;
+  mpfa_status rc = check_arch();
+  if (rc != MPFA_OK) return rc;
+  EncodeTiledFn enc;
+  rc = get_encoder(&enc);
+  if (rc != MPFA_OK) return rc;
+  CUtensorMap tq;
+  if ((rc = make_map(enc, &tq, q->codes, q_rows, 64)) != MPFA_OK) return rc;
+  PrefillParams p;
+  p.q_sf = q->sf;
+  p.k_sf = nullptr;
+  p.delta = static_cast<const __nv_bfloat16 *>(kv->delta_s_bf16);   // the kernel only tests it against null
+  p.q_gscale = st->q_gscale;
+  p.k_gscale = st->k_gscale;
+  p.out = static_cast<__nv_bfloat16 *>(out_bf16);
+  p.out_f32 = out_f32;
+  p.status = device_status;
+  p.B = q->B;
+  p.N_q = q->N;
+  p.N_kv = 0;
+  p.H_q = q->H;
+  p.H_kv = kv->H_kv;
+  p.nq_tiles = nq_tiles;
+  p.nk_tiles = 0;
+  p.causal = 1;
+  p.softmax_scale = softmax_scale;
+  p.v_scale = v_scale;
+  p.n_items = (int)n_cta;
+  PagedSrc pg;
+  pg.k_codes = kv->k_codes;
+  pg.k_sf = kv->k_sf;
+  pg.v_fp8 = kv->v_fp8;
+  pg.delta = static_cast<const __nv_bfloat16 *>(kv->delta_s_bf16);
+  pg.page_table = page_table;
+  pg.seq_lens = seq_lens;
+  pg.max_pages = max_pages_per_req;
+  pg.num_pages = kv->num_pages;
+  int dev = 0, n_sm = 0;
+  MPFA_CUDA_OK(cudaGetDevice(&dev));
+  MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  const unsigned grid = (unsigned)(n_cta < (uint64_t)n_sm ? n_cta : (uint64_t)n_sm);
+  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES_PAGED));
+  prefill_kernel<true><<<grid, NTHREADS, SMEM_BYTES_PAGED, static_cast<cudaStream_t>(stream)>>>(tq, tq, tq, p, pg);
   MPFA_LAUNCH_OK();
   return MPFA_OK;
 }
