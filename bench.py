@@ -215,6 +215,38 @@ def bench_decode(steps, warmup, peaks, small):
             "l2": "3.9 GB of cache per step vs 126 MB L2", "status": int(st.status.item())}
 
 
+def bench_prefill_paged(w, k, v, s1, out_ref, steps, warmup):
+    """The same prefill with K, V, scales and Delta_S read from a paged low-bit cache (64-token pages in a
+    shuffled pool) instead of contiguous tensors; the result must equal the contiguous kernel's bit for bit."""
+    from paper_2609_33135_b200 import binding as B_
+    dev = k.device
+    n_pages = (w.N_kv + 63) // 64
+    kv = B_.PagedKV.empty(n_pages, w.H_q, w.H_kv, with_delta=True, device=dev)
+    g = torch.Generator().manual_seed(1006)
+    table = torch.randperm(n_pages, generator=g).to(torch.int32).to(dev).view(1, -1).contiguous()
+    B_.mpfa_quantize_kv_paged(k[0], v[0], 0, w.H_q, B_.MPFA_SMOOTH | B_.MPFA_STATS_FROZEN, s1.stats.request(0), 1.0, kv,
+                              table[0], None)
+    seq = torch.tensor([w.N_kv], dtype=torch.int32, device=dev)
+    out = torch.empty_like(out_ref)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    run = lambda: B_.mpfa_prefill_paged(s1.q, kv, table, seq, s1.stats, 1.0, w.softmax_scale, out, None, status)
+    for _ in range(warmup):
+        run()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        a.record()
+        run()
+        b.record()
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in evs]
+    mean = sum(ms) / len(ms)
+    return {"workload": w.name + "_from_pages", "value": w.flops / (mean * 1e-3) / 1e12, "unit": "TFLOPS", "ms_mean": mean,
+            "ms_min": min(ms), "pages": n_pages, "page_order": "shuffled", "gpu_launches_per_step": 1,
+            "equals_contiguous_bitwise": bool(torch.equal(out.view(torch.uint16), out_ref.view(torch.uint16))),
+            "status": int(status.item())}
+
+
 def run_ours(args, rank, world, local):
     from paper_2609_33135_b200 import binding, workloads as wl
     binding.lib()  # fail loudly if the CUDA library is missing
@@ -357,6 +389,10 @@ def run_ours(args, rank, world, local):
                 result["decode"] = bench_decode(max(3, args.steps // 2), 3, peaks, args.small_decode)
             except Exception as e:  # decode is a secondary line; never lose the main one
                 result["decode"] = {"error": repr(e)}
+            try:
+                result["prefill_paged"] = bench_prefill_paged(w, k, v, s1, out, max(3, args.steps // 2), 3)
+            except Exception as e:
+                result["prefill_paged"] = {"error": repr(e)}
         if world == 1 and not args.no_cpu:
             cores = os.cpu_count() or 1
             fl, times, sample = cpu_oracle_sample(w, 1, rows_per_head=args.cpu_rows_per_head)
@@ -377,7 +413,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seq-len", type=int, default=16384)
-    ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-decode", action="store_true", help="skip the paged-cache workloads (decode, prefill from pages)")
     ap.add_argument("--small-decode", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-rows-per-head", type=int, default=8192)

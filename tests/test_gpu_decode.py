@@ -198,3 +198,36 @@ def test_append_into_partly_filled_pages_then_decode():
     torch.cuda.synchronize()
     assert int(st.status.item()) == 0
     compare(st, np.stack(refs))
+
+
+def test_decode_replays_from_a_cuda_graph():
+    """Section 5.3: the decode launch sequence (counter reset, split kernel, merge kernel) has a fixed shape, so
+    it can be captured once and replayed while sequence lengths, queries and cache contents change in place."""
+    from paper_2609_33135_b200 import binding as B_, decode_cache
+    w = wl.decode_workload("dec_graph", 91, 4, 8, 2, 300, 3000)
+    st = decode_cache.build_cache(w)
+    decode_cache.decode_step(st)          # eager run first: loads the kernels outside the capture
+    torch.cuda.synchronize()
+    eager_full = st.out.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        decode_cache.decode_step(st)
+    st.out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(st.status.item()) == 0
+    assert torch.equal(st.out.view(torch.uint16), eager_full.view(torch.uint16))
+    # shorter contexts and another query, written in place; the captured launches are reused unchanged
+    shorter = (w.seq_lens // 3 + 1).to(torch.int32)
+    st.seq_lens.copy_(shorter.to(st.seq_lens.device))
+    q2 = w.q_sample[:, 5:6].contiguous().cuda()
+    B_.mpfa_quantize_qk(q2, None, B_.MPFA_SMOOTH | B_.MPFA_STATS_FROZEN, st.stats, st.q4, None, None, None)
+    graph.replay()
+    torch.cuda.synchronize()
+    from_graph = st.out.clone()
+    st.out.zero_()
+    decode_cache.decode_step(st)
+    torch.cuda.synchronize()
+    assert int(st.status.item()) == 0
+    assert torch.equal(from_graph.view(torch.uint16), st.out.view(torch.uint16))
+    assert not torch.equal(from_graph.view(torch.uint16), eager_full.view(torch.uint16))
