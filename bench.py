@@ -247,6 +247,31 @@ def bench_prefill_paged(w, k, v, s1, out_ref, steps, warmup):
             "status": int(status.item())}
 
 
+def bench_compensation_overhead(binding, s1, w, reps=5):
+    """Cost of the rank-one compensation MMA (Section 5.2): the attention kernel with and without the Delta_S
+    operand, same quantized inputs, runs interleaved."""
+    dev = s1.q.codes.device
+    out = torch.empty(w.B, w.N_q, w.H_q, 128, dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    delta = s1.delta
+    t = {True: [], False: []}
+    try:
+        for i in range(2 * (reps + 1)):
+            with_delta = i % 2 == 0
+            s1.delta = delta if with_delta else None
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            binding.prefill(s1, w.causal, w.softmax_scale, out=out, status=status)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                t[with_delta].append(a.elapsed_time(b))
+    finally:
+        s1.delta = delta
+    on, off = sum(t[True]) / len(t[True]), sum(t[False]) / len(t[False])
+    return {"ms_with": on, "ms_without": off, "overhead_frac": on / off - 1.0, "status": int(status.item())}
+
+
 def run_ours(args, rank, world, local):
     from paper_2609_33135_b200 import binding, workloads as wl
     binding.lib()  # fail loudly if the CUDA library is missing
@@ -255,7 +280,10 @@ def run_ours(args, rank, world, local):
     peaks = load_peaks()
     dev = torch.device("cuda", local)
     N = args.seq_len
-    w = wl.config2_llama(N, seed=rank_seed(1002, rank))   # rank r: batch element r
+    if args.shape == "qwen":   # config 3: 40 q heads / 8 kv heads
+        w = wl.prefill_workload(f"cfg3_qwen14b_causal_{N}", rank_seed(1003, rank), 1, N, 40, 8, True)
+    else:
+        w = wl.config2_llama(N, seed=rank_seed(1002, rank))   # rank r: batch element r
     hq, hk, hv = w.q.pin_memory(), w.k.pin_memory(), w.v.pin_memory()
     q, k, v = hq.to(dev), hk.to(dev), hv.to(dev)
     s1 = binding.stage1(q, k, v)           # allocates outputs once; steps reuse them
@@ -366,7 +394,8 @@ def run_ours(args, rank, world, local):
         "vs_baseline": None, "dtype": "nvfp4 (QK^T) + fp8 e4m3 (PV), f32 accumulate", "data": "synthetic",
         "config": {"workload": w.name, "B_per_gpu": 1, "H_q": w.H_q, "H_kv": w.H_kv, "head_dim": 128, "N": N,
                    "causal": True, "parallelism": f"dp{world} (independent batch elements, no collective)",
-                   "l2": "inputs_exceed_l2 (Q+K+V 201 MB, output 134 MB per step vs 126 MB L2)",
+                   "l2": f"inputs_exceed_l2 (Q+K+V {(q.numel() + k.numel() + v.numel()) * 2 / 1e6:.0f} MB, "
+                         f"output {out.numel() * 2 / 1e6:.0f} MB per step vs 126 MB L2)",
                    "step": "quantize_qk + quantize_v + prefill"},
         "clocks": clocks,
         "e2e": {"value": whole_job_value(world, flops, e2e_ms), "unit": "TFLOPS", "ms_per_step": e2e_ms,
@@ -384,6 +413,10 @@ def run_ours(args, rank, world, local):
         "quantize_ms": ms_step - kernel_ms,
     }
     if rank == 0:
+        try:
+            result["compensation_mma"] = bench_compensation_overhead(binding, s1, w)
+        except Exception as e:
+            result["compensation_mma"] = {"error": repr(e)}
         if not args.no_decode:
             try:
                 result["decode"] = bench_decode(max(3, args.steps // 2), 3, peaks, args.small_decode)
@@ -413,6 +446,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seq-len", type=int, default=16384)
+    ap.add_argument("--shape", default="llama", choices=["llama", "qwen"], help="32:8 (configs 2, 4) or 40:8 heads (config 3)")
     ap.add_argument("--no-decode", action="store_true", help="skip the paged-cache workloads (decode, prefill from pages)")
     ap.add_argument("--small-decode", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
