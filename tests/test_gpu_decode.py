@@ -231,3 +231,23 @@ def test_decode_replays_from_a_cuda_graph():
     assert int(st.status.item()) == 0
     assert torch.equal(from_graph.view(torch.uint16), st.out.view(torch.uint16))
     assert not torch.equal(from_graph.view(torch.uint16), eager_full.view(torch.uint16))
+
+
+def test_decode_with_empty_contexts_in_the_batch():
+    """Degenerate case: requests whose context length is 0 (nothing to attend to) next to ordinary ones.  They
+    contribute no work item, their output is defined as zero, and the neighbours are unaffected."""
+    from paper_2609_33135_b200 import decode_cache
+    w = wl.decode_workload("dec_empty", 92, 5, 8, 2, 1, 1500, seq_lens=[5, 1300, 9, 1, 64])
+    st = decode_cache.build_cache(w)
+    st.seq_lens.copy_(torch.tensor([0, 1300, 0, 1, 0], dtype=torch.int32).to(st.seq_lens.device))
+    st.out.fill_(7.0)
+    st.out_f32.fill_(7.0)
+    decode_cache.decode_step(st)
+    torch.cuda.synchronize()
+    assert int(st.status.item()) == 0
+    got = st.out_f32.cpu().numpy()
+    for b in (0, 2, 4):
+        assert not got[b].any() and not st.out[b].float().cpu().numpy().any()
+    for b in (1, 3):
+        d = np.abs(got[b] - oracle_decode_one(w, b))
+        assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (b, float(d.max()), float(d.mean()))

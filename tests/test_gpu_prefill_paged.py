@@ -120,3 +120,31 @@ def test_paged_prefill_bad_page_is_reported_not_followed():
     B_.mpfa_prefill_paged(q4, st.kv, table, st.seq_lens, st.stats, 1.0, w.softmax_scale, out, None, status)
     torch.cuda.synchronize()
     assert int(status.item()) == B_.MPFA_DEV_BAD_PAGE
+
+
+def test_paged_prefill_more_queries_than_keys():
+    """Degenerate case: a chunk longer than the request's whole context (bottom-right aligned mask: the first
+    N_q - L rows see no key and must come out as zeros, a whole query tile may have no KV block at all) next to an
+    ordinary request in the same launch."""
+    from paper_2609_33135_b200 import binding as B_, decode_cache
+    L, N_q, H_q, H_kv = [50, 300], 200, 4, 2
+    w = wl.decode_workload("pp_short", 341, 2, H_q, H_kv, 1, 300, seq_lens=L)
+    st = decode_cache.build_cache(w)
+    q_chunk = w.q_sample[:, 10:10 + N_q].contiguous()
+    q4 = B_.Fp4Tensor.empty(2, H_q, N_q, "cuda")
+    B_.mpfa_quantize_qk(q_chunk.cuda(), None, B_.MPFA_SMOOTH | B_.MPFA_STATS_FROZEN, st.stats, q4, None, None, None)
+    out = torch.full((2, N_q, H_q, 128), 3.0, dtype=torch.bfloat16, device="cuda")
+    o32 = torch.full((2, N_q, H_q, 128), 3.0, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B_.mpfa_prefill_paged(q4, st.kv, st.page_table, st.seq_lens, st.stats, 1.0, w.softmax_scale, out, o32, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o16n, o32n = out.view(torch.uint16).cpu().numpy(), o32.cpu().numpy()
+    assert not o32n[0, :N_q - 50].any() and not o16n[0, :N_q - 50].any()
+    for b in range(2):
+        k, v = w.kv_for_request(b)
+        z0 = orc.stage1(orc.bf16_bits(w.q_sample[b:b + 1].contiguous()), orc.bf16_bits(k), orc.bf16_bits(v))
+        z = orc.stage1(orc.bf16_bits(q_chunk[b:b + 1].contiguous()), orc.bf16_bits(k), orc.bf16_bits(v), frozen=z0)
+        rows = orc.all_rows(1, H_q, N_q)
+        ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
+        compare(o16n[b:b + 1], o32n[b:b + 1], rows, ref32, f"request {b}")
