@@ -248,28 +248,28 @@ def bench_prefill_paged(w, k, v, s1, out_ref, steps, warmup):
 
 
 def bench_compensation_overhead(binding, s1, w, reps=5):
-    """Cost of the rank-one compensation MMA (Section 5.2): the attention kernel with and without the Delta_S
-    operand, same quantized inputs, runs interleaved."""
+    """Cost of the compensation term by placement (Sections 5.2 and 7.4): the attention kernel with the rank-one
+    seed MMA, without Delta_S, and with Delta_S added element-wise by the softmax threads; same quantized
+    inputs, runs interleaved."""
     dev = s1.q.codes.device
     out = torch.empty(w.B, w.N_q, w.H_q, 128, dtype=torch.bfloat16, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    delta = s1.delta
-    t = {True: [], False: []}
-    try:
-        for i in range(2 * (reps + 1)):
-            with_delta = i % 2 == 0
-            s1.delta = delta if with_delta else None
+    modes = {"mma": (s1.delta, 0), "none": (None, 0), "elementwise": (s1.delta, binding.MPFA_VARIANT_COMP_ELEMENTWISE)}
+    t = {m: [] for m in modes}
+    for i in range(reps + 1):
+        for m, (delta, variant) in modes.items():
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
-            binding.prefill(s1, w.causal, w.softmax_scale, out=out, status=status)
+            binding.mpfa_prefill_variant(s1.q, s1.k, s1.v_fp8, delta, s1.stats, s1.v_scale, w.causal, w.softmax_scale,
+                                         variant, out, None, status)
             b.record()
             torch.cuda.synchronize()
-            if i >= 2:
-                t[with_delta].append(a.elapsed_time(b))
-    finally:
-        s1.delta = delta
-    on, off = sum(t[True]) / len(t[True]), sum(t[False]) / len(t[False])
-    return {"ms_with": on, "ms_without": off, "overhead_frac": on / off - 1.0, "status": int(status.item())}
+            if i >= 1:
+                t[m].append(a.elapsed_time(b))
+    ms = {m: sum(v) / len(v) for m, v in t.items()}
+    return {"ms_with": ms["mma"], "ms_without": ms["none"], "overhead_frac": ms["mma"] / ms["none"] - 1.0,
+            "ms_elementwise": ms["elementwise"], "elementwise_overhead_frac": ms["elementwise"] / ms["none"] - 1.0,
+            "status": int(status.item())}
 
 
 def run_ours(args, rank, world, local):

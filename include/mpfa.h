@@ -197,6 +197,21 @@ mpfa_status mpfa_prefill(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tensor *h_k,
                          float softmax_scale, void *out_bf16, float *out_f32, int32_t *device_status,
                          void *stream);
 
+/* Ablation variants of mpfa_prefill (Section 7.4; same arguments, same outputs):
+ *   variant 0                             the product path, identical to mpfa_prefill;
+ *   MPFA_VARIANT_COMP_ELEMENTWISE         compensation placed on the softmax path (Section 3.2): the BF16 seed
+ *                                         MMA is not issued; the softmax threads load the same BF16 Delta_S values
+ *                                         and add them to the FP32 scores one by one, before masking and the
+ *                                         running maximum.  Same term, one FP32 rounding placed differently; it
+ *                                         exists to measure what the rank-one MMA saves.  With delta_s_bf16 == NULL
+ *                                         it is the same as variant 0.
+ * Any other value: MPFA_ERR_INVALID_ARG. */
+enum { MPFA_VARIANT_COMP_ELEMENTWISE = 1 };
+mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tensor *h_k, const uint8_t *v_fp8,
+                                 const void *delta_s_bf16, const mpfa_stats *h_stats, float v_scale, int causal,
+                                 float softmax_scale, int variant, void *out_bf16, float *out_f32,
+                                 int32_t *device_status, void *stream);
+
 /* QK4PV8 prefill of a chunk of queries against the paged cache (Section 6: the serving path keeps
  * K/V only in low-bit pages; a later chunk of the prompt, or a prompt with a cached prefix,
  * attends to them there).  q: [B, H_q, N_q] tile-layout tensor holding, for every request, the

@@ -353,13 +353,12 @@ static int visible_keys(int i, int Nq, int Nkv, int causal) {
  * Quantized inputs are the logical row-major arrays written by the quantizers
  * above.  delta may be NULL (no compensation).  out_f32: [n_rows, D] before the
  * final BF16 rounding, out_bf16: [n_rows, D]. */
-void mpfa_oracle_prefill_rows(const uint8_t *q_codes, const uint8_t *q_sf, const uint8_t *k_codes,
+static void prefill_rows_impl(const uint8_t *q_codes, const uint8_t *q_sf, const uint8_t *k_codes,
                               const uint8_t *k_sf, const uint8_t *v_codes, const uint16_t *delta,
                               const float *dq, const float *dk, float v_scale, float softmax_scale,
-                              int causal, int B, int Nq, int Nkv, int Hq, int Hkv, int block_kv,
-                              int reverse, int p_fp8, const int32_t *rows, int n_rows, float *out_f32,
-                              uint16_t *out_bf16) {
-  (void)B;
+                              int causal, int Nq, int Nkv, int Hq, int Hkv, int block_kv, int reverse,
+                              int p_fp8, int delta_elementwise, const int32_t *rows, int n_rows,
+                              float *out_f32, uint16_t *out_bf16) {
   init_tables();
   int grp = Hq / Hkv;
 #pragma omp parallel for schedule(dynamic, 1)
@@ -372,7 +371,12 @@ void mpfa_oracle_prefill_rows(const uint8_t *q_codes, const uint8_t *q_sf, const
                   q_sf + (((size_t)b * Hq + hq) * Nq + i) * NBLK,
                   k_codes + ((size_t)b * Hkv + hk) * Nkv * (D / 2),
                   k_sf + ((size_t)b * Hkv + hk) * Nkv * NBLK,
-                  delta ? delta + ((size_t)b * Hq + hq) * Nkv : NULL, n, s);
+                  (delta && !delta_elementwise) ? delta + ((size_t)b * Hq + hq) * Nkv : NULL, n, s);
+    if (delta && delta_elementwise) {
+      /* Section 7.4, element-wise placement: the same BF16 term added to the finished FP32 score */
+      const uint16_t *dr = delta + ((size_t)b * Hq + hq) * Nkv;
+      for (int j = 0; j < n; ++j) s[j] = s[j] + mpfa_oracle_bf16_to_f32(dr[j]);
+    }
     float lam = ((softmax_scale * 1.4426950408889634f) * dq[b]) * dk[b];
     softmax_state st;
     online_softmax_pv(s, 0, n, lam, v_codes + ((size_t)b * Hkv + hk) * Nkv * D, NULL, block_kv,
@@ -384,6 +388,32 @@ void mpfa_oracle_prefill_rows(const uint8_t *q_codes, const uint8_t *q_sf, const
     }
     free(s);
   }
+}
+
+void mpfa_oracle_prefill_rows(const uint8_t *q_codes, const uint8_t *q_sf, const uint8_t *k_codes,
+                              const uint8_t *k_sf, const uint8_t *v_codes, const uint16_t *delta,
+                              const float *dq, const float *dk, float v_scale, float softmax_scale,
+                              int causal, int B, int Nq, int Nkv, int Hq, int Hkv, int block_kv,
+                              int reverse, int p_fp8, const int32_t *rows, int n_rows, float *out_f32,
+                              uint16_t *out_bf16) {
+  (void)B;
+  prefill_rows_impl(q_codes, q_sf, k_codes, k_sf, v_codes, delta, dq, dk, v_scale, softmax_scale, causal, Nq, Nkv,
+                    Hq, Hkv, block_kv, reverse, p_fp8, 0, rows, n_rows, out_f32, out_bf16);
+}
+
+/* Ablation variant (Section 7.4, compensation placement): identical to the function above except that
+ * Delta_S is not the seed of the score accumulator but is added, in FP32, to the finished score of the
+ * block-scaled products ("element-wise placement uses FP32 scalar addition").  The BF16 values of Delta_S
+ * are the same in both placements here, so the two differ by where one FP32 rounding falls. */
+void mpfa_oracle_prefill_rows_elementwise(const uint8_t *q_codes, const uint8_t *q_sf, const uint8_t *k_codes,
+                                          const uint8_t *k_sf, const uint8_t *v_codes, const uint16_t *delta,
+                                          const float *dq, const float *dk, float v_scale, float softmax_scale,
+                                          int causal, int B, int Nq, int Nkv, int Hq, int Hkv, int block_kv,
+                                          int reverse, int p_fp8, const int32_t *rows, int n_rows,
+                                          float *out_f32, uint16_t *out_bf16) {
+  (void)B;
+  prefill_rows_impl(q_codes, q_sf, k_codes, k_sf, v_codes, delta, dq, dk, v_scale, softmax_scale, causal, Nq, Nkv,
+                    Hq, Hkv, block_kv, reverse, p_fp8, 1, rows, n_rows, out_f32, out_bf16);
 }
 
 /* QK4PV8 decode (Section 5.3): one query token per request against its first

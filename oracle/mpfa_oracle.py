@@ -192,8 +192,9 @@ def stage1(q: np.ndarray, k: np.ndarray, v: np.ndarray, smooth: bool = True, v_s
 # --- stage 2 -------------------------------------------------------------------
 def prefill_rows(z: Quantized, rows: np.ndarray, softmax_scale: float, causal: bool,
                  block_kv: int = BLOCK_KV, reverse: bool = True, p_fp8: bool = True,
-                 use_delta: bool = True):
-    """QK4PV8 prefill outputs for rows [n,3]=(b,hq,i): (FP32 [n,128], BF16 bits [n,128])."""
+                 use_delta: bool = True, elementwise: bool = False):
+    """QK4PV8 prefill outputs for rows [n,3]=(b,hq,i): (FP32 [n,128], BF16 bits [n,128]).
+    elementwise=True: the ablation placement of Section 7.4 (Delta_S added to the finished FP32 score)."""
     rows = _c(rows, np.int32)
     B, Hq, Nq, _ = z.q_codes.shape
     Hkv, Nkv = z.k_codes.shape[1], z.k_codes.shape[2]
@@ -201,11 +202,10 @@ def prefill_rows(z: Quantized, rows: np.ndarray, softmax_scale: float, causal: b
     o32 = np.empty((n, D), np.float32)
     o16 = np.empty((n, D), np.uint16)
     delta = z.delta if use_delta else None
-    lib().mpfa_oracle_prefill_rows(_p(z.q_codes), _p(z.q_sf), _p(z.k_codes), _p(z.k_sf), _p(z.v_codes),
-                                   _p(delta), _p(_c(z.dq, np.float32)), _p(_c(z.dk, np.float32)),
-                                   ctypes.c_float(z.v_scale), ctypes.c_float(softmax_scale), int(causal),
-                                   B, Nq, Nkv, Hq, Hkv, block_kv, int(reverse), int(p_fp8), _p(rows), n,
-                                   _p(o32), _p(o16))
+    fn = lib().mpfa_oracle_prefill_rows_elementwise if elementwise else lib().mpfa_oracle_prefill_rows
+    fn(_p(z.q_codes), _p(z.q_sf), _p(z.k_codes), _p(z.k_sf), _p(z.v_codes), _p(delta), _p(_c(z.dq, np.float32)),
+       _p(_c(z.dk, np.float32)), ctypes.c_float(z.v_scale), ctypes.c_float(softmax_scale), int(causal), B, Nq, Nkv, Hq,
+       Hkv, block_kv, int(reverse), int(p_fp8), _p(rows), n, _p(o32), _p(o16))
     return o32, o16
 
 

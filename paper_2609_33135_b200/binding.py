@@ -20,6 +20,7 @@ MPFA_SMOOTH = 1
 MPFA_STATS_FROZEN = 2
 MPFA_DEV_TIMEOUT = 1
 MPFA_DEV_BAD_PAGE = 2
+MPFA_VARIANT_COMP_ELEMENTWISE = 1
 HEAD_DIM = 128
 PAGE = 64
 
@@ -90,6 +91,9 @@ def lib() -> ctypes.CDLL:
         L.mpfa_decode.restype = i
         L.mpfa_decode.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_PagedKV), vp, i, vp, ctypes.POINTER(_Stats),
                                   f, f, vp, vp, vp, sz, vp, vp]
+        L.mpfa_prefill_variant.restype = i
+        L.mpfa_prefill_variant.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_Fp4), vp, vp, ctypes.POINTER(_Stats), f, i,
+                                           f, i, vp, vp, vp, vp]
         L.mpfa_prefill_paged.restype = i
         L.mpfa_prefill_paged.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_PagedKV), vp, i, vp,
                                          ctypes.POINTER(_Stats), f, f, vp, vp, vp, vp]
@@ -268,6 +272,16 @@ def mpfa_prefill(q: Fp4Tensor, k: Fp4Tensor, v_fp8: torch.Tensor, delta: Optiona
     rc = lib().mpfa_prefill(ctypes.byref(qc), ctypes.byref(kc), _ptr(v_fp8), _ptr(delta), ctypes.byref(sc), v_scale,
                             int(causal), softmax_scale, _ptr(out), _ptr(out_f32), _ptr(device_status), _stream())
     _check(rc, "mpfa_prefill")
+
+
+def mpfa_prefill_variant(q: Fp4Tensor, k: Fp4Tensor, v_fp8: torch.Tensor, delta: Optional[torch.Tensor], stats: Stats,
+                         v_scale: float, causal: bool, softmax_scale: float, variant: int, out: torch.Tensor,
+                         out_f32: Optional[torch.Tensor], device_status: torch.Tensor) -> None:
+    sc, qc, kc = stats.c(), q.c(), k.c()
+    rc = lib().mpfa_prefill_variant(ctypes.byref(qc), ctypes.byref(kc), _ptr(v_fp8), _ptr(delta), ctypes.byref(sc), v_scale,
+                                    int(causal), softmax_scale, int(variant), _ptr(out), _ptr(out_f32),
+                                    _ptr(device_status), _stream())
+    _check(rc, "mpfa_prefill_variant")
 
 
 def decode_workspace(B: int, H_q: int, H_kv: int, max_pages: int, device="cuda") -> torch.Tensor:

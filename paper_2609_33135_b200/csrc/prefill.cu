@@ -273,7 +273,9 @@ struct TileWalk {
   }
 };
 
-template <bool PAGED>
+// EW: ablation variant of Section 7.4 (compensation placement): Delta_S is not seeded by the BF16 MMA but
+// loaded by the softmax warps and added to the scores element by element in FP32, before masking and the maximum.
+template <bool PAGED, bool EW>
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const PrefillParams p, const PagedSrc pg) {
@@ -333,7 +335,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   tc_fence_after();
   const uint32_t tm = *tmem_slot;
 
-  const bool has_delta = p.delta != nullptr;
+  const bool has_delta = !EW && p.delta != nullptr;   // operand of the seed MMA
   TR_INIT();
   if (warp == 12) TR(0, 255, 2);   // roles start (after setup)
 
@@ -619,6 +621,21 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           tmem_ld32(tS + 64, s2);
           tmem_ld32(tS + 96, s3);
         }
+        if constexpr (EW) {
+          const uint4 *dp = reinterpret_cast<const uint4 *>(
+              p.delta + ((size_t)tl.b * p.H_q + tl.hq) * (size_t)(p.nk_tiles * TILE) + key0);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint4 d = __ldg(dp + i);
+            const uint32_t w[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              s[8 * i + 2 * j] = __float_as_uint(__fadd_rn(__uint_as_float(s[8 * i + 2 * j]), __uint_as_float(w[j] << 16)));
+              s[8 * i + 2 * j + 1] =
+                  __float_as_uint(__fadd_rn(__uint_as_float(s[8 * i + 2 * j + 1]), __uint_as_float(w[j] & 0xFFFF0000u)));
+            }
+          }
+        }
         if (ragged) {
 #pragma unroll
           for (int i = 0; i < 64; ++i)
@@ -637,6 +654,22 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         tc_fence_before();
         warp_arrive(cx.bar(BAR_S_EMPTY), lane);   // the row is in registers: Q K^T of block c+1 may overwrite it
         TR(2 + grp, c, 2);
+        if constexpr (EW) {
+          const uint4 *dp = reinterpret_cast<const uint4 *>(
+              p.delta + ((size_t)tl.b * p.H_q + tl.hq) * (size_t)(p.nk_tiles * TILE) + key0 + 64);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint4 d = __ldg(dp + i);
+            const uint32_t w[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              s[64 + 8 * i + 2 * j] =
+                  __float_as_uint(__fadd_rn(__uint_as_float(s[64 + 8 * i + 2 * j]), __uint_as_float(w[j] << 16)));
+              s[64 + 8 * i + 2 * j + 1] =
+                  __float_as_uint(__fadd_rn(__uint_as_float(s[64 + 8 * i + 2 * j + 1]), __uint_as_float(w[j] & 0xFFFF0000u)));
+            }
+          }
+        }
         if (ragged) {
 #pragma unroll
           for (int i = 64; i < 128; ++i)
@@ -906,6 +939,16 @@ extern "C" mpfa_status mpfa_prefill(const mpfa_fp4_tensor *q, const mpfa_fp4_ten
                                     const void *delta_s_bf16, const mpfa_stats *st, float v_scale, int causal,
                                     float softmax_scale, void *out_bf16, float *out_f32, int32_t *device_status,
                                     void *stream) {
+  return mpfa_prefill_variant(q, k, v_fp8, delta_s_bf16, st, v_scale, causal, softmax_scale, 0, out_bf16, out_f32,
+                              device_status, stream);
+}
+
+extern "C" mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *q, const mpfa_fp4_tensor *k, const uint8_t *v_fp8,
+                                            const void *delta_s_bf16, const mpfa_stats *st, float v_scale, int causal,
+                                            float softmax_scale, int variant, void *out_bf16, float *out_f32,
+                                            int32_t *device_status, void *stream) {
+  if (variant != 0 && variant != MPFA_VARIANT_COMP_ELEMENTWISE) return MPFA_ERR_INVALID_ARG;
+  const bool ew = variant == MPFA_VARIANT_COMP_ELEMENTWISE && delta_s_bf16 != nullptr;
   if (!q || !k || !v_fp8 || !st || !out_bf16 || !device_status) return MPFA_ERR_INVALID_ARG;
   if (!q->codes || !q->sf || !k->codes || !k->sf || !st->q_gscale || !st->k_gscale) return MPFA_ERR_INVALID_ARG;
   if (q->B <= 0 || q->B != k->B || q->H <= 0 || k->H <= 0 || q->N <= 0 || k->N <= 0) return MPFA_ERR_INVALID_ARG;
@@ -952,8 +995,13 @@ extern "C" mpfa_status mpfa_prefill(const mpfa_fp4_tensor *q, const mpfa_fp4_ten
   MPFA_CUDA_OK(cudaGetDevice(&dev));
   MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
   const unsigned grid = (unsigned)(n_cta < (uint64_t)n_sm ? n_cta : (uint64_t)n_sm);   // one persistent CTA per SM
-  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-  prefill_kernel<false><<<grid, NTHREADS, SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+  if (ew) {
+    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    prefill_kernel<false, true><<<grid, NTHREADS, SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+  } else {
+    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    prefill_kernel<false, false><<<grid, NTHREADS, SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+  }
   MPFA_LAUNCH_OK();
   return MPFA_OK;
 }
@@ -1016,8 +1064,8 @@ extern "C" mpfa_status mpfa_prefill_paged(const mpfa_fp4_tensor *q, const mpfa_p
   MPFA_CUDA_OK(cudaGetDevice(&dev));
   MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
   const unsigned grid = (unsigned)(n_cta < (uint64_t)n_sm ? n_cta : (uint64_t)n_sm);
-  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES_PAGED));
-  prefill_kernel<true><<<grid, NTHREADS, SMEM_BYTES_PAGED, static_cast<cudaStream_t>(stream)>>>(tq, tq, tq, p, pg);
+  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES_PAGED));
+  prefill_kernel<true, false><<<grid, NTHREADS, SMEM_BYTES_PAGED, static_cast<cudaStream_t>(stream)>>>(tq, tq, tq, p, pg);
   MPFA_LAUNCH_OK();
   return MPFA_OK;
 }

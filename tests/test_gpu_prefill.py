@@ -111,3 +111,34 @@ def test_prefill_multi_tile_sampled_rows():
     ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
     o16, o32 = run_gpu(w)
     compare(o16, o32, rows, ref32, "4k")
+
+
+def test_prefill_elementwise_compensation_variant():
+    """Ablation variant (Section 7.4): Delta_S added by the softmax threads instead of the seed MMA.  Checked against
+    the oracle's statement of that placement; against the product path the outputs may differ by the place of one
+    FP32 rounding per score (on small inputs they are often identical)."""
+    from paper_2609_33135_b200 import binding as B_
+    w = wl.prefill_workload("ew", 59, 2, 333, 4, 2, True, q_bias=True)
+    s1 = B_.stage1(w.q.cuda(), w.k.cuda(), w.v.cuda())
+    out = torch.empty(w.B, w.N_q, w.H_q, 128, dtype=torch.bfloat16, device="cuda")
+    o32 = torch.empty(w.B, w.N_q, w.H_q, 128, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B_.mpfa_prefill_variant(s1.q, s1.k, s1.v_fp8, s1.delta, s1.stats, 1.0, True, w.softmax_scale,
+                            B_.MPFA_VARIANT_COMP_ELEMENTWISE, out, o32, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+    rows = orc.all_rows(w.B, w.H_q, w.N_q)
+    ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True, elementwise=True)
+    compare(out.view(torch.uint16).cpu().numpy(), o32.cpu().numpy(), rows, ref32, "elementwise")
+    _, seeded32, _ = B_.prefill(s1, True, w.softmax_scale, want_f32=True)
+    torch.cuda.synchronize()
+    d = (seeded32 - o32).abs()
+    assert float(d.mean()) < 1e-4
+    # variant 0 is the product path itself
+    o32b = torch.empty_like(o32)
+    B_.mpfa_prefill_variant(s1.q, s1.k, s1.v_fp8, s1.delta, s1.stats, 1.0, True, w.softmax_scale, 0, out, o32b, status)
+    torch.cuda.synchronize()
+    assert torch.equal(o32b, seeded32)
+    with pytest.raises(Exception):
+        B_.mpfa_prefill_variant(s1.q, s1.k, s1.v_fp8, s1.delta, s1.stats, 1.0, True, w.softmax_scale, 7, out, o32b, status)

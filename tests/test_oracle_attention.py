@@ -178,3 +178,34 @@ def test_decode_single_split_equals_prefill_row_and_merge_is_lse():
     z0, _ = orc.decode(qc, qs, z.k_codes, z.k_sf, z.v_codes, z.delta, z.dq, z.dk, 1.0, w.softmax_scale,
                        np.array([0], np.int32))
     assert not z0.any()
+
+
+def test_elementwise_placement_adds_the_same_term_after_the_products():
+    """Section 7.4 (compensation placement): the ablation variant adds Delta_S to the finished FP32 score instead of
+    seeding the accumulator with it.  Pinned against an FP64 recomputation from the decoded operands (a dropped
+    term or a wrong sign would be off by the size of Delta_S itself), against the seeded placement (same term: only
+    rounding-level differences), and without Delta_S the two must be the same function."""
+    from test_oracle_stage1 import _dequant
+    w = wl.config1b_tiny_qbias()
+    z = _stage1(w)
+    rows = np.array([[0, 0, 0], [0, 0, 3], [0, 0, 127], [0, 0, 128], [0, 0, 255]], np.int32)
+    ew32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True, p_fp8=False, elementwise=True)
+    qd = _dequant(z.q_codes, z.q_sf, np.ones(1, np.float32)).astype(np.float64)[0, 0]
+    kd = _dequant(z.k_codes, z.k_sf, np.ones(1, np.float32)).astype(np.float64)[0, 0]
+    dl = orc.bits_to_f32(z.delta[0, 0]).astype(np.float64)
+    vd = np.vectorize(lambda c: e4m3_value(int(c)))(z.v_codes[0, 0]).astype(np.float64)
+    lam = float(np.float32(w.softmax_scale)) * float(z.dq[0]) * float(z.dk[0])
+    assert np.abs(dl).max() * lam > 0.5            # the term matters in this workload
+    for r, i in enumerate(rows[:, 2]):
+        s = (kd[:i + 1] @ qd[i] + dl[:i + 1]) * lam
+        p = np.exp(s - s.max())
+        ref = (p / p.sum()) @ vd[:i + 1]
+        assert np.max(np.abs(ew32[r] - ref)) <= 2e-5 * max(1.0, np.abs(ref).max()), i
+    all_rows = orc.all_rows(1, 1, 256)
+    seeded, _ = orc.prefill_rows(z, all_rows, w.softmax_scale, True)
+    added, _ = orc.prefill_rows(z, all_rows, w.softmax_scale, True, elementwise=True)
+    d = np.abs(seeded - added)
+    assert d.mean() < 1e-4 and d.max() < 0.05     # an FP32 rounding of S can flip an E4M3 code of P now and then
+    a, _ = orc.prefill_rows(z, all_rows, w.softmax_scale, True, use_delta=False)
+    b, _ = orc.prefill_rows(z, all_rows, w.softmax_scale, True, use_delta=False, elementwise=True)
+    assert np.array_equal(a, b)
