@@ -413,10 +413,11 @@ def run_ours(args, rank, world, local):
         "quantize_ms": ms_step - kernel_ms,
     }
     if rank == 0:
-        try:
-            result["compensation_mma"] = bench_compensation_overhead(binding, s1, w)
-        except Exception as e:
-            result["compensation_mma"] = {"error": repr(e)}
+        if args.compensation or not args.no_decode:
+            try:
+                result["compensation_mma"] = bench_compensation_overhead(binding, s1, w)
+            except Exception as e:
+                result["compensation_mma"] = {"error": repr(e)}
         if not args.no_decode:
             try:
                 result["decode"] = bench_decode(max(3, args.steps // 2), 3, peaks, args.small_decode)
@@ -447,7 +448,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seq-len", type=int, default=16384)
     ap.add_argument("--shape", default="llama", choices=["llama", "qwen"], help="32:8 (configs 2, 4) or 40:8 heads (config 3)")
-    ap.add_argument("--no-decode", action="store_true", help="skip the paged-cache workloads (decode, prefill from pages)")
+    ap.add_argument("--no-decode", action="store_true",
+                    help="main line only: skip decode, prefill from pages and the compensation-placement timing")
+    ap.add_argument("--compensation", action="store_true", help="time the compensation placements even with --no-decode")
     ap.add_argument("--small-decode", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-rows-per-head", type=int, default=8192)
