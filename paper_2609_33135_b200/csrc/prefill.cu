@@ -46,6 +46,16 @@ constexpr int VSTAGES = 3;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM clock: far beyond any legitimate wait
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;       // drain path only
 constexpr int NTHREADS = 512;
+// setmaxnreg only moves registers inside the pool the CTA got at launch (512 threads x the 128 registers of the
+// launch bound); a request beyond the pool would block forever, so the split is checked here.
+#ifndef MPFA_REGS_SOFTMAX
+#define MPFA_REGS_SOFTMAX 168
+#define MPFA_REGS_UTIL 88
+#define MPFA_REGS_CORR 88
+#endif
+constexpr int REGS_SOFTMAX = MPFA_REGS_SOFTMAX, REGS_UTIL = MPFA_REGS_UTIL, REGS_CORR = MPFA_REGS_CORR;
+static_assert(4 * REGS_UTIL + 8 * REGS_SOFTMAX + 4 * REGS_CORR <= 16 * 128, "register pool");
+static_assert(REGS_SOFTMAX % 8 == 0 && REGS_UTIL % 8 == 0 && REGS_CORR % 8 == 0 && REGS_UTIL >= 24 && REGS_CORR >= 24, "setmaxnreg granularity");
 
 constexpr uint32_t OFF_Q = 0;                               // 2 tiles (the next tile's queries are prefetched)
 constexpr uint32_t OFF_K = OFF_Q + 2 * 8192;
@@ -349,7 +359,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   uint32_t gb = 0;   // KV blocks of the items already walked
   uint32_t ti = 0;   // index of the current item in this CTA's list
 
-  if (warp < 4) setmaxnreg_dec<88>();
+  if (warp < 4) setmaxnreg_dec<REGS_UTIL>();
   if (warp == 0) {
     // =========================== TMA producer ===========================
     // The whole warp runs the loop (uniform control flow keeps addresses and barrier handles in
@@ -569,7 +579,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
   } else if (warp >= 4 && warp < 12) {
     // =========================== softmax groups ===========================
-    setmaxnreg_inc<168>();
+    setmaxnreg_inc<REGS_SOFTMAX>();
     const int grp = (warp - 4) >> 2;                 // takes the KV blocks whose running count has this parity
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
@@ -759,7 +769,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
   } else if (warp >= 12) {
     // =========================== correction + epilogue ===========================
-    setmaxnreg_dec<88>();
+    setmaxnreg_dec<REGS_CORR>();
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const float *s_m = reinterpret_cast<const float *>(smem + OFF_M);
