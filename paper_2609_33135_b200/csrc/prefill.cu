@@ -26,7 +26,8 @@
 //                (the older one times the last alpha) and writes O / (448 l) * v_scale as BF16.
 // Tensor memory (512 columns): S [0,128) O0 [128,256) O1 [256,384), P_hat0 [384,416)
 // P_hat1 [416,448), scale factors of Q [448,456) and of two K blocks [456,464) [464,472).
-// Register budget is moved between the roles with setmaxnreg (88 / 168 / 168 / 88).
+// Register budget is moved between the roles with setmaxnreg (56 for warps 0-3, 168 for the softmax warps,
+// 120 for the correction warps, whose epilogue holds two accumulator chunks at once).
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises MPFA_DEV_TIMEOUT in
 // *device_status, all roles leave their loops, outstanding TMA copies are drained and
@@ -48,14 +49,19 @@ constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;       // drain path only
 constexpr int NTHREADS = 512;
 // setmaxnreg only moves registers inside the pool the CTA got at launch (512 threads x the 128 registers of the
 // launch bound); a request beyond the pool would block forever, so the split is checked here.
-#ifndef MPFA_REGS_SOFTMAX
-#define MPFA_REGS_SOFTMAX 168
-#define MPFA_REGS_UTIL 88
-#define MPFA_REGS_CORR 88
+#ifndef MPFA_REGS_UTIL_PAGED
+#define MPFA_REGS_UTIL_PAGED 88
+#define MPFA_REGS_CORR_PAGED 88
 #endif
-constexpr int REGS_SOFTMAX = MPFA_REGS_SOFTMAX, REGS_UTIL = MPFA_REGS_UTIL, REGS_CORR = MPFA_REGS_CORR;
-static_assert(4 * REGS_UTIL + 8 * REGS_SOFTMAX + 4 * REGS_CORR <= 16 * 128, "register pool");
-static_assert(REGS_SOFTMAX % 8 == 0 && REGS_UTIL % 8 == 0 && REGS_CORR % 8 == 0 && REGS_UTIL >= 24 && REGS_CORR >= 24, "setmaxnreg granularity");
+constexpr int REGS_SOFTMAX = 168;
+// measured: the contiguous kernel gains 4 % when the correction warps' epilogue (two accumulator chunks in
+// registers) does not spill; the paged variant's producer and re-tiling warps want the registers instead
+template <bool PAGED> constexpr int REGS_UTIL = PAGED ? MPFA_REGS_UTIL_PAGED : 56;
+template <bool PAGED> constexpr int REGS_CORR = PAGED ? MPFA_REGS_CORR_PAGED : 120;
+static_assert(4 * REGS_UTIL<false> + 8 * REGS_SOFTMAX + 4 * REGS_CORR<false> <= 16 * 128, "register pool");
+static_assert(4 * REGS_UTIL<true> + 8 * REGS_SOFTMAX + 4 * REGS_CORR<true> <= 16 * 128, "register pool");
+static_assert(REGS_SOFTMAX % 8 == 0 && REGS_UTIL<false> % 8 == 0 && REGS_CORR<false> % 8 == 0 && REGS_UTIL<true> % 8 == 0 &&
+              REGS_CORR<true> % 8 == 0, "setmaxnreg granularity");
 
 constexpr uint32_t OFF_Q = 0;                               // 2 tiles (the next tile's queries are prefetched)
 constexpr uint32_t OFF_K = OFF_Q + 2 * 8192;
@@ -359,7 +365,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   uint32_t gb = 0;   // KV blocks of the items already walked
   uint32_t ti = 0;   // index of the current item in this CTA's list
 
-  if (warp < 4) setmaxnreg_dec<REGS_UTIL>();
+  if (warp < 4) setmaxnreg_dec<REGS_UTIL<PAGED>>();
   if (warp == 0) {
     // =========================== TMA producer ===========================
     // The whole warp runs the loop (uniform control flow keeps addresses and barrier handles in
@@ -769,7 +775,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
   } else if (warp >= 12) {
     // =========================== correction + epilogue ===========================
-    setmaxnreg_dec<REGS_CORR>();
+    setmaxnreg_dec<REGS_CORR<PAGED>>();
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const float *s_m = reinterpret_cast<const float *>(smem + OFF_M);
