@@ -814,12 +814,25 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const float *__restri
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
   float l = 0.0f, o = 0.0f;
-  for (int s = 0; s < ns; ++s) {
-    const float ms = base[(size_t)s * PART_FLOATS];
-    if (ms == -INFINITY) continue;
-    const float w = ex2_approx(__fmul_rn(ms - M, lam));
-    l = __fadd_rn(l, __fmul_rn(w, base[(size_t)s * PART_FLOATS + 1]));
-    o = __fadd_rn(o, __fmul_rn(w, base[(size_t)s * PART_FLOATS + 2 + c]));
+  // partitions in ascending order; the loads of eight partitions are issued together (a dependent load per
+  // partition made this kernel 40 us for 36 MB of states)
+  for (int s0 = 0; s0 < ns; s0 += 8) {
+    float ms[8], ls[8], os[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const bool in = s0 + j < ns;
+      const float *ps = base + (size_t)(in ? s0 + j : s0) * PART_FLOATS;
+      ms[j] = in ? ps[0] : -INFINITY;
+      ls[j] = ps[1];
+      os[j] = ps[2 + c];
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (ms[j] == -INFINITY) continue;
+      const float w = ex2_approx(__fmul_rn(ms[j] - M, lam));
+      l = __fadd_rn(l, __fmul_rn(w, ls[j]));
+      o = __fadd_rn(o, __fmul_rn(w, os[j]));
+    }
   }
   const float r = (l > 0.0f) ? __fmul_rn(__fdiv_rn(o, __fmul_rn(448.0f, l)), v_scale) : 0.0f;
   const size_t idx = ((size_t)b * H_q + hq) * HEAD_DIM + c;
