@@ -222,9 +222,13 @@ mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tens
  * blocks counted from key 0, visited last to first); lambda uses q_gscale[b] * k_gscale[b].
  * Delta_S is applied when the cache has a delta_s pool.  A page-table entry outside
  * [0, num_pages) raises MPFA_DEV_BAD_PAGE in *device_status (output of that request undefined,
- * no out-of-pool access).  out_bf16 [B, N_q, H_q, 128]; out_f32 optional. */
+ * no out-of-pool access).  q_lens (device, may be NULL): per-request number of queries, 0 <= q_lens[b] <= N_q
+ * (a batch of chunks of different lengths): request b's queries are rows 0 .. q_lens[b]-1 of its slab of q and
+ * are the last q_lens[b] tokens of its context; the outputs of the remaining rows are zero.
+ * out_bf16 [B, N_q, H_q, 128]; out_f32 optional. */
 mpfa_status mpfa_prefill_paged(const mpfa_fp4_tensor *h_q, const mpfa_paged_kv *h_kv, const int32_t *page_table,
-                               int max_pages_per_req, const int32_t *seq_lens, const mpfa_stats *h_stats,
+                               int max_pages_per_req, const int32_t *seq_lens, const int32_t *q_lens,
+                               const mpfa_stats *h_stats,
                                float v_scale, float softmax_scale, void *out_bf16, float *out_f32,
                                int32_t *device_status, void *stream);
 

@@ -95,7 +95,7 @@ def lib() -> ctypes.CDLL:
         L.mpfa_prefill_variant.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_Fp4), vp, vp, ctypes.POINTER(_Stats), f, i,
                                            f, i, vp, vp, vp, vp]
         L.mpfa_prefill_paged.restype = i
-        L.mpfa_prefill_paged.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_PagedKV), vp, i, vp,
+        L.mpfa_prefill_paged.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_PagedKV), vp, i, vp, vp,
                                          ctypes.POINTER(_Stats), f, f, vp, vp, vp, vp]
         _lib = L
     return _lib
@@ -302,12 +302,13 @@ def mpfa_decode(q: Fp4Tensor, kv: PagedKV, page_table: torch.Tensor, seq_lens: t
 
 def mpfa_prefill_paged(q: Fp4Tensor, kv: PagedKV, page_table: torch.Tensor, seq_lens: torch.Tensor, stats: Stats,
                        v_scale: float, softmax_scale: float, out: torch.Tensor, out_f32: Optional[torch.Tensor],
-                       device_status: torch.Tensor) -> None:
+                       device_status: torch.Tensor, q_lens: Optional[torch.Tensor] = None) -> None:
     assert page_table.dtype == torch.int32 and page_table.is_contiguous() and seq_lens.dtype == torch.int32
+    assert q_lens is None or q_lens.dtype == torch.int32
     sc, qc, kc = stats.c(), q.c(), kv.c()
     rc = lib().mpfa_prefill_paged(ctypes.byref(qc), ctypes.byref(kc), _ptr(page_table), page_table.shape[1],
-                                  _ptr(seq_lens), ctypes.byref(sc), v_scale, softmax_scale, _ptr(out), _ptr(out_f32),
-                                  _ptr(device_status), _stream())
+                                  _ptr(seq_lens), _ptr(q_lens), ctypes.byref(sc), v_scale, softmax_scale, _ptr(out),
+                                  _ptr(out_f32), _ptr(device_status), _stream())
     _check(rc, "mpfa_prefill_paged")
 
 

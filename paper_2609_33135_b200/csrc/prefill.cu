@@ -50,8 +50,8 @@ constexpr int NTHREADS = 512;
 // setmaxnreg only moves registers inside the pool the CTA got at launch (512 threads x the 128 registers of the
 // launch bound); a request beyond the pool would block forever, so the split is checked here.
 #ifndef MPFA_REGS_UTIL_PAGED
-#define MPFA_REGS_UTIL_PAGED 88
-#define MPFA_REGS_CORR_PAGED 88
+#define MPFA_REGS_UTIL_PAGED 96
+#define MPFA_REGS_CORR_PAGED 80
 #endif
 constexpr int REGS_SOFTMAX = 168;
 // measured: the contiguous kernel gains 4 % when the correction warps' epilogue (two accumulator chunks in
@@ -129,7 +129,8 @@ struct PagedSrc {
   const uint8_t *k_codes, *k_sf, *v_fp8;
   const __nv_bfloat16 *delta;   // may be null
   const int32_t *page_table;    // [B, max_pages]
-  const int32_t *seq_lens;      // [B] keys of each request (the last N_q of them are the queries' own)
+  const int32_t *seq_lens;      // [B] keys of each request (the last q_lens[b] of them are the queries' own)
+  const int32_t *q_lens;        // [B] queries of each request, <= N_q; null: N_q for all
   int max_pages, num_pages;
 };
 
@@ -257,7 +258,7 @@ struct PageLookup {
 // One work item: a 128-row query tile of one q head.
 struct Tile {
   int b, hq, hk, qt, row0, T;   // T: KV blocks to visit
-  int nkv;                      // keys of this item's request
+  int nkv, nq;                  // keys and queries of this item's request
 };
 
 // The list of work items of this CTA.  Items are ordered by length (latest query tile first; all heads of a
@@ -280,11 +281,13 @@ struct TileWalk {
     t.hq = h % pp.H_q;
     t.hk = t.hq / (pp.H_q / pp.H_kv);
     t.row0 = t.qt * TILE;
-    const int last_row = min(pp.N_q - 1, t.row0 + TILE - 1);
+    const int n_q = (PAGED && pg.q_lens) ? min(pg.q_lens[t.b], pp.N_q) : pp.N_q;
+    const int last_row = min(n_q - 1, t.row0 + TILE - 1);
     const int n_kv = PAGED ? pg.seq_lens[t.b] : pp.N_kv;
     t.nkv = n_kv;
-    const int last_key = pp.causal ? min(n_kv - 1, last_row + (n_kv - pp.N_q)) : n_kv - 1;   // bottom-right aligned
-    t.T = last_key < 0 ? 0 : last_key / TILE + 1;
+    t.nq = n_q;
+    const int last_key = pp.causal ? min(n_kv - 1, last_row + (n_kv - n_q)) : n_kv - 1;   // bottom-right aligned
+    t.T = (last_key < 0 || (PAGED && t.row0 >= n_q)) ? 0 : last_key / TILE + 1;
     return true;
   }
 };
@@ -598,7 +601,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int T = tl.T;
       const int r_abs = tl.row0 + row;
       const int n_kv = PAGED ? tl.nkv : p.N_kv;
-      const int limit = p.causal ? min(n_kv - 1, r_abs + (n_kv - p.N_q)) : n_kv - 1;   // last visible key
+      const int n_q = PAGED ? tl.nq : p.N_q;
+      const int limit = (PAGED && r_abs >= n_q) ? -1   // a row past the request's own query count sees nothing
+                        : p.causal ? min(n_kv - 1, r_abs + (n_kv - n_q)) : n_kv - 1;   // last visible key
       const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), gq[tl.b]), gk[tl.b]);
       float m_own = -INFINITY;   // running maximum after this group's previous block
       float l_own = 0.0f;        // sum of 448 P over this group's blocks, relative to m_own
@@ -1023,7 +1028,8 @@ extern "C" mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *q, const mpfa
 }
 
 extern "C" mpfa_status mpfa_prefill_paged(const mpfa_fp4_tensor *q, const mpfa_paged_kv *kv, const int32_t *page_table,
-                                          int max_pages_per_req, const int32_t *seq_lens, const mpfa_stats *st,
+                                          int max_pages_per_req, const int32_t *seq_lens, const int32_t *q_lens,
+                                          const mpfa_stats *st,
                                           float v_scale, float softmax_scale, void *out_bf16, float *out_f32,
                                           int32_t *device_status, void *stream) {
   if (!q || !kv || !page_table || !seq_lens || !st || !out_bf16 || !device_status) return MPFA_ERR_INVALID_ARG;
@@ -1074,6 +1080,7 @@ extern "C" mpfa_status mpfa_prefill_paged(const mpfa_fp4_tensor *q, const mpfa_p
   pg.delta = static_cast<const __nv_bfloat16 *>(kv->delta_s_bf16);
   pg.page_table = page_table;
   pg.seq_lens = seq_lens;
+  pg.q_lens = q_lens;
   pg.max_pages = max_pages_per_req;
   pg.num_pages = kv->num_pages;
   int dev = 0, n_sm = 0;

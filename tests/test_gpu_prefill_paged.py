@@ -148,3 +148,36 @@ def test_paged_prefill_more_queries_than_keys():
         rows = orc.all_rows(1, H_q, N_q)
         ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
         compare(o16n[b:b + 1], o32n[b:b + 1], rows, ref32, f"request {b}")
+
+
+def test_paged_prefill_batch_of_chunks_of_different_lengths():
+    """Requests with different numbers of new queries in one launch (q_lens): request b's queries are the first
+    q_lens[b] rows of its slab and the last q_lens[b] tokens of its context; rows past that come out as zeros.
+    Includes a request with no query at all and one whose count ends inside a query tile."""
+    from paper_2609_33135_b200 import binding as B_, decode_cache
+    H_q, H_kv, N_q = 8, 2, 150
+    L, QL = [391, 200, 700, 90], [150, 37, 129, 0]
+    B = len(L)
+    w = wl.decode_workload("pp_varlen", 351, B, H_q, H_kv, 1, max(L), seq_lens=L)
+    st = decode_cache.build_cache(w)   # whole contexts in the cache; statistics frozen from them
+    q_all = w.q_sample[:, 200:200 + N_q].contiguous()
+    q4 = B_.Fp4Tensor.empty(B, H_q, N_q, "cuda")
+    B_.mpfa_quantize_qk(q_all.cuda(), None, B_.MPFA_SMOOTH | B_.MPFA_STATS_FROZEN, st.stats, q4, None, None, None)
+    out = torch.full((B, N_q, H_q, 128), 5.0, dtype=torch.bfloat16, device="cuda")
+    o32 = torch.full((B, N_q, H_q, 128), 5.0, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B_.mpfa_prefill_paged(q4, st.kv, st.page_table, st.seq_lens, st.stats, 1.0, w.softmax_scale, out, o32, status,
+                          q_lens=torch.tensor(QL, dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o16n, o32n = out.view(torch.uint16).cpu().numpy(), o32.cpu().numpy()
+    for b in range(B):
+        assert not o32n[b, QL[b]:].any() and not o16n[b, QL[b]:].any(), b
+        if QL[b] == 0:
+            continue
+        k, v = w.kv_for_request(b)
+        z0 = orc.stage1(orc.bf16_bits(w.q_sample[b:b + 1].contiguous()), orc.bf16_bits(k), orc.bf16_bits(v))
+        z = orc.stage1(orc.bf16_bits(q_all[b:b + 1, :QL[b]].contiguous()), orc.bf16_bits(k), orc.bf16_bits(v), frozen=z0)
+        rows = orc.all_rows(1, H_q, QL[b])
+        ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
+        compare(o16n[b:b + 1], o32n[b:b + 1], rows, ref32, f"request {b}")

@@ -63,7 +63,7 @@ def test_argument_errors_without_gpu(built):
     assert L.mpfa_prefill(None, None, None, None, None, 1.0, 0, 1.0, None, None, None, None) == -1
     assert L.mpfa_prefill_variant(None, None, None, None, None, 1.0, 0, 1.0, 0, None, None, None, None) == -1
     assert L.mpfa_prefill_variant(None, None, None, None, None, 1.0, 0, 1.0, 5, None, None, None, None) == -1
-    assert L.mpfa_prefill_paged(None, None, None, 1, None, None, 1.0, 1.0, None, None, None, None) == -1
+    assert L.mpfa_prefill_paged(None, None, None, 1, None, None, None, 1.0, 1.0, None, None, None, None) == -1
     assert L.mpfa_decode(None, None, None, 1, None, None, 1.0, 1.0, None, None, None, 0, None, None) == -1
     assert L.mpfa_quantize_kv_paged(None, None, 1, 0, 1, 1, 0, None, 1.0, None, None, None, 0, None) == -1
 
@@ -77,7 +77,7 @@ def test_paged_entry_points_validate_shapes_before_any_cuda_call(built):
     st = binding._Stats(a, a, a, a)
     q = binding._Fp4(a, a, 1, 8, 100)
     kv = binding._PagedKV(a, a, a, a, 4, 64, 8, 2)
-    args = (ctypes.byref(q), ctypes.byref(kv), ctypes.c_void_p(a), 4, ctypes.c_void_p(a), ctypes.byref(st), 1.0, 0.088,
+    args = (ctypes.byref(q), ctypes.byref(kv), ctypes.c_void_p(a), 4, ctypes.c_void_p(a), None, ctypes.byref(st), 1.0, 0.088,
             ctypes.c_void_p(a), None, ctypes.c_void_p(a), None)
     kv_bad_page = binding._PagedKV(a, a, a, a, 4, 32, 8, 2)
     assert L.mpfa_prefill_paged(args[0], ctypes.byref(kv_bad_page), *args[2:]) == -2          # page_size != 64
@@ -87,5 +87,5 @@ def test_paged_entry_points_validate_shapes_before_any_cuda_call(built):
     assert L.mpfa_prefill_paged(args[0], ctypes.byref(kv_bad_group), *args[2:]) == -2         # H_q % H_kv != 0
     kv_unaligned = binding._PagedKV(a + 8, a, a, a, 4, 64, 8, 2)
     assert L.mpfa_prefill_paged(args[0], ctypes.byref(kv_unaligned), *args[2:]) == -3         # pool not 256-byte aligned
-    assert L.mpfa_prefill_paged(*args[:6], 0.0, *args[7:]) == -1                               # v_scale must be positive
+    assert L.mpfa_prefill_paged(*args[:7], 0.0, *args[8:]) == -1                               # v_scale must be positive
     assert L.mpfa_prefill_paged(*args[:3], 0, *args[4:]) == -1                                 # max_pages_per_req
