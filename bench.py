@@ -33,7 +33,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 METRIC = "QK4PV8 prefill TFLOPS @16K-128K; decode KV GB/s vs HBM peak"
-KERNELS_PER_STEP = 11  # column statistics, mean+amax, scale (x2 tensors), fp4 quantize x2, Delta_S, V quantize, prefill
+KERNELS_PER_STEP = 7  # column statistics, mean+amax, scale, fp4 quantize (each one launch for Q and K), Delta_S, V quantize, prefill
 # Nominal dense tensor rates relative to BF16: FP4 4x, FP8 2x.  Per (query, key) pair the path does
 # 2d FP4 FLOP and 2d FP8 FLOP, so F attention FLOPs take (F/2)/(4P) + (F/2)/(2P) = 3F/(8P): the
 # mixed-precision bound in attention FLOP/s is 8/3 of the BF16 peak P.

@@ -11,6 +11,7 @@
 #include <cuda_fp4.h>
 #include <cuda_fp8.h>
 
+#include <algorithm>
 #include <mutex>
 
 #include "common.cuh"
@@ -59,14 +60,24 @@ __device__ __forceinline__ float from_ordered_key(unsigned int k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
-__global__ void __launch_bounds__(256) colstat_kernel(const __nv_bfloat16 *__restrict__ x, int N, int cols,
-                                                      double *__restrict__ sums, unsigned int *__restrict__ kmax,
-                                                      unsigned int *__restrict__ knegmax) {
+// One launch covers up to two tensors (Q and K): blockIdx.y runs over the 256-column groups of the first, then
+// of the second; blocks past a tensor's last token tile leave at once.
+struct ColTensor {
+  const __nv_bfloat16 *x;   // null: tensor absent (ygroups = 0)
+  int N, cols, ygroups;
+  double *sums;
+  unsigned int *kmax, *knegmax;
+};
+
+__device__ __forceinline__ void colstat_body(const __nv_bfloat16 *__restrict__ x, const int N, const int cols,
+                                             double *__restrict__ sums, unsigned int *__restrict__ kmax,
+                                             unsigned int *__restrict__ knegmax, const int yg) {
   __shared__ double s_sum[8][COLSTAT_COLS];
   __shared__ float s_max[8][COLSTAT_COLS], s_neg[8][COLSTAT_COLS];
+  if ((int)blockIdx.x * COLSTAT_TOKENS >= N) return;
   const int b = blockIdx.z;
   const int tl = threadIdx.x >> 5, cg = threadIdx.x & 31;
-  const int col = blockIdx.y * COLSTAT_COLS + cg * 8;
+  const int col = yg * COLSTAT_COLS + cg * 8;
   const int t0 = blockIdx.x * COLSTAT_TOKENS;
   const int t1 = min(N, t0 + COLSTAT_TOKENS);
   double acc[8];
@@ -99,7 +110,7 @@ __global__ void __launch_bounds__(256) colstat_kernel(const __nv_bfloat16 *__res
 #pragma unroll
   for (int i = 0; i < 8; ++i) s_sum[tl][cg * 8 + i] = acc[i], s_max[tl][cg * 8 + i] = mx[i], s_neg[tl][cg * 8 + i] = ng[i];
   __syncthreads();
-  const int c = blockIdx.y * COLSTAT_COLS + threadIdx.x;
+  const int c = yg * COLSTAT_COLS + threadIdx.x;
   if (c < cols) {
     double a = 0.0;
     float m = -INFINITY, g = -INFINITY;
@@ -112,13 +123,35 @@ __global__ void __launch_bounds__(256) colstat_kernel(const __nv_bfloat16 *__res
   }
 }
 
+__global__ void __launch_bounds__(256) colstat_kernel(const ColTensor a0, const ColTensor a1) {
+  if ((int)blockIdx.y < a0.ygroups)
+    colstat_body(a0.x, a0.N, a0.cols, a0.sums, a0.kmax, a0.knegmax, (int)blockIdx.y);
+  else
+    colstat_body(a1.x, a1.N, a1.cols, a1.sums, a1.kmax, a1.knegmax, (int)blockIdx.y - a0.ygroups);
+}
+
 // Per column: mean = fl(sum / N) (0 without smoothing); per batch element: max |x - mean| from the
 // column extremes.  grid (ceil(cols / 256), B).
-__global__ void __launch_bounds__(256) finalize_stats_kernel(const double *__restrict__ sums,
-                                                             const unsigned int *__restrict__ kmax,
-                                                             const unsigned int *__restrict__ knegmax, int cols, int N,
-                                                             int smooth, float *__restrict__ mean,
-                                                             unsigned int *__restrict__ amax) {
+struct FinTensor {
+  const double *sums;   // null: tensor absent
+  const unsigned int *kmax, *knegmax;
+  int cols, N;
+  float *mean;
+  unsigned int *amax;
+  float *gscale;
+};
+
+// grid (ceil(max cols / 256), B, 2): blockIdx.z selects the tensor.
+__global__ void __launch_bounds__(256) finalize_stats_kernel(const FinTensor a0, const FinTensor a1, int smooth) {
+  const bool second = blockIdx.z != 0;
+  const double *__restrict__ sums = second ? a1.sums : a0.sums;
+  if (!sums) return;
+  const unsigned int *__restrict__ kmax = second ? a1.kmax : a0.kmax;
+  const unsigned int *__restrict__ knegmax = second ? a1.knegmax : a0.knegmax;
+  const int cols = second ? a1.cols : a0.cols, N = second ? a1.N : a0.N;
+  float *__restrict__ mean = second ? a1.mean : a0.mean;
+  unsigned int *__restrict__ amax = second ? a1.amax : a0.amax;
+  if ((int)blockIdx.x * 256 >= cols) return;
   const int b = blockIdx.y, c = blockIdx.x * 256 + threadIdx.x;
   float m = 0.0f;
   if (c < cols) {
@@ -141,11 +174,17 @@ __global__ void __launch_bounds__(256) finalize_stats_kernel(const double *__res
   }
 }
 
-__global__ void finalize_scale_kernel(const unsigned int *__restrict__ amax, int B, float *__restrict__ gscale) {
+__global__ void finalize_scale_kernel(const FinTensor a0, const FinTensor a1, int B) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < B) {
-    float a = __uint_as_float(amax[i]);
-    gscale[i] = a > 0.0f ? __fdiv_rn(a, 2688.0f) : 1.0f;
+    if (a0.sums) {
+      float a = __uint_as_float(a0.amax[i]);
+      a0.gscale[i] = a > 0.0f ? __fdiv_rn(a, 2688.0f) : 1.0f;
+    }
+    if (a1.sums) {
+      float a = __uint_as_float(a1.amax[i]);
+      a1.gscale[i] = a > 0.0f ? __fdiv_rn(a, 2688.0f) : 1.0f;
+    }
   }
 }
 
@@ -181,15 +220,22 @@ __device__ __forceinline__ void load_center16(const __nv_bfloat16 *row, const fl
   for (int i = 0; i < 8; ++i) xc[8 + i] = __fsub_rn(f[i], mu[8 + i]);
 }
 
-// grid (N_pad/128, H, B); one 128-token tile of one head per block.
-__global__ void __launch_bounds__(256) quantize_fp4_tile_kernel(const __nv_bfloat16 *__restrict__ x,
-                                                                const float *__restrict__ mean,
-                                                                const float *__restrict__ gscale, int N, int H,
-                                                                uint8_t *__restrict__ codes, uint8_t *__restrict__ sf) {
+struct QuantTensor {
+  const __nv_bfloat16 *x;   // null: tensor absent (H = 0)
+  const float *mean, *gscale;
+  int N, H, tiles;
+  uint8_t *codes, *sf;
+};
+
+__device__ __forceinline__ void quantize_tile_body(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ mean,
+                                                   const float *__restrict__ gscale, const int N, const int H,
+                                                   const int tiles, uint8_t *__restrict__ codes,
+                                                   uint8_t *__restrict__ sf, const int h) {
   __shared__ float mu[HEAD_DIM];
   __shared__ __align__(16) uint8_t sf_tile[1024];
-  const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  const int n_pad = gridDim.x * TILE;
+  const int tile = blockIdx.x, b = blockIdx.z;
+  if (tile >= tiles) return;
+  const int n_pad = tiles * TILE;
   if (threadIdx.x < HEAD_DIM) mu[threadIdx.x] = mean[((size_t)b * H + h) * HEAD_DIM + threadIdx.x];
   __syncthreads();
   const float d = gscale[b];
@@ -209,16 +255,25 @@ __global__ void __launch_bounds__(256) quantize_fp4_tile_kernel(const __nv_bfloa
     sf_tile[(g >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (g & 3)] = sc;
   }
   __syncthreads();
-  uint32_t *dst = reinterpret_cast<uint32_t *>(sf + (((size_t)b * H + h) * gridDim.x + tile) * 1024);
+  uint32_t *dst = reinterpret_cast<uint32_t *>(sf + (((size_t)b * H + h) * tiles + tile) * 1024);
   dst[threadIdx.x] = reinterpret_cast<const uint32_t *>(sf_tile)[threadIdx.x];
 }
 
-// Eq. 9, one thread per key token: Delta_S[hq][t] = qmean[hq] . (k[t] - kmean), FP64
-// accumulation with channels ascending, expressed in units of gscale_q * gscale_k and
-// rounded once to BF16.  grid (N_pad/128, H_kv, B).  dst_stride / dst_base let the same
+// grid (max tiles, H of the first + H of the second tensor, B); one 128-token tile of one head per block.
+__global__ void __launch_bounds__(256) quantize_fp4_tile_kernel(const QuantTensor a0, const QuantTensor a1) {
+  if ((int)blockIdx.y < a0.H)
+    quantize_tile_body(a0.x, a0.mean, a0.gscale, a0.N, a0.H, a0.tiles, a0.codes, a0.sf, (int)blockIdx.y);
+  else
+    quantize_tile_body(a1.x, a1.mean, a1.gscale, a1.N, a1.H, a1.tiles, a1.codes, a1.sf, (int)blockIdx.y - a0.H);
+}
+
+// Eq. 9: Delta_S[hq][t] = qmean[hq] . (k[t] - kmean), FP64 accumulation with channels ascending,
+// expressed in units of gscale_q * gscale_k and rounded once to BF16.  Two threads per key token
+// (256 threads per 128-token tile): thread (key, part) takes the heads g = part, part + 2, ... of the
+// group, each as its own sequential chain.  grid (N_pad/128, H_kv, B).  dst_stride / dst_base let the same
 // kernel write the dense [B, H_q, N_pad] vector or one page of the paged side cache.
 template <bool PAGED>
-__global__ void __launch_bounds__(128) delta_s_kernel(const __nv_bfloat16 *__restrict__ k,
+__global__ void __launch_bounds__(256) delta_s_kernel(const __nv_bfloat16 *__restrict__ k,
                                                       const float *__restrict__ q_mean,
                                                       const float *__restrict__ k_mean,
                                                       const float *__restrict__ q_gscale,
@@ -231,15 +286,16 @@ __global__ void __launch_bounds__(128) delta_s_kernel(const __nv_bfloat16 *__res
   const int tile = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int G = H_q / H_kv;
   const int n_pad = gridDim.x * TILE;
-  kmu[threadIdx.x] = k_mean[((size_t)b * H_kv + hk) * HEAD_DIM + threadIdx.x];
-  for (int g = 0; g < G; ++g) qmu[g][threadIdx.x] = (double)q_mean[((size_t)b * H_q + hk * G + g) * HEAD_DIM + threadIdx.x];
+  if (threadIdx.x < HEAD_DIM) kmu[threadIdx.x] = k_mean[((size_t)b * H_kv + hk) * HEAD_DIM + threadIdx.x];
+  for (int j = threadIdx.x; j < G * HEAD_DIM; j += 256)
+    qmu[j >> 7][j & 127] = (double)q_mean[((size_t)b * H_q + hk * G + (j >> 7)) * HEAD_DIM + (j & 127)];
   __syncthreads();
   // The tile's K rows are staged in shared memory with coalesced 16-byte loads (a row is 256 contiguous
   // bytes, rows of one head are H_kv * 256 bytes apart); each thread then walks its own row.  Row pitch
   // 272 bytes: the 16-byte reads of 8 consecutive threads fall into 8 different bank groups.
   constexpr int PITCH = 272;
   __shared__ __align__(16) uint8_t rows[TILE * PITCH];
-  for (int i = threadIdx.x; i < TILE * 16; i += 128) {
+  for (int i = threadIdx.x; i < TILE * 16; i += 256) {
     const int r = i >> 4, ch = i & 15;
     const int tt = tile * TILE + r;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -247,12 +303,13 @@ __global__ void __launch_bounds__(128) delta_s_kernel(const __nv_bfloat16 *__res
     *reinterpret_cast<uint4 *>(rows + r * PITCH + ch * 16) = v;
   }
   __syncthreads();
-  const int t = tile * TILE + threadIdx.x;
-  double acc[MAXG];
+  const int key = threadIdx.x & 127, part = threadIdx.x >> 7;
+  const int t = tile * TILE + key;
+  double acc[MAXG / 2];
 #pragma unroll
-  for (int g = 0; g < MAXG; ++g) acc[g] = 0.0;
+  for (int u = 0; u < MAXG / 2; ++u) acc[u] = 0.0;
   if (t < N) {
-    const uint8_t *row = rows + threadIdx.x * PITCH;
+    const uint8_t *row = rows + key * PITCH;
     for (int c0 = 0; c0 < HEAD_DIM; c0 += 8) {
       float f[8];
       unpack8(*reinterpret_cast<const uint4 *>(row + c0 * 2), f);
@@ -260,16 +317,17 @@ __global__ void __launch_bounds__(128) delta_s_kernel(const __nv_bfloat16 *__res
       for (int i = 0; i < 8; ++i) {
         const double kc = (double)__fsub_rn(f[i], kmu[c0 + i]);
 #pragma unroll
-        for (int g = 0; g < MAXG; ++g)
-          if (g < G) acc[g] = fma(qmu[g][c0 + i], kc, acc[g]);
+        for (int u = 0; u < MAXG / 2; ++u)
+          if (2 * u + part < G) acc[u] = fma(qmu[2 * u + part][c0 + i], kc, acc[u]);
       }
     }
   }
   const double denom = (double)q_gscale[b] * (double)k_gscale[b];
 #pragma unroll
-  for (int g = 0; g < MAXG; ++g) {
+  for (int u = 0; u < MAXG / 2; ++u) {
+    const int g = 2 * u + part;
     if (g < G) {
-      const float v = (t < N) ? __double2float_rn(__ddiv_rn(acc[g], denom)) : 0.0f;
+      const float v = (t < N) ? __double2float_rn(__ddiv_rn(acc[u], denom)) : 0.0f;
       if (PAGED) {
         if ((t >> 6) < (N + PAGE - 1) / PAGE) {   // slots past N inside the last page are zero-filled
           const int page = page_row[t >> 6];
@@ -472,17 +530,37 @@ StatsWorkspace carve(void *ws, int B, int H_q, int H_kv) {
   return w;
 }
 
-// Means and per-tensor scale of one tensor [B, N, H, 128]: one pass over the data.
-mpfa_status tensor_stats(const __nv_bfloat16 *x, int B, int N, int H, bool smooth, double *sums, unsigned int *kmax,
-                         unsigned int *knegmax, unsigned int *amax, float *mean, float *gscale, cudaStream_t st) {
-  const int cols = H * HEAD_DIM;
-  dim3 grid((N + COLSTAT_TOKENS - 1) / COLSTAT_TOKENS, (cols + COLSTAT_COLS - 1) / COLSTAT_COLS, B);
-  colstat_kernel<<<grid, 256, 0, st>>>(x, N, cols, sums, kmax, knegmax);
+// One tensor [B, N, H, 128] of a statistics pass (x == nullptr: absent).
+struct StatsJob {
+  const __nv_bfloat16 *x;
+  int N, H;
+  double *sums;
+  unsigned int *kmax, *knegmax, *amax;
+  float *mean, *gscale;
+};
+
+// Means and per-tensor scales of up to two tensors: one pass over the data, three launches in all.
+mpfa_status tensor_stats(const StatsJob &j0, const StatsJob &j1, int B, bool smooth, cudaStream_t st) {
+  ColTensor c[2];
+  FinTensor f[2];
+  int tiles = 0, colgroups = 0;
+  const StatsJob *jobs[2] = {&j0, &j1};
+  for (int i = 0; i < 2; ++i) {
+    const StatsJob &j = *jobs[i];
+    const int cols = j.H * HEAD_DIM;
+    c[i] = ColTensor{j.x, j.x ? j.N : 0, cols, j.x ? (cols + COLSTAT_COLS - 1) / COLSTAT_COLS : 0, j.sums, j.kmax, j.knegmax};
+    f[i] = FinTensor{j.x ? j.sums : nullptr, j.kmax, j.knegmax, cols, j.N, j.mean, j.amax, j.gscale};
+    if (j.x) {
+      tiles = std::max(tiles, (j.N + COLSTAT_TOKENS - 1) / COLSTAT_TOKENS);
+      colgroups = std::max(colgroups, (cols + 255) / 256);
+    }
+  }
+  if (c[0].ygroups + c[1].ygroups == 0) return MPFA_OK;
+  colstat_kernel<<<dim3(tiles, c[0].ygroups + c[1].ygroups, B), 256, 0, st>>>(c[0], c[1]);
   MPFA_LAUNCH_OK();
-  finalize_stats_kernel<<<dim3((cols + 255) / 256, B), 256, 0, st>>>(sums, kmax, knegmax, cols, N, smooth ? 1 : 0, mean,
-                                                                    amax);
+  finalize_stats_kernel<<<dim3(colgroups, B, 2), 256, 0, st>>>(f[0], f[1], smooth ? 1 : 0);
   MPFA_LAUNCH_OK();
-  finalize_scale_kernel<<<(B + 127) / 128, 128, 0, st>>>(amax, B, gscale);
+  finalize_scale_kernel<<<(B + 127) / 128, 128, 0, st>>>(f[0], f[1], B);
   MPFA_LAUNCH_OK();
   return MPFA_OK;
 }
@@ -530,26 +608,23 @@ extern "C" mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, 
   const __nv_bfloat16 *k = static_cast<const __nv_bfloat16 *>(k_bf16);
   if (!frozen) {
     MPFA_CUDA_OK(cudaMemsetAsync(workspace, 0, w.bytes, s));
-    if (q) {
-      rc = tensor_stats(q, B, N_q, H_q, smooth, w.sums_q, w.max_q, w.neg_q, w.amax_q, st->q_mean, st->q_gscale, s);
-      if (rc != MPFA_OK) return rc;
-    }
-    if (k) {
-      rc = tensor_stats(k, B, N_kv, H_kv, smooth, w.sums_k, w.max_k, w.neg_k, w.amax_k, st->k_mean, st->k_gscale, s);
-      if (rc != MPFA_OK) return rc;
-    }
+    rc = tensor_stats(StatsJob{q, N_q, H_q, w.sums_q, w.max_q, w.neg_q, w.amax_q, st->q_mean, st->q_gscale},
+                      StatsJob{k, N_kv, H_kv, w.sums_k, w.max_k, w.neg_k, w.amax_k, st->k_mean, st->k_gscale}, B, smooth, s);
+    if (rc != MPFA_OK) return rc;
   }
-  if (q) {
-    dim3 grid(pad128(N_q) / TILE, H_q, B);
-    quantize_fp4_tile_kernel<<<grid, 256, 0, s>>>(q, st->q_mean, st->q_gscale, N_q, H_q, q_out->codes, q_out->sf);
+  {
+    // Q and K tiles in one launch
+    QuantTensor tq{q, st->q_mean, st->q_gscale, N_q, q ? H_q : 0, q ? pad128(N_q) / TILE : 0, q ? q_out->codes : nullptr,
+                   q ? q_out->sf : nullptr};
+    QuantTensor tk{k, st->k_mean, st->k_gscale, N_kv, k ? H_kv : 0, k ? pad128(N_kv) / TILE : 0,
+                   k ? k_out->codes : nullptr, k ? k_out->sf : nullptr};
+    quantize_fp4_tile_kernel<<<dim3(std::max(tq.tiles, tk.tiles), tq.H + tk.H, B), 256, 0, s>>>(tq, tk);
     MPFA_LAUNCH_OK();
   }
   if (k) {
     dim3 grid(pad128(N_kv) / TILE, H_kv, B);
-    quantize_fp4_tile_kernel<<<grid, 256, 0, s>>>(k, st->k_mean, st->k_gscale, N_kv, H_kv, k_out->codes, k_out->sf);
-    MPFA_LAUNCH_OK();
     if (smooth) {
-      delta_s_kernel<false><<<grid, 128, 0, s>>>(k, st->q_mean, st->k_mean, st->q_gscale, st->k_gscale, N_kv, H_q,
+      delta_s_kernel<false><<<grid, 256, 0, s>>>(k, st->q_mean, st->k_mean, st->q_gscale, st->k_gscale, N_kv, H_q,
                                                  H_kv, static_cast<__nv_bfloat16 *>(delta_s_bf16), nullptr, 0);
       MPFA_LAUNCH_OK();
     }
@@ -601,7 +676,8 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
   const __nv_bfloat16 *v = static_cast<const __nv_bfloat16 *>(v_bf16);
   if (!frozen) {
     MPFA_CUDA_OK(cudaMemsetAsync(workspace, 0, w.bytes, s));
-    rc = tensor_stats(k, 1, N_tokens, H_kv, smooth, w.sums_k, w.max_k, w.neg_k, w.amax_k, st->k_mean, st->k_gscale, s);
+    rc = tensor_stats(StatsJob{k, N_tokens, H_kv, w.sums_k, w.max_k, w.neg_k, w.amax_k, st->k_mean, st->k_gscale},
+                      StatsJob{nullptr, 0, 0, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr}, 1, smooth, s);
     if (rc != MPFA_OK) return rc;
   }
   if (first_token % PAGE != 0) {
@@ -621,7 +697,7 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
                                                               kv->num_pages, kv->k_codes, kv->k_sf, kv->v_fp8);
   MPFA_LAUNCH_OK();
   if (smooth) {
-    delta_s_kernel<true><<<dim3(pad128(N_tokens) / TILE, H_kv, 1), 128, 0, s>>>(
+    delta_s_kernel<true><<<dim3(pad128(N_tokens) / TILE, H_kv, 1), 256, 0, s>>>(
         k, st->q_mean, st->k_mean, st->q_gscale, st->k_gscale, N_tokens, H_q, H_kv,
         static_cast<__nv_bfloat16 *>(kv->delta_s_bf16), page_table_row + first_token / PAGE, kv->num_pages);
     MPFA_LAUNCH_OK();
