@@ -251,3 +251,44 @@ def test_decode_with_empty_contexts_in_the_batch():
     for b in (1, 3):
         d = np.abs(got[b] - oracle_decode_one(w, b))
         assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (b, float(d.max()), float(d.mean()))
+
+
+def test_decode_loop_append_one_token_then_attend():
+    """The decode configuration sustained over several steps (Section 6): every step appends one new token per
+    request to its pages with the frozen statistics, raises the request's length and decodes; each step's output is
+    compared with the oracle's decode over the same prefix."""
+    from paper_2609_33135_b200 import binding as B_, decode_cache
+    L0, steps = [127, 64, 1000], 5
+    L1 = [l + steps for l in L0]
+    w_full = wl.decode_workload("dec_loop", 93, 3, 8, 2, 1, max(L1), seq_lens=L1)
+    w0 = wl.decode_workload("dec_loop", 93, 3, 8, 2, 1, max(L1), seq_lens=L0)
+    w0.page_table, w0.num_pages = w_full.page_table, w_full.num_pages
+    kv_full = [w_full.kv_for_request(b) for b in range(3)]
+    w0.kv_for_request = lambda b, device="cpu": (kv_full[b][0][:, :L0[b]].contiguous(), kv_full[b][1][:, :L0[b]].contiguous())
+    st = decode_cache.build_cache(w0)
+    st.w = w_full
+    flags = B_.MPFA_SMOOTH | B_.MPFA_STATS_FROZEN
+    z0 = [orc.stage1(orc.bf16_bits(w_full.q_sample[b:b + 1].contiguous()), orc.bf16_bits(kv_full[b][0][:, :L0[b]].contiguous()),
+                     orc.bf16_bits(kv_full[b][1][:, :L0[b]].contiguous())) for b in range(3)]
+    kd = [(kv_full[b][0][0].cuda(), kv_full[b][1][0].cuda()) for b in range(3)]
+    for s in range(steps):
+        for b in range(3):
+            pos = L0[b] + s
+            B_.mpfa_quantize_kv_paged(kd[b][0][pos:pos + 1].contiguous(), kd[b][1][pos:pos + 1].contiguous(), pos, w_full.H_q,
+                                      flags, st.stats.request(b), 1.0, st.kv, st.page_table[b], None)
+        lens = torch.tensor([l + s + 1 for l in L0], dtype=torch.int32)
+        st.seq_lens.copy_(lens.to(st.seq_lens.device))
+        q_step = w_full.q_sample[:, 10 + s:11 + s].contiguous()
+        B_.mpfa_quantize_qk(q_step.cuda(), None, flags, st.stats, st.q4, None, None, None)
+        decode_cache.decode_step(st)
+        torch.cuda.synchronize()
+        assert int(st.status.item()) == 0
+        got = st.out_f32.cpu().numpy()
+        for b in range(3):
+            n = int(lens[b])
+            kb, vb = kv_full[b][0][:, :n].contiguous(), kv_full[b][1][:, :n].contiguous()
+            z = orc.stage1(orc.bf16_bits(q_step[b:b + 1].contiguous()), orc.bf16_bits(kb), orc.bf16_bits(vb), frozen=z0[b])
+            ref, _ = orc.decode(z.q_codes[:, :, 0], z.q_sf[:, :, 0], z.k_codes, z.k_sf, z.v_codes, z.delta, z.dq, z.dk, 1.0,
+                                w_full.softmax_scale, np.array([n], np.int32))
+            d = np.abs(got[b] - ref[0])
+            assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (s, b, float(d.max()), float(d.mean()))
