@@ -182,6 +182,19 @@ mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_bf16, int N
                                    const mpfa_paged_kv *h_kv, const int32_t *page_table_row,
                                    void *workspace, size_t workspace_bytes, void *stream);
 
+/* Decode-time append for a whole batch in one launch (Section 6): request b gets ONE new token,
+ * k_bf16 / v_bf16 [B, 1, H_kv, 128], written at token index positions[b] (device int32 [B]; normally the
+ * request's length before the call; negative: the request is skipped) of the pages page_table[b, :]
+ * ([B, max_pages_per_req], device).  The token is centered with the request's frozen k_mean, quantized with
+ * its frozen k_gscale (stats holds [B, ...] arrays and is only read), V with v_scale, and with MPFA_SMOOTH its
+ * Delta_S entries are written for the H_q / H_kv heads of each group.  A token that starts a page zeroes the
+ * other 63 slots of that page.  Same bytes as B calls of mpfa_quantize_kv_paged with N_tokens = 1 and
+ * MPFA_STATS_FROZEN.  A position without a page-table entry or a page id outside the pool is skipped. */
+mpfa_status mpfa_append_kv_paged(const void *k_bf16, const void *v_bf16, int B, int H_q, int H_kv, int flags,
+                                 const mpfa_stats *h_stats, float v_scale, const mpfa_paged_kv *h_kv,
+                                 const int32_t *page_table, int max_pages_per_req, const int32_t *positions,
+                                 void *stream);
+
 /* ---- stage 2: Algorithm 1 lines 6-20 -------------------------------------------------- */
 
 /* QK4PV8 prefill.  q: [B, H_q, N_q] tile-layout tensor, k: [B, H_kv, N_kv], v_fp8 and

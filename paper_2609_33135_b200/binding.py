@@ -85,6 +85,9 @@ def lib() -> ctypes.CDLL:
         L.mpfa_quantize_kv_paged.restype = i
         L.mpfa_quantize_kv_paged.argtypes = [vp, vp, i, i, i, i, i, ctypes.POINTER(_Stats), f,
                                              ctypes.POINTER(_PagedKV), vp, vp, sz, vp]
+        L.mpfa_append_kv_paged.restype = i
+        L.mpfa_append_kv_paged.argtypes = [vp, vp, i, i, i, i, ctypes.POINTER(_Stats), f, ctypes.POINTER(_PagedKV), vp, i,
+                                           vp, vp]
         L.mpfa_prefill.restype = i
         L.mpfa_prefill.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_Fp4), vp, vp, ctypes.POINTER(_Stats), f, i,
                                    f, vp, vp, vp, vp]
@@ -263,6 +266,19 @@ def mpfa_quantize_kv_paged(k: torch.Tensor, v: torch.Tensor, first_token: int, H
                                       ctypes.byref(kc), _ptr(page_table_row), _ptr(workspace),
                                       0 if workspace is None else workspace.numel(), _stream())
     _check(rc, "mpfa_quantize_kv_paged")
+
+
+def mpfa_append_kv_paged(k: torch.Tensor, v: torch.Tensor, H_q: int, flags: int, stats: Stats, v_scale: float,
+                         kv: PagedKV, page_table: torch.Tensor, positions: torch.Tensor) -> None:
+    """k, v: [B, 1, H_kv, 128] bf16; one new token per request at positions[b]."""
+    assert k.dtype == torch.bfloat16 and k.is_contiguous() and v.is_contiguous() and k.shape == v.shape
+    assert page_table.dtype == torch.int32 and page_table.is_contiguous() and positions.dtype == torch.int32
+    B, one, H_kv, _ = k.shape
+    assert one == 1
+    sc, kc = stats.c(), kv.c()
+    rc = lib().mpfa_append_kv_paged(_ptr(k), _ptr(v), B, H_q, H_kv, flags, ctypes.byref(sc), v_scale, ctypes.byref(kc),
+                                    _ptr(page_table), page_table.shape[1], _ptr(positions), _stream())
+    _check(rc, "mpfa_append_kv_paged")
 
 
 def mpfa_prefill(q: Fp4Tensor, k: Fp4Tensor, v_fp8: torch.Tensor, delta: Optional[torch.Tensor], stats: Stats,

@@ -447,11 +447,28 @@ __global__ void __launch_bounds__(256) append_kv_kernel(const __nv_bfloat16 *__r
                                                         int H_q, int H_kv, float inv_vscale, int smooth,
                                                         const int32_t *__restrict__ page_row, int num_pages,
                                                         uint8_t *__restrict__ k_codes, uint8_t *__restrict__ k_sf,
-                                                        uint8_t *__restrict__ v_fp8, __nv_bfloat16 *__restrict__ delta) {
+                                                        uint8_t *__restrict__ v_fp8, __nv_bfloat16 *__restrict__ delta,
+                                                        const int32_t *__restrict__ positions, int max_pages) {
   constexpr int MAXG = 8;
   __shared__ float kmu[HEAD_DIM];
   __shared__ double qmu[MAXG][HEAD_DIM];
   __shared__ float kc[32][HEAD_DIM + 4];   // centered K rows of the block's tokens (for Delta_S)
+  if (positions) {
+    // batch form: request blockIdx.z appends the one token k[b] / v[b] at index positions[b] with its own
+    // statistics and page-table row; a negative position skips the request
+    const int b = blockIdx.z;
+    first_token = positions[b];
+    if (first_token < 0) return;
+    N = 1;
+    k += (size_t)b * H_kv * HEAD_DIM;
+    v += (size_t)b * H_kv * HEAD_DIM;
+    q_mean += (size_t)b * H_q * HEAD_DIM;
+    k_mean += (size_t)b * H_kv * HEAD_DIM;
+    q_gscale += b;
+    k_gscale += b;
+    page_row += (size_t)b * max_pages;
+    if ((first_token >> 6) >= max_pages) return;   // no page-table entry for that position
+  }
   const int h = blockIdx.y, G = H_q / H_kv;
   const int slot = threadIdx.x >> 3, g = threadIdx.x & 7;
   const int i = blockIdx.x * 32 + slot;          // index among the slots this call covers
@@ -687,7 +704,7 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
     append_kv_kernel<<<dim3((n_slots + 31) / 32, H_kv), 256, 0, s>>>(
         k, v, st->q_mean, st->k_mean, st->q_gscale, st->k_gscale, N_tokens, first_token, H_q, H_kv, 1.0f / v_scale,
         smooth ? 1 : 0, page_table_row, kv->num_pages, kv->k_codes, kv->k_sf, kv->v_fp8,
-        static_cast<__nv_bfloat16 *>(kv->delta_s_bf16));
+        static_cast<__nv_bfloat16 *>(kv->delta_s_bf16), nullptr, 0);
     MPFA_LAUNCH_OK();
     return MPFA_OK;
   }
@@ -706,6 +723,33 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
 }
 
 // ---------------------------------------------------------------------------------------
+extern "C" mpfa_status mpfa_append_kv_paged(const void *k_bf16, const void *v_bf16, int B, int H_q, int H_kv, int flags,
+                                            const mpfa_stats *st, float v_scale, const mpfa_paged_kv *kv,
+                                            const int32_t *page_table, int max_pages_per_req,
+                                            const int32_t *positions, void *stream) {
+  const bool smooth = flags & MPFA_SMOOTH;
+  if (!k_bf16 || !v_bf16 || !st || !kv || !page_table || !positions || B <= 0 || H_q <= 0 || H_kv <= 0 ||
+      max_pages_per_req <= 0 || !(v_scale > 0.0f))
+    return MPFA_ERR_INVALID_ARG;
+  if (!st->k_mean || !st->k_gscale || (smooth && (!st->q_mean || !st->q_gscale))) return MPFA_ERR_INVALID_ARG;
+  if (!kv->k_codes || !kv->k_sf || !kv->v_fp8 || kv->num_pages <= 0) return MPFA_ERR_INVALID_ARG;
+  if (smooth && !kv->delta_s_bf16) return MPFA_ERR_INVALID_ARG;
+  if (kv->page_size != PAGE || H_q % H_kv != 0 || H_q / H_kv > 8 || B > 65535) return MPFA_ERR_UNSUPPORTED;
+  if (kv->H_q != H_q || kv->H_kv != H_kv) return MPFA_ERR_INVALID_ARG;
+  if (!aligned(k_bf16, 16) || !aligned(v_bf16, 16) || !aligned(kv->k_codes, 256) || !aligned(kv->k_sf, 256) ||
+      !aligned(kv->v_fp8, 256) || !aligned(kv->delta_s_bf16, 256))
+    return MPFA_ERR_ALIGNMENT;
+  mpfa_status rc = check_arch();
+  if (rc != MPFA_OK) return rc;
+  // 64 slots per request: the token's own and, when it starts a page, the 63 to be zeroed after it
+  append_kv_kernel<<<dim3(2, H_kv, B), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16 *>(k_bf16), static_cast<const __nv_bfloat16 *>(v_bf16), st->q_mean, st->k_mean,
+      st->q_gscale, st->k_gscale, 1, 0, H_q, H_kv, 1.0f / v_scale, smooth ? 1 : 0, page_table, kv->num_pages,
+      kv->k_codes, kv->k_sf, kv->v_fp8, static_cast<__nv_bfloat16 *>(kv->delta_s_bf16), positions, max_pages_per_req);
+  MPFA_LAUNCH_OK();
+  return MPFA_OK;
+}
+
 // mpfa_quantize_qk_static: the same stage-1 call for callers that cannot provide scratch.
 // ---------------------------------------------------------------------------------------
 namespace mpfa {

@@ -272,10 +272,16 @@ def test_decode_loop_append_one_token_then_attend():
                      orc.bf16_bits(kv_full[b][1][:, :L0[b]].contiguous())) for b in range(3)]
     kd = [(kv_full[b][0][0].cuda(), kv_full[b][1][0].cuda()) for b in range(3)]
     for s in range(steps):
-        for b in range(3):
-            pos = L0[b] + s
-            B_.mpfa_quantize_kv_paged(kd[b][0][pos:pos + 1].contiguous(), kd[b][1][pos:pos + 1].contiguous(), pos, w_full.H_q,
-                                      flags, st.stats.request(b), 1.0, st.kv, st.page_table[b], None)
+        if s % 2 == 0:   # the whole batch in one launch
+            k_new = torch.stack([kd[b][0][L0[b] + s:L0[b] + s + 1] for b in range(3)]).contiguous()
+            v_new = torch.stack([kd[b][1][L0[b] + s:L0[b] + s + 1] for b in range(3)]).contiguous()
+            pos = torch.tensor([l + s for l in L0], dtype=torch.int32, device="cuda")
+            B_.mpfa_append_kv_paged(k_new, v_new, w_full.H_q, B_.MPFA_SMOOTH, st.stats, 1.0, st.kv, st.page_table, pos)
+        else:            # request by request
+            for b in range(3):
+                pos = L0[b] + s
+                B_.mpfa_quantize_kv_paged(kd[b][0][pos:pos + 1].contiguous(), kd[b][1][pos:pos + 1].contiguous(), pos,
+                                          w_full.H_q, flags, st.stats.request(b), 1.0, st.kv, st.page_table[b], None)
         lens = torch.tensor([l + s + 1 for l in L0], dtype=torch.int32)
         st.seq_lens.copy_(lens.to(st.seq_lens.device))
         q_step = w_full.q_sample[:, 10 + s:11 + s].contiguous()
@@ -292,3 +298,43 @@ def test_decode_loop_append_one_token_then_attend():
                                 w_full.softmax_scale, np.array([n], np.int32))
             d = np.abs(got[b] - ref[0])
             assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (s, b, float(d.max()), float(d.mean()))
+
+
+def test_batched_append_writes_the_same_bytes_as_per_request_appends():
+    """mpfa_append_kv_paged against mpfa_quantize_kv_paged with one token: every pool byte equal, over positions that
+    start a page (the rest of the page is zeroed), end a page, and with one request skipped (negative position)."""
+    from paper_2609_33135_b200 import binding as B_, decode_cache
+    L0 = [64, 63, 200, 5]          # request 0 starts a new page, request 1 fills the last slot of its page
+    w_full = wl.decode_workload("dec_batch_append", 94, 4, 8, 2, 1, 300, seq_lens=[l + 3 for l in L0])
+    kv_full = [w_full.kv_for_request(b) for b in range(4)]
+    states = []
+    for mode in ("batched", "single"):
+        w0 = wl.decode_workload("dec_batch_append", 94, 4, 8, 2, 1, 300, seq_lens=L0)
+        w0.page_table, w0.num_pages = w_full.page_table, w_full.num_pages
+        w0.kv_for_request = lambda b, device="cpu": (kv_full[b][0][:, :L0[b]].contiguous(), kv_full[b][1][:, :L0[b]].contiguous())
+        st = decode_cache.build_cache(w0)
+        for t in (st.kv.k_codes, st.kv.k_sf, st.kv.v_fp8):   # stale bytes in the pages the appends will start
+            t[int(w_full.page_table[0, 1])].fill_(0x7F)
+        st.kv.delta[int(w_full.page_table[0, 1])].fill_(float("nan"))
+        for s in range(3):
+            active = [b for b in range(4) if not (b == 3 and s == 1)]   # request 3 sits out step 1
+            if mode == "batched":
+                k_new = torch.stack([kv_full[b][0][0, L0[b] + s:L0[b] + s + 1] for b in range(4)]).contiguous().cuda()
+                v_new = torch.stack([kv_full[b][1][0, L0[b] + s:L0[b] + s + 1] for b in range(4)]).contiguous().cuda()
+                pos = torch.tensor([L0[b] + s if b in active else -1 for b in range(4)], dtype=torch.int32, device="cuda")
+                B_.mpfa_append_kv_paged(k_new, v_new, w_full.H_q, B_.MPFA_SMOOTH, st.stats, 1.0, st.kv, st.page_table, pos)
+            else:
+                for b in active:
+                    p = L0[b] + s
+                    B_.mpfa_quantize_kv_paged(kv_full[b][0][0, p:p + 1].contiguous().cuda(), kv_full[b][1][0, p:p + 1].contiguous().cuda(),
+                                              p, w_full.H_q, B_.MPFA_SMOOTH | B_.MPFA_STATS_FROZEN, st.stats.request(b), 1.0,
+                                              st.kv, st.page_table[b], None)
+        torch.cuda.synchronize()
+        states.append(st)
+    a, b = states
+    used = sorted({int(p) for r in range(4) for p in w_full.page_table[r] if int(p) >= 0})
+    for name in ("k_codes", "k_sf", "v_fp8"):
+        assert torch.equal(getattr(a.kv, name)[used], getattr(b.kv, name)[used]), name
+    assert torch.equal(a.kv.delta[used].view(torch.int16), b.kv.delta[used].view(torch.int16))
+    pg = int(w_full.page_table[0, 1])
+    assert not a.kv.k_codes[pg].view(-1, 4096)[:, :].reshape(2, 8, 512)[:, 1:].any()   # slots 8.. of the started page are zero

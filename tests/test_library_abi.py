@@ -66,6 +66,7 @@ def test_argument_errors_without_gpu(built):
     assert L.mpfa_prefill_paged(None, None, None, 1, None, None, None, 1.0, 1.0, None, None, None, None) == -1
     assert L.mpfa_decode(None, None, None, 1, None, None, 1.0, 1.0, None, None, None, 0, None, None) == -1
     assert L.mpfa_quantize_kv_paged(None, None, 1, 0, 1, 1, 0, None, 1.0, None, None, None, 0, None) == -1
+    assert L.mpfa_append_kv_paged(None, None, 1, 1, 1, 0, None, 1.0, None, None, 1, None, None) == -1
 
 
 def test_paged_entry_points_validate_shapes_before_any_cuda_call(built):
