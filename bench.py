@@ -209,7 +209,22 @@ def bench_decode(steps, warmup, peaks, small):
     bytes_ = float(w.total_tokens) * w.H_kv * KV_BYTES_PER_TOKEN_HEAD
     mean = sum(ms) / len(ms)
     gbs = bytes_ / (mean * 1e-3) / 1e9
+    # the serving step: write one new token per request into the cache (frozen statistics), then decode
+    from paper_2609_33135_b200 import binding as B_
+    g = torch.Generator(device="cuda").manual_seed(1007)
+    k_new = torch.randn(w.B, 1, w.H_kv, 128, generator=g, device="cuda").to(torch.bfloat16)
+    v_new = torch.randn(w.B, 1, w.H_kv, 128, generator=g, device="cuda").to(torch.bfloat16)
+    pos = (st.seq_lens - 1).to(torch.int32)   # the slot of each request's last token (always has a page)
+    evs2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs2:
+        a.record()
+        B_.mpfa_append_kv_paged(k_new, v_new, w.H_q, B_.MPFA_SMOOTH, st.stats, st.v_scale, st.kv, st.page_table, pos)
+        decode_cache.decode_step(st)
+        b.record()
+    torch.cuda.synchronize()
+    ms_append = sum(a.elapsed_time(b) for a, b in evs2) / len(evs2)
     return {"workload": w.name, "value": gbs, "unit": "GB/s", "ms_mean": mean, "ms_min": min(ms),
+            "ms_append_plus_decode": ms_append,
             "kv_bytes": bytes_, "tokens": w.total_tokens, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
             "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "gpu_launches_per_step": 2,
             "l2": "3.9 GB of cache per step vs 126 MB L2", "status": int(st.status.item())}
