@@ -798,46 +798,69 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
 
 // Merge of the partition states (Section 5.3): M = max m_s, w_s = 2^(lam (m_s - M)),
 // l = sum w_s l_s, O = sum w_s O_s, out = O / (448 l) * v_scale.  grid (H_q, B), 128 threads.
-__global__ void __launch_bounds__(128) decode_merge_kernel(const float *__restrict__ parts,
+__global__ void __launch_bounds__(256) decode_merge_kernel(const float *__restrict__ parts,
                                                            const int32_t *__restrict__ seq_lens,
                                                            const float *__restrict__ q_gscale,
                                                            const float *__restrict__ k_gscale, int H_q, int n_split,
                                                            float softmax_scale, float v_scale,
                                                            __nv_bfloat16 *__restrict__ out, float *__restrict__ out_f32) {
-  const int hq = blockIdx.x, b = blockIdx.y, c = threadIdx.x, lane = threadIdx.x & 31;
+  // 8 warps: warp w takes the partitions s = w, w + 8, ... in ascending order (the loads of four of them in
+  // flight together), lane l the channels l, l + 32, l + 64, l + 96; the eight partial sums are then added in
+  // warp order.  A fixed order, so the result is reproducible; with one thread walking all partitions a
+  // single long request (128 partitions, 32 blocks in the grid) spent 25 us here.
+  __shared__ float s_red[8], s_l[8], s_o[8][HEAD_DIM];
+  const int hq = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int L = seq_lens[b];
   const int ns = min(n_split, (L + DECODE_SPLIT - 1) / DECODE_SPLIT);
   const float *base = parts + ((size_t)b * H_q + hq) * n_split * PART_FLOATS;
   const float lam = __fmul_rn(__fmul_rn(__fmul_rn(softmax_scale, 1.4426950408889634f), q_gscale[b]), k_gscale[b]);
   float M = -INFINITY;
-  for (int s = lane; s < ns; s += 32) M = fmaxf(M, base[(size_t)s * PART_FLOATS]);
+  for (int s = tid; s < ns; s += 256) M = fmaxf(M, base[(size_t)s * PART_FLOATS]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-  float l = 0.0f, o = 0.0f;
-  // partitions in ascending order; the loads of eight partitions are issued together (a dependent load per
-  // partition made this kernel 40 us for 36 MB of states)
-  for (int s0 = 0; s0 < ns; s0 += 8) {
-    float ms[8], ls[8], os[8];
+  if (lane == 0) s_red[warp] = M;
+  __syncthreads();
+  M = s_red[0];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const bool in = s0 + j < ns;
-      const float *ps = base + (size_t)(in ? s0 + j : s0) * PART_FLOATS;
+  for (int w = 1; w < 8; ++w) M = fmaxf(M, s_red[w]);
+  float l = 0.0f, o[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+  for (int s0 = warp; s0 < ns; s0 += 32) {
+    float ms[4], ls[4], os[4][4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int sp = s0 + 8 * j;
+      const bool in = sp < ns;
+      const float *ps = base + (size_t)(in ? sp : s0) * PART_FLOATS;
       ms[j] = in ? ps[0] : -INFINITY;
       ls[j] = ps[1];
-      os[j] = ps[2 + c];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) os[j][q] = ps[2 + lane + 32 * q];
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < 4; ++j) {
       if (ms[j] == -INFINITY) continue;
       const float w = ex2_approx(__fmul_rn(ms[j] - M, lam));
       l = __fadd_rn(l, __fmul_rn(w, ls[j]));
-      o = __fadd_rn(o, __fmul_rn(w, os[j]));
+#pragma unroll
+      for (int q = 0; q < 4; ++q) o[q] = __fadd_rn(o[q], __fmul_rn(w, os[j][q]));
     }
   }
-  const float r = (l > 0.0f) ? __fmul_rn(__fdiv_rn(o, __fmul_rn(448.0f, l)), v_scale) : 0.0f;
-  const size_t idx = ((size_t)b * H_q + hq) * HEAD_DIM + c;
-  out[idx] = __float2bfloat16_rn(r);
-  if (out_f32) out_f32[idx] = r;
+  if (lane == 0) s_l[warp] = l;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) s_o[warp][lane + 32 * q] = o[q];
+  __syncthreads();
+  if (tid < HEAD_DIM) {
+    float lt = s_l[0], ot = s_o[0][tid];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) {
+      lt = __fadd_rn(lt, s_l[w]);
+      ot = __fadd_rn(ot, s_o[w][tid]);
+    }
+    const float r = (lt > 0.0f) ? __fmul_rn(__fdiv_rn(ot, __fmul_rn(448.0f, lt)), v_scale) : 0.0f;
+    const size_t idx = ((size_t)b * H_q + hq) * HEAD_DIM + tid;
+    out[idx] = __float2bfloat16_rn(r);
+    if (out_f32) out_f32[idx] = r;
+  }
 }
 
 }  // namespace
@@ -931,7 +954,7 @@ extern "C" mpfa_status mpfa_decode(const mpfa_fp4_tensor *q, const mpfa_paged_kv
   MPFA_CUDA_OK(cudaMemsetAsync(p.ticket, 0, sizeof(unsigned int), s));   // a memory-set node, no allocation
   kern<<<grid, D_THREADS, D_SMEM, s>>>(p);
   MPFA_LAUNCH_OK();
-  decode_merge_kernel<<<dim3(H_q, B), 128, 0, s>>>(p.parts, seq_lens, st->q_gscale, st->k_gscale, H_q, (int)n_split,
+  decode_merge_kernel<<<dim3(H_q, B), 256, 0, s>>>(p.parts, seq_lens, st->q_gscale, st->k_gscale, H_q, (int)n_split,
                                                    softmax_scale, v_scale, static_cast<__nv_bfloat16 *>(out_bf16),
                                                    out_f32);
   MPFA_LAUNCH_OK();
