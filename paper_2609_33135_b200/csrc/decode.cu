@@ -797,7 +797,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
 }
 
 // Merge of the partition states (Section 5.3): M = max m_s, w_s = 2^(lam (m_s - M)),
-// l = sum w_s l_s, O = sum w_s O_s, out = O / (448 l) * v_scale.  grid (H_q, B), 128 threads.
+// l = sum w_s l_s, O = sum w_s O_s, out = O / (448 l) * v_scale.  grid (H_q, B), 256 threads.
 __global__ void __launch_bounds__(256) decode_merge_kernel(const float *__restrict__ parts,
                                                            const int32_t *__restrict__ seq_lens,
                                                            const float *__restrict__ q_gscale,
