@@ -338,3 +338,59 @@ def test_batched_append_writes_the_same_bytes_as_per_request_appends():
     assert torch.equal(a.kv.delta[used].view(torch.int16), b.kv.delta[used].view(torch.int16))
     pg = int(w_full.page_table[0, 1])
     assert not a.kv.k_codes[pg].view(-1, 4096)[:, :].reshape(2, 8, 512)[:, 1:].any()   # slots 8.. of the started page are zero
+
+
+def test_serving_step_captured_once_and_replayed():
+    """The whole decode-time step - write the batch's new K/V token into the pages, quantize the new query with the
+    frozen statistics, attend - captured in one CUDA graph and replayed: positions, inputs and lengths change in
+    place between replays; every replay is compared with the oracle."""
+    from paper_2609_33135_b200 import binding as B_, decode_cache
+    L0, steps = [190, 63, 2047], 4
+    L1 = [l + steps for l in L0]
+    w_full = wl.decode_workload("dec_graph_step", 95, 3, 8, 2, 1, max(L1), seq_lens=L1)
+    w0 = wl.decode_workload("dec_graph_step", 95, 3, 8, 2, 1, max(L1), seq_lens=L0)
+    w0.page_table, w0.num_pages = w_full.page_table, w_full.num_pages
+    kv_full = [w_full.kv_for_request(b) for b in range(3)]
+    w0.kv_for_request = lambda b, device="cpu": (kv_full[b][0][:, :L0[b]].contiguous(), kv_full[b][1][:, :L0[b]].contiguous())
+    st = decode_cache.build_cache(w0)
+    flags = B_.MPFA_SMOOTH | B_.MPFA_STATS_FROZEN
+    z0 = [orc.stage1(orc.bf16_bits(w_full.q_sample[b:b + 1].contiguous()), orc.bf16_bits(kv_full[b][0][:, :L0[b]].contiguous()),
+                     orc.bf16_bits(kv_full[b][1][:, :L0[b]].contiguous())) for b in range(3)]
+    k_new = torch.empty(3, 1, 2, 128, dtype=torch.bfloat16, device="cuda")
+    v_new = torch.empty_like(k_new)
+    q_new = torch.empty(3, 1, 8, 128, dtype=torch.bfloat16, device="cuda")
+    pos = torch.tensor(L0, dtype=torch.int32, device="cuda")
+
+    def step():
+        B_.mpfa_append_kv_paged(k_new, v_new, w_full.H_q, B_.MPFA_SMOOTH, st.stats, 1.0, st.kv, st.page_table, pos)
+        torch.add(pos, 1, out=st.seq_lens)
+        B_.mpfa_quantize_qk(q_new, None, flags, st.stats, st.q4, None, None, None)
+        decode_cache.decode_step(st)
+
+    def load_inputs(s):
+        k_new.copy_(torch.stack([kv_full[b][0][0, L0[b] + s:L0[b] + s + 1] for b in range(3)]))
+        v_new.copy_(torch.stack([kv_full[b][1][0, L0[b] + s:L0[b] + s + 1] for b in range(3)]))
+        q_new.copy_(w_full.q_sample[:, 20 + s:21 + s])
+        pos.copy_(torch.tensor([l + s for l in L0], dtype=torch.int32))
+
+    load_inputs(0)
+    step()                      # eager once: loads the kernels outside the capture (idempotent: same token, same slot)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for s in range(steps):
+        load_inputs(s)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert int(st.status.item()) == 0
+        got = st.out_f32.cpu().numpy()
+        for b in range(3):
+            n = L0[b] + s + 1
+            kb, vb = kv_full[b][0][:, :n].contiguous(), kv_full[b][1][:, :n].contiguous()
+            z = orc.stage1(orc.bf16_bits(w_full.q_sample[b:b + 1, 20 + s:21 + s].contiguous()), orc.bf16_bits(kb), orc.bf16_bits(vb),
+                           frozen=z0[b])
+            ref, _ = orc.decode(z.q_codes[:, :, 0], z.q_sf[:, :, 0], z.k_codes, z.k_sf, z.v_codes, z.delta, z.dq, z.dk, 1.0,
+                                w_full.softmax_scale, np.array([n], np.int32))
+            d = np.abs(got[b] - ref[0])
+            assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (s, b, float(d.max()), float(d.mean()))
