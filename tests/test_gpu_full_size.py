@@ -88,3 +88,39 @@ def test_decode_full_size_sampled_requests():
         assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (b, float(d.max()), float(d.mean()))
         assert bf16_neighbours_ok(out16[b], ref32[0]).all()
     print(f"decode cfg5: {len(sample)} requests checked, worst max-abs {worst:.2e}")
+
+
+def test_error_against_exact_attention_with_and_without_compensation(capsys):
+    """Reported, not gated beyond sanity: the kernel's error against exact (FP64) softmax attention on the unquantized
+    inputs, for the three ways of running it - smoothing + compensation (the method), smoothing with the compensation
+    term dropped, and the direct variant (no smoothing) - on the tiny configs (all rows) and on a row sample of the
+    16K benchmark config.  The figures are copied into the design notes."""
+    from paper_2609_33135_b200 import binding
+    table = []
+    for name, make, n_rows in (("cfg1", wl.config1_tiny, None), ("cfg1b_qbias", wl.config1b_tiny_qbias, None),
+                               ("cfg2_llama_16k", lambda: wl.config2_llama(16384), 512)):
+        w = make()
+        q, k, v = orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v)
+        rows = orc.all_rows(w.B, w.H_q, w.N_q) if n_rows is None else wl.sample_rows(8100, w.B, w.H_q, w.N_q, n_rows).numpy()
+        exact = orc.exact_rows(q, k, v, rows, w.softmax_scale, w.causal)
+        idx = [torch.from_numpy(rows[:, c].astype(np.int64)).cuda() for c in (0, 2, 1)]
+        errs = {}
+        for label, smooth, use_delta in (("method", True, True), ("no_compensation", True, False), ("direct", False, False)):
+            s1 = binding.stage1(w.q.cuda(), w.k.cuda(), w.v.cuda(), smooth=smooth)
+            if not use_delta:
+                s1.delta = None
+            out, _, status = binding.prefill(s1, w.causal, w.softmax_scale)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            got = out[idx[0], idx[1], idx[2]].float().cpu().numpy().astype(np.float64)
+            assert np.isfinite(got).all()
+            d = np.abs(got - exact)
+            errs[label] = (float(d.mean()), float(d.max()))
+        table.append((name, errs))
+        assert errs["method"][0] < 0.1
+    # where the query mean is not ~0 the compensation term must pay off
+    e1b = dict(table)["cfg1b_qbias"]
+    assert e1b["method"][0] < e1b["no_compensation"][0]
+    with capsys.disabled():
+        for name, errs in table:
+            print(f"{name}: " + "; ".join(f"{k} mean {m:.3e} max {x:.3e}" for k, (m, x) in errs.items()))
