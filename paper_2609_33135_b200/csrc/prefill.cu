@@ -60,6 +60,11 @@ template <bool PAGED> constexpr int REGS_UTIL = PAGED ? MPFA_REGS_UTIL_PAGED : 5
 template <bool PAGED> constexpr int REGS_CORR = PAGED ? MPFA_REGS_CORR_PAGED : 120;
 static_assert(4 * REGS_UTIL<false> + 8 * REGS_SOFTMAX + 4 * REGS_CORR<false> <= 16 * 128, "register pool");
 static_assert(4 * REGS_UTIL<true> + 8 * REGS_SOFTMAX + 4 * REGS_CORR<true> <= 16 * 128, "register pool");
+// the utility and correction warps give registers back (setmaxnreg.dec: the target must not exceed the 128 of the
+// launch, or the instruction is illegal), the softmax warps take them (setmaxnreg.inc: not below 128)
+static_assert(REGS_UTIL<false> <= 128 && REGS_UTIL<true> <= 128 && REGS_CORR<false> <= 128 && REGS_CORR<true> <= 128 &&
+              REGS_UTIL<false> >= 24 && REGS_UTIL<true> >= 24 && REGS_CORR<false> >= 24 && REGS_CORR<true> >= 24 &&
+              REGS_SOFTMAX >= 128 && REGS_SOFTMAX <= 255, "setmaxnreg direction");
 static_assert(REGS_SOFTMAX % 8 == 0 && REGS_UTIL<false> % 8 == 0 && REGS_CORR<false> % 8 == 0 && REGS_UTIL<true> % 8 == 0 &&
               REGS_CORR<true> % 8 == 0, "setmaxnreg granularity");
 
