@@ -1,9 +1,14 @@
 // QK4PV8 prefill (Algorithm 1 lines 6-20) for sm_100a.
 //
-// One CTA owns one 128-row query tile of one q head and walks its KV blocks (128 keys)
-// from the last visible block down to block 0 (Section 4.1).  Roles (512 threads):
-//   warp 0       TMA producer: K codes (tensor map, 64B swizzle), K scale factors and
-//                Delta_S (bulk copies) and V (tensor map, 128B swizzle) into 3-stage rings;
+// A work item is one 128-row query tile of one q head; its KV blocks (128 keys) are visited from the last
+// visible block down to block 0 (Section 4.1).  One persistent CTA per SM walks a static list of work items
+// (struct TileWalk) and keeps its pipeline running across item boundaries.  Roles (512 threads):
+//   warp 0       producer: K codes (tensor map, 64B swizzle), K scale factors and Delta_S (bulk copies)
+//                and V (tensor map, 128B swizzle) into rings of 4 (K) and 3 (V) stages; in the paged
+//                variant (template parameter PAGED, entry point mpfa_prefill_paged) every tile half is
+//                one bulk copy of a 64-token page slab, found through the page table;
+//   warp 2       paged variant only: re-tiles the pages' row-major K scales for tcgen05.cp and un-swizzles
+//                their Delta_S rows (idle otherwise; it also owns the tensor-memory allocation);
 //   warp 1       Q K^T issuer: per block a rank-one BF16 MMA seeds S with 1 x Delta_S
 //                (Eq. 11) and two block-scaled FP4 MMAs (K = 64 each) accumulate Q K^T into
 //                the same TMEM columns;
@@ -25,9 +30,11 @@
 //                between two dependent MMAs; the epilogue adds the two accumulators
 //                (the older one times the last alpha) and writes O / (448 l) * v_scale as BF16.
 // Tensor memory (512 columns): S [0,128) O0 [128,256) O1 [256,384), P_hat0 [384,416)
-// P_hat1 [416,448), scale factors of Q [448,456) and of two K blocks [456,464) [464,472).
+// P_hat1 [416,448), scale factors of two query tiles [448,464) and of two K blocks [464,472) [472,480).
 // Register budget is moved between the roles with setmaxnreg (56 for warps 0-3, 168 for the softmax warps,
 // 120 for the correction warps, whose epilogue holds two accumulator chunks at once).
+// Template parameter EW: the compensation-placement ablation (mpfa_prefill_variant): no seed MMA, Delta_S added
+// element by element by the softmax threads.
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises MPFA_DEV_TIMEOUT in
 // *device_status, all roles leave their loops, outstanding TMA copies are drained and
