@@ -62,9 +62,9 @@ def test_prefill_full_size_sampled_rows(name):
           f"vs exact FP64 attention (256 rows) mean {np.abs(got[:256] - exact).mean():.3e}")
 
 
-def test_decode_full_size_sampled_requests():
+def test_decode_full_size_all_requests():
     """Config 5 (32 requests, 16K..128K tokens, shuffled 64-token pages) exactly as bench.py runs it; the
-    oracle recomputes a sample of the requests (their K/V are read back from the GPU generator)."""
+    oracle recomputes every request (their K/V are read back from the GPU generator)."""
     from paper_2609_33135_b200 import decode_cache
     w = wl.config5_decode()
     st = decode_cache.build_cache(w, kv_device="cuda", want_f32=True)
@@ -72,7 +72,7 @@ def test_decode_full_size_sampled_requests():
     torch.cuda.synchronize()
     assert int(st.status.item()) == 0
     lens = w.seq_lens.numpy()
-    sample = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 0, 7, 19, 31})
+    sample = range(w.B)   # every request, all 32 heads each
     out32 = st.out_f32.cpu().numpy()
     out16 = st.out.view(torch.uint16).cpu().numpy()
     worst = 0.0
@@ -87,7 +87,7 @@ def test_decode_full_size_sampled_requests():
         worst = max(worst, float(d.max()))
         assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (b, float(d.max()), float(d.mean()))
         assert bf16_neighbours_ok(out16[b], ref32[0]).all()
-    print(f"decode cfg5: {len(sample)} requests checked, worst max-abs {worst:.2e}")
+    print(f"decode cfg5: {w.B} requests checked, worst max-abs {worst:.2e}")
 
 
 def test_error_against_exact_attention_with_and_without_compensation(capsys):
