@@ -18,8 +18,8 @@ pytestmark = pytest.mark.gpu
 CASES = {
     "cfg2_llama_16k": (lambda: wl.config2_llama(16384), 2048),
     "cfg3_qwen_32k": (lambda: wl.config3_qwen(32768), 2048),
-    "cfg3_qwen_64k": (lambda: wl.config3_qwen(65536), 1024),
-    "cfg4_long_128k": (lambda: wl.config4_long(131072), 1024),
+    "cfg3_qwen_64k": (lambda: wl.config3_qwen(65536), 2048),
+    "cfg4_long_128k": (lambda: wl.config4_long(131072), 2048),
 }
 
 
