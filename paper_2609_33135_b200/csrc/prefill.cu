@@ -57,8 +57,8 @@ constexpr int NTHREADS = 512;
 // setmaxnreg only moves registers inside the pool the CTA got at launch (512 threads x the 128 registers of the
 // launch bound); a request beyond the pool would block forever, so the split is checked here.
 #ifndef MPFA_REGS_UTIL_PAGED
-#define MPFA_REGS_UTIL_PAGED 96
-#define MPFA_REGS_CORR_PAGED 80
+#define MPFA_REGS_UTIL_PAGED 88
+#define MPFA_REGS_CORR_PAGED 88
 #endif
 constexpr int REGS_SOFTMAX = 168;
 // measured: the contiguous kernel gains 4 % when the correction warps' epilogue (two accumulator chunks in
@@ -764,9 +764,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
               mul2(q2, q3, EX2_(x2), EX2_(x3), 448.0f);
               acc2(sum0, sum1, q0, q1);
               acc2(sum2, sum3, q2, q3);
-              const uint32_t lo = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q0, q1), __NV_SATFINITE, __NV_E4M3);
-              const uint32_t hi = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(q2, q3), __NV_SATFINITE, __NV_E4M3);
-              packed[i] = (lo & 0xFFFFu) | (hi << 16);
+              // two conversions written into the halves of one register (no separate merge instruction)
+              asm("{.reg .b16 lo, hi;\n\t"
+                  "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+                  "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+                  "mov.b32 %0, {lo, hi};}"
+                  : "=r"(packed[i])
+                  : "f"(q0), "f"(q1), "f"(q2), "f"(q3));
             }
 #ifndef MPFA_ABLATE_NO_PST
             tmem_st8(tP + (c0 >> 2), packed);
