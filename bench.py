@@ -486,8 +486,8 @@ def run_ours(args, rank, world, local):
 
 
 # DRAM bytes per prefill launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum);
-# from profiles/prefill_kernel_llama_shape.md (65,322,240 read + 81,366,528 written), keyed by sequence length.
-NCU_TRAFFIC_BYTES = {16384: 146688768}
+# from profiles/prefill_kernel_llama_shape.md (65,293,056 read + 80,688,640 written), keyed by sequence length.
+NCU_TRAFFIC_BYTES = {16384: 145981696}
 
 
 def main():
