@@ -235,7 +235,8 @@ mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tens
  * blocks counted from key 0, visited last to first); lambda uses q_gscale[b] * k_gscale[b].
  * Delta_S is applied when the cache has a delta_s pool.  A page-table entry outside
  * [0, num_pages) raises MPFA_DEV_BAD_PAGE in *device_status (output of that request undefined,
- * no out-of-pool access).  q_lens (device, may be NULL): per-request number of queries, 0 <= q_lens[b] <= N_q
+ * no out-of-pool access); a seq_lens[b] above 64 * max_pages_per_req is treated as that bound.
+ * q_lens (device, may be NULL): per-request number of queries, 0 <= q_lens[b] <= N_q
  * (a batch of chunks of different lengths): request b's queries are rows 0 .. q_lens[b]-1 of its slab of q and
  * are the last q_lens[b] tokens of its context; the outputs of the remaining rows are zero.
  * out_bf16 [B, N_q, H_q, 128]; out_f32 optional. */

@@ -295,7 +295,8 @@ struct TileWalk {
     t.row0 = t.qt * TILE;
     const int n_q = (PAGED && pg.q_lens) ? min(pg.q_lens[t.b], pp.N_q) : pp.N_q;
     const int last_row = min(n_q - 1, t.row0 + TILE - 1);
-    const int n_kv = PAGED ? pg.seq_lens[t.b] : pp.N_kv;
+    // a length beyond what the page-table row can address is cut to it (no read past the row)
+    const int n_kv = PAGED ? min(pg.seq_lens[t.b], pg.max_pages * 64) : pp.N_kv;
     t.nkv = n_kv;
     t.nq = n_q;
     const int last_key = pp.causal ? min(n_kv - 1, last_row + (n_kv - n_q)) : n_kv - 1;   // bottom-right aligned

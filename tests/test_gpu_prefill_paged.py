@@ -181,3 +181,24 @@ def test_paged_prefill_batch_of_chunks_of_different_lengths():
         rows = orc.all_rows(1, H_q, QL[b])
         ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
         compare(o16n[b:b + 1], o32n[b:b + 1], rows, ref32, f"request {b}")
+
+
+def test_paged_prefill_length_beyond_the_page_table_is_cut_not_followed():
+    """A seq_lens entry larger than the page-table row can address must not make the kernel read past the row: the
+    length is treated as 64 * max_pages (here the same as the true length, so the result is unchanged)."""
+    from paper_2609_33135_b200 import binding as B_, decode_cache
+    w = wl.decode_workload("pp_clip", 361, 1, 4, 2, 1, 256, seq_lens=[256])   # exactly 4 pages, table row of 4
+    st = decode_cache.build_cache(w)
+    q4 = B_.Fp4Tensor.empty(1, 4, 64, "cuda")
+    B_.mpfa_quantize_qk(w.q_sample[:, :64].contiguous().cuda(), None, B_.MPFA_SMOOTH | B_.MPFA_STATS_FROZEN, st.stats, q4,
+                        None, None, None)
+    outs = []
+    for L in (256, 100000):
+        out = torch.empty(1, 64, 4, 128, dtype=torch.bfloat16, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B_.mpfa_prefill_paged(q4, st.kv, st.page_table, torch.tensor([L], dtype=torch.int32, device="cuda"), st.stats, 1.0,
+                              w.softmax_scale, out, None, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        outs.append(out)
+    assert torch.equal(outs[0].view(torch.uint16), outs[1].view(torch.uint16))
