@@ -101,3 +101,40 @@ def test_deterministic_and_argument_errors():
         binding.mpfa_quantize_qk(q[:, :255].contiguous(), None, 0, st, bad, None, None, ws)
     with pytest.raises(binding.MpfaError, match="invalid"):
         binding.mpfa_quantize_qk(q, None, 0, st, binding.Fp4Tensor(q4.codes, q4.sf, 1, 1, 128), None, None, ws)
+
+
+def _adversarial(kind: str, seed: int):
+    """Small tensors with the values that break sloppy quantizers: hand-built, not drawn from the workload recipe."""
+    import dataclasses
+    g = torch.Generator().manual_seed(seed)
+    B, N, Hq, Hkv = 2, 300, 4, 2
+    q = torch.randn(B, N, Hq, 128, generator=g)
+    k = torch.randn(B, N, Hkv, 128, generator=g)
+    v = torch.randn(B, N, Hkv, 128, generator=g)
+    if kind == "zeros":                 # an all-zero batch element (tensor scale 1) next to an ordinary one
+        q[0].zero_(); k[0].zero_(); v[0].zero_()
+    elif kind == "zero_blocks":         # blocks and whole heads of zeros inside a non-zero tensor, negative zeros
+        k[:, :, 0, :].zero_(); q[:, :, 1, 32:48] = 0.0; q[:, ::2, 2, :] = -0.0; v[:, 5:9] = -0.0
+    elif kind == "dynamic_range":       # 2^-120 .. 2^100 in one tensor: scales underflow to 0 and saturate at 448
+        e = torch.randint(-120, 100, (B, N, Hkv, 128), generator=g).float()
+        k = k.sign() * torch.exp2(e)
+        q = q * 1e-30
+        v = v * 1e30
+    elif kind == "ties":                # values on the E2M1 and E4M3 rounding boundaries after scaling
+        grid = torch.tensor([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 0.0, 7.0])
+        idx = torch.randint(0, 16, (B, N, Hkv, 128), generator=g)
+        k = grid[idx] * k.sign()
+        k[:, 0, :, 0] = 6.0 * 448.0 / 448.0
+        q = (torch.randint(-8, 9, (B, N, Hq, 128), generator=g).float()) * 0.25
+        v = torch.randint(-32, 33, (B, N, Hkv, 128), generator=g).float() * 0.0625 + 448.0 * (torch.rand(B, N, Hkv, 128, generator=g) < 0.01)
+    elif kind == "constant":            # every token identical: centered values are exactly zero
+        q = q[:, :1].expand(B, N, Hq, 128).clone(); k = k[:, :1].expand(B, N, Hkv, 128).clone()
+    w = wl.prefill_workload("adv", 1, B, N, Hq, Hkv, True)
+    return dataclasses.replace(w, q=q.to(torch.bfloat16), k=k.to(torch.bfloat16), v=v.to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("kind", ["zeros", "zero_blocks", "dynamic_range", "ties", "constant"])
+def test_stage1_bit_exact_on_adversarial_values(kind):
+    w = _adversarial(kind, 400 + len(kind))
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+    check_stage1(w, run_stage1_gpu(w), z)
