@@ -15,7 +15,10 @@
  * Pins (tests/test_oracle_*.py): brute-force nearest-value enumeration of all
  * 16 E2M1 and 256 E4M3 codes, exact integer column sums, Eq. 8 identity in
  * FP64, the identity-quantizer special case against textbook FP64 softmax
- * attention, softmax rows summing to one, traversal-order invariance in FP64.
+ * attention, softmax rows summing to one, traversal-order invariance in FP64;
+ * the reverse block order, the fixed scale 448 of P-hat (codes of a worked row,
+ * subnormal codes included) and the GQA head mapping against NumPy statements
+ * of the same steps on operands built code by code.
  * Parity unpinned (the paper prints no worked example for them, they are
  * readings fixed by this file): the per-tensor scale recipe, reciprocal-multiply
  * element scaling, the unit in which the compensation vector is stored, FP32
@@ -296,10 +299,12 @@ typedef struct {
  * from key 0, visited in descending order when `reverse` (Section 4.1).
  * s: logits in MMA units; lam: lambda' = softmax_scale * log2(e) * dQ * dK.
  * v: E4M3 codes [n, D] (v_f32 == NULL) or FP32 values [n, D].
- * p_fp8: quantize P to E4M3 with the fixed scale 448 (else keep FP32 P * 448). */
+ * p_fp8: quantize P to E4M3 with the fixed scale 448 (else keep FP32 P * 448).
+ * phat_out (optional, inspection only): receives, per key index, the E4M3 code
+ * the loop gave that key's P when its block was visited. */
 static void online_softmax_pv(const float *s, int k0, int k1, float lam, const uint8_t *v,
                               const float *v_f32, int block, int reverse, int p_fp8,
-                              softmax_state *st) {
+                              softmax_state *st, uint8_t *phat_out) {
   st->m = -INFINITY;
   st->l = 0.0f;
   for (int c = 0; c < D; ++c) st->o[c] = 0.0f;
@@ -327,7 +332,11 @@ static void online_softmax_pv(const float *s, int k0, int k1, float lam, const u
     for (int c = 0; c < D; ++c) acc[c] = alpha * st->o[c];
     for (int j = a; j < b; ++j) {
       float ph = p[j - a] * 448.0f;
-      if (p_fp8) ph = e4m3_tab[mpfa_oracle_e4m3_encode(ph)];
+      if (p_fp8) {
+        uint8_t code = mpfa_oracle_e4m3_encode(ph);
+        if (phat_out) phat_out[j] = code;
+        ph = e4m3_tab[code];
+      }
       if (v_f32) {
         const float *vr = v_f32 + (size_t)j * D;
         for (int c = 0; c < D; ++c) acc[c] += ph * vr[c];
@@ -380,7 +389,7 @@ static void prefill_rows_impl(const uint8_t *q_codes, const uint8_t *q_sf, const
     float lam = ((softmax_scale * 1.4426950408889634f) * dq[b]) * dk[b];
     softmax_state st;
     online_softmax_pv(s, 0, n, lam, v_codes + ((size_t)b * Hkv + hk) * Nkv * D, NULL, block_kv,
-                      reverse, p_fp8, &st);
+                      reverse, p_fp8, &st, NULL);
     for (int c = 0; c < D; ++c) {
       float o = (st.l > 0.0f) ? st.o[c] / (448.0f * st.l) * v_scale : 0.0f;
       out_f32[(size_t)r * D + c] = o;
@@ -447,7 +456,7 @@ void mpfa_oracle_decode(const uint8_t *q_codes, const uint8_t *q_sf, const uint8
       for (int sp = 0; sp < n_split; ++sp) {
         int k0 = sp * split, k1 = (sp + 1) * split > L ? L : (sp + 1) * split;
         online_softmax_pv(s, k0, k1, lam, v_codes + ((size_t)b * Hkv + hk) * Lmax * D, NULL, block_kv,
-                          reverse, p_fp8, &parts[sp]);
+                          reverse, p_fp8, &parts[sp], NULL);
         if (parts[sp].m > M) M = parts[sp].m;
       }
       float l = 0.0f, o[D];
@@ -487,7 +496,7 @@ void mpfa_oracle_mainloop_identity(const float *q, const float *k, const float *
     }
     float lam = softmax_scale * 1.4426950408889634f;
     softmax_state st;
-    online_softmax_pv(s, 0, n, lam, NULL, v, block_kv, reverse, 0, &st);
+    online_softmax_pv(s, 0, n, lam, NULL, v, block_kv, reverse, 0, &st, NULL);
     for (int c = 0; c < D; ++c) out_f32[(size_t)r * D + c] = (st.l > 0.0f) ? st.o[c] / (448.0f * st.l) : 0.0f;
     /* sum over keys of the final normalised probabilities, for the rows-sum-to-one pin */
     double tot = 0.0;
@@ -548,5 +557,38 @@ void mpfa_oracle_logits_rows(const uint8_t *q_codes, const uint8_t *q_sf, const 
                   q_sf + (((size_t)b * Hq + hq) * Nq + i) * NBLK,
                   k_codes + ((size_t)b * Hkv + hk) * Nkv * (D / 2), k_sf + ((size_t)b * Hkv + hk) * Nkv * NBLK,
                   delta ? delta + ((size_t)b * Hq + hq) * Nkv : NULL, Nkv, s_out + (size_t)r * Nkv);
+  }
+}
+
+/* Inspection entry point for the pins: the E4M3 codes of P-hat that the main
+ * loop assigns to every visible key of the listed rows (Section 4.1: fixed
+ * scale 448, quantized against the running maximum of the traversal), plus the
+ * final (m, l) of each row.  Same calls as prefill_rows_impl; nothing is
+ * computed differently.  codes_out: [n_rows, Nkv] (keys a row cannot see stay 0),
+ * ml_out: [n_rows, 2]. */
+void mpfa_oracle_phat_rows(const uint8_t *q_codes, const uint8_t *q_sf, const uint8_t *k_codes,
+                           const uint8_t *k_sf, const uint8_t *v_codes, const uint16_t *delta,
+                           const float *dq, const float *dk, float softmax_scale, int causal, int Nq, int Nkv,
+                           int Hq, int Hkv, int block_kv, int reverse, const int32_t *rows, int n_rows,
+                           uint8_t *codes_out, float *ml_out) {
+  init_tables();
+  int grp = Hq / Hkv;
+  for (int r = 0; r < n_rows; ++r) {
+    int b = rows[3 * r], hq = rows[3 * r + 1], i = rows[3 * r + 2];
+    int hk = hq / grp;
+    int n = visible_keys(i, Nq, Nkv, causal);
+    float *s = (float *)malloc(sizeof(float) * (size_t)(n > 0 ? n : 1));
+    logits_row_q4(q_codes + (((size_t)b * Hq + hq) * Nq + i) * (D / 2),
+                  q_sf + (((size_t)b * Hq + hq) * Nq + i) * NBLK,
+                  k_codes + ((size_t)b * Hkv + hk) * Nkv * (D / 2), k_sf + ((size_t)b * Hkv + hk) * Nkv * NBLK,
+                  delta ? delta + ((size_t)b * Hq + hq) * Nkv : NULL, n, s);
+    float lam = ((softmax_scale * 1.4426950408889634f) * dq[b]) * dk[b];
+    softmax_state st;
+    memset(codes_out + (size_t)r * Nkv, 0, (size_t)Nkv);
+    online_softmax_pv(s, 0, n, lam, v_codes + ((size_t)b * Hkv + hk) * Nkv * D, NULL, block_kv, reverse, 1, &st,
+                      codes_out + (size_t)r * Nkv);
+    ml_out[2 * r] = st.m;
+    ml_out[2 * r + 1] = st.l;
+    free(s);
   }
 }

@@ -262,3 +262,18 @@ def logits_rows(z: Quantized, rows, use_delta=True) -> np.ndarray:
                                   _p(z.delta if use_delta else None), Nq, Nkv, Hq, Hkv, _p(rows),
                                   rows.shape[0], _p(out))
     return out
+
+
+def phat_rows(z: Quantized, rows, softmax_scale: float, causal: bool, block_kv: int = BLOCK_KV,
+              reverse: bool = True, use_delta: bool = True):
+    """Inspection: E4M3 codes of P-hat per visible key [n,Nkv] and the final (m, l) [n,2] of rows [n,3]."""
+    rows = _c(rows, np.int32)
+    B, Hq, Nq, _ = z.q_codes.shape
+    Hkv, Nkv = z.k_codes.shape[1], z.k_codes.shape[2]
+    codes = np.empty((rows.shape[0], Nkv), np.uint8)
+    ml = np.empty((rows.shape[0], 2), np.float32)
+    lib().mpfa_oracle_phat_rows(_p(z.q_codes), _p(z.q_sf), _p(z.k_codes), _p(z.k_sf), _p(z.v_codes),
+                                _p(z.delta if use_delta else None), _p(_c(z.dq, np.float32)),
+                                _p(_c(z.dk, np.float32)), ctypes.c_float(softmax_scale), int(causal), Nq, Nkv, Hq,
+                                Hkv, block_kv, int(reverse), _p(rows), rows.shape[0], _p(codes), _p(ml))
+    return codes, ml

@@ -44,7 +44,8 @@ def test_traversal_order_only_changes_rounding():
     n_vis = np.full(8, 512, np.int32)
     a, _ = orc.mainloop_identity(q, k, v, n_vis, 1 / np.sqrt(128), 128, True)
     b, _ = orc.mainloop_identity(q, k, v, n_vis, 1 / np.sqrt(128), 128, False)
-    assert 0 < np.max(np.abs(a - b)) < 2e-6 or np.array_equal(a, b)
+    # FP32 P: the two orders are the same sum in another order, so they differ, but only by rounding
+    assert 0 < np.max(np.abs(a - b)) < 2e-6
 
 
 def _stage1(w, **kw):
