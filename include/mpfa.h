@@ -146,7 +146,8 @@ mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, int B, int 
  * part of the library image: every GPU that loads the library carries it until the
  * process exits.  Shapes whose statistics need more (mpfa_quantize_workspace_bytes(B, H_q,
  * H_kv) > MPFA_STATIC_SCRATCH_BYTES, i.e. roughly B * (H_q + H_kv) > 250) are rejected
- * with MPFA_ERR_WORKSPACE and nothing is launched.  The call allocates nothing and frees
+ * with MPFA_ERR_WORKSPACE and nothing is launched; with MPFA_STATS_FROZEN no statistics are
+ * accumulated, the buffer is not used and no limit applies.  The call allocates nothing and frees
  * nothing.  The first call on each device looks up the buffer's device address (with that
  * device current); make that first call before starting any stream capture.  All calls on
  * a device share the one buffer, which keeps whatever the previous call left in it: each
@@ -258,6 +259,20 @@ mpfa_status mpfa_decode(const mpfa_fp4_tensor *h_q, const mpfa_paged_kv *h_kv, c
                         int max_pages_per_req, const int32_t *seq_lens, const mpfa_stats *h_stats,
                         float v_scale, float softmax_scale, void *out_bf16, float *out_f32, void *workspace,
                         size_t workspace_bytes, int32_t *device_status, void *stream);
+
+/* ---- measurement aid ------------------------------------------------------------------- */
+
+/* (Not a step of the paper's method: the roofline denominator for Sections 5.1-5.2's three MMA kinds.)
+ * Launches one CTA per SM that issues 4 * iters back-to-back tcgen05.mma instructions of one kind,
+ * M = 128, N = n_cols (128 or 256), on operands resident in shared / tensor memory, and waits for the last:
+ *   kind 0  kind::f16, BF16 x BF16, K = 16 (the rank-one seed of Eq. 11)
+ *   kind 1  kind::f8f6f4, E4M3 x E4M3, K = 32, both operands in shared memory
+ *   kind 2  kind::f8f6f4, E4M3 x E4M3, K = 32, A in tensor memory (the P V form)
+ *   kind 3  kind::mxf4nvf4.block_scale.scale_vec::4X, E2M1 x E2M1, K = 64 (the Q K^T form)
+ * The caller times the call with CUDA events; mpfa_bench_mma_flops gives the FLOPs ONE CTA issued
+ * (multiply by the SM count).  Results are not meaningful data.  device_status as for the attention calls. */
+mpfa_status mpfa_bench_mma_peak(int kind, int n_cols, int iters, int32_t *device_status, void *stream);
+double mpfa_bench_mma_flops(int kind, int n_cols, int iters);
 
 /* ---- sizes, layout maps, diagnostics (host only, no CUDA calls) ----------------------- */
 size_t mpfa_quantize_workspace_bytes(int B, int H_q, int H_kv);

@@ -100,6 +100,10 @@ def lib() -> ctypes.CDLL:
         L.mpfa_prefill_paged.restype = i
         L.mpfa_prefill_paged.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_PagedKV), vp, i, vp, vp,
                                          ctypes.POINTER(_Stats), f, f, vp, vp, vp, vp]
+        L.mpfa_bench_mma_peak.restype = i
+        L.mpfa_bench_mma_peak.argtypes = [i, i, i, vp, vp]
+        L.mpfa_bench_mma_flops.restype = ctypes.c_double
+        L.mpfa_bench_mma_flops.argtypes = [i, i, i]
         _lib = L
     return _lib
 
@@ -373,3 +377,10 @@ def prefill(s1: Stage1, causal: bool, softmax_scale: float, want_f32: bool = Fal
         status = torch.zeros(1, dtype=torch.int32, device=dev)
     mpfa_prefill(s1.q, s1.k, s1.v_fp8, s1.delta, s1.stats, s1.v_scale, causal, softmax_scale, out, o32, status)
     return out, o32, status
+
+
+def mpfa_bench_mma_peak(kind: int, n_cols: int, iters: int, status: torch.Tensor) -> float:
+    """Enqueue the tensor-core rate probe; returns the FLOPs the whole grid issues (one CTA per SM)."""
+    _check(lib().mpfa_bench_mma_peak(kind, n_cols, iters, _ptr(status), _stream()), "mpfa_bench_mma_peak")
+    n_sm = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    return float(lib().mpfa_bench_mma_flops(kind, n_cols, iters)) * n_sm

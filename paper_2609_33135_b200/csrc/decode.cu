@@ -13,7 +13,7 @@
 //   S^T[key, head] = K Q^T       tcgen05.mma kind::mxf4nvf4 (E2M1 codes, UE4M3 block scales),
 //                                M = 128 keys, N = 16, K = 2 x 64 channels, FP32 in TMEM,
 //                                one 16-column slot per block of the item;
-//   softmax        one thread per key.  As each S^T lands: + Delta_S (Eq. 10), warp maximum.
+//   softmax        one thread per key.  As each S^T lands: + Delta_S (Eq. 11), warp maximum.
 //                  After the item's last block one exchange gives every block u the running
 //                  maximum m_u of the reverse traversal (max over the blocks visited so far),
 //                  then P = 2^(lam S - lam m_u), P_hat = E4M3(448 P) for all blocks at once,
@@ -508,7 +508,7 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
           const uint64_t d_q = smem_desc(sbase + D_OFF_Q + par * 1024, 16, 512, SWZ_64B);
           const uint32_t tS = tm + TM_S + (par * MAXBLK + t) * 16;
           if (has_delta) {
-            // S^T = Delta_S^T I (Eq. 10 seed): A = the stage's Delta_S rows, MN-major (keys contiguous), its
+            // S^T = Delta_S^T I (Eq. 11 seed): A = the stage's Delta_S rows, MN-major (keys contiguous), its
             // second group of eight K rows read from the zero block; B = identity
             const uint32_t a_ds = sbase + D_OFF_K + st * KST_BYTES + KST_DELTA;
             mma_bf16_ss(tS, smem_desc(a_ds, 1024, sbase + D_OFF_ZERO - a_ds, SWZ_128B), d_ident, id_ds, 0u);

@@ -101,10 +101,12 @@ enum {
   BAR_M_FULL = BAR_P_EMPTY + 2,         // [2] running maximum and alpha of block t published
   BAR_O_FULL = BAR_M_FULL + 2,          // [2] P V of block t accumulated into O[t & 1]
   BAR_O_READY = BAR_O_FULL + 2,         // [2] O[t & 1] rescaled for block t
-  BAR_L_FULL = BAR_O_READY + 2,         // [4] row sums of work item i published, slot i & 3.  The softmax warps can
-                                        //     be at most three (one-block) items ahead of the epilogue - P_hat of
-                                        //     block c needs P V of block c-2, which needs the correction warps - so
-                                        //     a slot is never two phases ahead of its reader
+  BAR_L_FULL = BAR_O_READY + 2,         // [4] row sums of the u-th item that has KV blocks (T > 0), slot u & 3.  The
+                                        //     softmax warps can be at most three (one-block) such items ahead of the
+                                        //     epilogue - P_hat of block c needs P V of block c-2, which needs the
+                                        //     correction warps - so a slot is never two phases ahead of its reader.
+                                        //     Items without blocks stay out of the ring: nothing bounds how many of
+                                        //     them the softmax warps could run through
   BAR_O_FREE = BAR_L_FULL + 4,          // the epilogue has read both accumulators (phase = items with T > 0)
   BAR_SF_READY = BAR_O_FREE + 1,        // [KSTAGES] paged source only: scales and Delta_S of the stage re-tiled
   NUM_BARS = BAR_SF_READY + KSTAGES
@@ -610,8 +612,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t tS = tm + TM_S + lane_off;
     const uint32_t tP = tm + (grp ? TM_P1 : TM_P0) + lane_off;
     bool ok = true;
+    uint32_t n_used = 0;   // items so far with T > 0: only those go through the row-sum ring
     for (; ok && walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
       const int T = tl.T;
+      if (T == 0) continue;   // nothing to attend to: the epilogue writes zeros without waiting for this role
       const int r_abs = tl.row0 + row;
       const int n_kv = PAGED ? tl.nkv : p.N_kv;
       const int n_q = PAGED ? tl.nq : p.N_q;
@@ -790,10 +794,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       if (!ok) break;
       // which group took the item's last block decides how the epilogue combines the two accumulators
-      float *s_fin = reinterpret_cast<float *>(smem + OFF_L) + (ti & 3) * 512;
+      float *s_fin = reinterpret_cast<float *>(smem + OFF_L) + (n_used & 3) * 512;
       s_fin[(grp * 2 + 0) * 128 + row] = l_own;
       s_fin[(grp * 2 + 1) * 128 + row] = m_own;
-      warp_arrive(cx.bar(BAR_L_FULL + (ti & 3)), lane);
+      warp_arrive(cx.bar(BAR_L_FULL + (n_used & 3)), lane);
+      ++n_used;
     }
   } else if (warp >= 12) {
     // =========================== correction + epilogue ===========================
@@ -803,6 +808,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const float *s_m = reinterpret_cast<const float *>(smem + OFF_M);
     const uint32_t tO0 = tm + TM_O0 + lane_off, tO1 = tm + TM_O1 + lane_off;
     bool ok = true;
+    uint32_t n_used = 0;   // items so far with T > 0 (slot and phase of the row-sum ring)
     for (; walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
       const int T = tl.T;
       const int r_abs = tl.row0 + row;
@@ -857,11 +863,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (ok) {
         if (T > 0) ok = cx.wait(BAR_O_FULL + last, ((gb + T - 1) >> 1) & 1u);
         if (ok && T > 1) ok = cx.wait(BAR_O_FULL + (last ^ 1), ((gb + T - 2) >> 1) & 1u);
-        ok = ok && cx.wait(BAR_L_FULL + (ti & 3), (ti >> 2) & 1u);
+        if (T > 0) ok = ok && cx.wait(BAR_L_FULL + (n_used & 3), (n_used >> 2) & 1u);
         tc_fence_after();
         if (ok && T > 0) {
           const float lam = lam_c;
-          const float *s_fin = reinterpret_cast<const float *>(smem + OFF_L) + (ti & 3) * 512;
+          const float *s_fin = reinterpret_cast<const float *>(smem + OFF_L) + (n_used & 3) * 512;
           const float l0 = s_fin[0 * 128 + row], m0 = s_fin[1 * 128 + row];
           const float l1 = s_fin[2 * 128 + row], m1 = s_fin[3 * 128 + row];
           const float mf = fmaxf(m0, m1);
@@ -916,6 +922,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
         }
       }
+      if (T > 0) ++n_used;
       if (!ok) break;
     }
   }

@@ -788,6 +788,10 @@ extern "C" mpfa_status mpfa_quantize_qk_static(const void *q_bf16, const void *k
                                                int H_q, int H_kv, int flags, mpfa_stats *st, mpfa_fp4_tensor *q_out,
                                                mpfa_fp4_tensor *k_out, void *delta_s_bf16, void *stream) {
   if (B <= 0 || H_q <= 0 || H_kv <= 0) return MPFA_ERR_INVALID_ARG;
+  // with frozen statistics nothing is accumulated: no scratch is touched, so no size limit applies
+  if (flags & MPFA_STATS_FROZEN)
+    return mpfa_quantize_qk(q_bf16, k_bf16, B, N_q, N_kv, H_q, H_kv, flags, st, q_out, k_out, delta_s_bf16, nullptr, 0,
+                            stream);
   if (carve(nullptr, B, H_q, H_kv).bytes > STATIC_SCRATCH_BYTES) return MPFA_ERR_WORKSPACE;
   void *scratch = nullptr;
   mpfa_status rc = static_scratch_address(&scratch);

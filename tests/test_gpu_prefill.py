@@ -168,3 +168,27 @@ def test_prefill_on_degenerate_inputs(kind):
     assert row_max.max() <= 3e-2 and d.mean() <= MEAN_ABS, (kind, float(row_max.max()), float(d.mean()))
     keep = row_max <= MAX_ABS
     compare(o16, o32, rows[keep], ref32[keep], kind)
+
+
+def test_prefill_many_items_without_keys_per_cta():
+    """Causal, far more queries than keys (N_q = 8192, N_kv = 128, 32 heads): 63 of the 64 query tiles see no key at
+    all, so every persistent CTA walks a dozen and more empty work items in a row.  They must come out as zeros,
+    the live tile must match the oracle, and no bounded wait may run out (status 0)."""
+    w = wl.prefill_workload("empty_items", 61, 1, 128, 32, 8, True, N_q=8192, q_bias=True)
+    from paper_2609_33135_b200 import binding
+    s1 = binding.stage1(w.q.cuda(), w.k.cuda(), w.v.cuda())
+    for _ in range(2):
+        out, o32, status = binding.prefill(s1, True, w.softmax_scale, want_f32=True)
+        out.fill_(3.0)
+        o32.fill_(3.0)
+        status.zero_()
+        binding.mpfa_prefill(s1.q, s1.k, s1.v_fp8, s1.delta, s1.stats, 1.0, True, w.softmax_scale, out, o32, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        o16n, o32n = out.view(torch.uint16).cpu().numpy(), o32.cpu().numpy()
+        assert not o32n[0, :8192 - 128].any() and not o16n[0, :8192 - 128].any()
+        z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+        rows = orc.all_rows(1, 32, 8192)
+        rows = rows[rows[:, 2] >= 8192 - 128]
+        ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
+        compare(o16n, o32n, rows, ref32, "empty items")

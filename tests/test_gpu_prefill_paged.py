@@ -202,3 +202,32 @@ def test_paged_prefill_length_beyond_the_page_table_is_cut_not_followed():
         assert int(status.item()) == 0
         outs.append(out)
     assert torch.equal(outs[0].view(torch.uint16), outs[1].view(torch.uint16))
+
+
+def test_paged_prefill_many_query_tiles_past_the_request_length():
+    """q_lens far below N_q (128 queries of 8192 slots, 32 heads): 63 of 64 query tiles of every head are empty work
+    items that precede the live ones in every CTA's list.  Zeros there, oracle parity on the live rows, status 0."""
+    from paper_2609_33135_b200 import binding as B_, decode_cache
+    H_q, H_kv, N_q, L = 32, 8, 8192, 1000
+    w = wl.decode_workload("pp_empty", 371, 1, H_q, H_kv, 1, L, seq_lens=[L], n_stat_tokens=256)
+    st = decode_cache.build_cache(w)
+    q_live = w.q_sample[:, :128].contiguous()
+    q_all = torch.zeros(1, N_q, H_q, 128, dtype=torch.bfloat16)
+    q_all[:, :128] = q_live
+    q4 = B_.Fp4Tensor.empty(1, H_q, N_q, "cuda")
+    B_.mpfa_quantize_qk(q_all.cuda(), None, B_.MPFA_SMOOTH | B_.MPFA_STATS_FROZEN, st.stats, q4, None, None, None)
+    out = torch.full((1, N_q, H_q, 128), 5.0, dtype=torch.bfloat16, device="cuda")
+    o32 = torch.full((1, N_q, H_q, 128), 5.0, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B_.mpfa_prefill_paged(q4, st.kv, st.page_table, st.seq_lens, st.stats, 1.0, w.softmax_scale, out, o32, status,
+                          q_lens=torch.tensor([128], dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o16n, o32n = out.view(torch.uint16).cpu().numpy(), o32.cpu().numpy()
+    assert not o32n[0, 128:].any() and not o16n[0, 128:].any()
+    k, v = w.kv_for_request(0)
+    z0 = orc.stage1(orc.bf16_bits(w.q_sample[0:1].contiguous()), orc.bf16_bits(k), orc.bf16_bits(v))
+    z = orc.stage1(orc.bf16_bits(q_live), orc.bf16_bits(k), orc.bf16_bits(v), frozen=z0)
+    rows = orc.all_rows(1, H_q, 128)
+    ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
+    compare(o16n[:, :128], o32n[:, :128], rows, ref32, "live tile")

@@ -61,3 +61,34 @@ def test_static_scratch_rejects_oversized_shapes():
     q4 = binding.Fp4Tensor.empty(B, Hq, 4)
     with pytest.raises(binding.MpfaError, match="workspace too small"):
         binding.mpfa_quantize_qk_static(q, None, 0, st, q4, None, None)
+
+
+def test_static_scratch_frozen_statistics_have_no_size_limit_and_nothing_is_allocated():
+    """With frozen statistics the quantizer accumulates nothing, so the fixed buffer is not used and the size limit
+    does not apply: the decode-time query batch of the paged-decode configuration (32 requests, 32 + 8 heads) goes
+    through although its statistics would not fit.  Also checks what the entry point is for: across the call the
+    device allocator's books and the driver's free-memory figure do not move."""
+    from paper_2609_33135_b200 import binding
+    B, Hq, Hkv = 32, 32, 8
+    assert binding.lib().mpfa_quantize_workspace_bytes(B, Hq, Hkv) > binding.lib().mpfa_static_scratch_bytes()
+    g = torch.Generator(device="cpu").manual_seed(5)
+    q = torch.randn(B, 1, Hq, 128, generator=g).to(torch.bfloat16).cuda()
+    st = binding.Stats.empty(B, Hq, Hkv)
+    st.q_mean.copy_(torch.randn(B, Hq, 128, generator=g) * 0.1)
+    st.q_gscale.fill_(0.002)
+    st.k_gscale.fill_(0.01)
+    flags = binding.MPFA_SMOOTH | binding.MPFA_STATS_FROZEN
+    ref = binding.Fp4Tensor.empty(B, Hq, 1)
+    binding.mpfa_quantize_qk(q, None, flags, st, ref, None, None, None)
+    out = binding.Fp4Tensor.empty(B, Hq, 1)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(2):
+        binding.mpfa_quantize_qk_static(q, None, flags, st, out, None, None)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    assert free1 == free0
+    assert torch.equal(out.codes, ref.codes) and torch.equal(out.sf, ref.sf)
+    assert out.codes.any()
