@@ -226,6 +226,16 @@ mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tens
                                  float softmax_scale, int variant, void *out_bf16, float *out_f32,
                                  int32_t *device_status, void *stream);
 
+/* The prefill calls have two work arrangements with identical per-row arithmetic (every row visits the same
+ * 128-key blocks in the same order, so outputs agree to FP32 rounding of the accumulator rescaling):
+ *   0 (default) one query tile per CTA, two softmax groups alternating over the KV blocks, two output
+ *     accumulators so that the rescaling of one is off the critical path of the MMAs into the other;
+ *   1 two adjacent query tiles per CTA, each with its own softmax warpgroup and output accumulator (the two query
+ *     stages of Section 5.1), every K/V block loaded once for both.  Measured slower on B200 (the single
+ *     accumulator per tile puts the rescaling between dependent MMAs); kept for that comparison.
+ * Process-wide switch (mpfa_prefill, mpfa_prefill_variant, mpfa_prefill_paged); MPFA_ERR_INVALID_ARG for other values. */
+int mpfa_set_prefill_arrangement(int arrangement);
+
 /* QK4PV8 prefill of a chunk of queries against the paged cache (Section 6: the serving path keeps
  * K/V only in low-bit pages; a later chunk of the prompt, or a prompt with a cached prefix,
  * attends to them there).  q: [B, H_q, N_q] tile-layout tensor holding, for every request, the

@@ -100,6 +100,8 @@ def lib() -> ctypes.CDLL:
         L.mpfa_prefill_paged.restype = i
         L.mpfa_prefill_paged.argtypes = [ctypes.POINTER(_Fp4), ctypes.POINTER(_PagedKV), vp, i, vp, vp,
                                          ctypes.POINTER(_Stats), f, f, vp, vp, vp, vp]
+        L.mpfa_set_prefill_arrangement.restype = i
+        L.mpfa_set_prefill_arrangement.argtypes = [i]
         L.mpfa_bench_mma_peak.restype = i
         L.mpfa_bench_mma_peak.argtypes = [i, i, i, vp, vp]
         L.mpfa_bench_mma_flops.restype = ctypes.c_double
@@ -384,3 +386,8 @@ def mpfa_bench_mma_peak(kind: int, n_cols: int, iters: int, status: torch.Tensor
     _check(lib().mpfa_bench_mma_peak(kind, n_cols, iters, _ptr(status), _stream()), "mpfa_bench_mma_peak")
     n_sm = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
     return float(lib().mpfa_bench_mma_flops(kind, n_cols, iters)) * n_sm
+
+
+def mpfa_set_prefill_arrangement(arrangement: int) -> None:
+    """0 (default): one query tile per CTA; 1: two query tiles per CTA.  Same arithmetic row by row."""
+    _check(lib().mpfa_set_prefill_arrangement(arrangement), "mpfa_set_prefill_arrangement")

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmpfa.so")
-SOURCES = ["quantize.cu", "prefill.cu", "decode.cu", "api.cu", "mma_peak.cu"]
+SOURCES = ["quantize.cu", "prefill.cu", "prefill_pair.cu", "decode.cu", "api.cu", "mma_peak.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
 

@@ -45,14 +45,13 @@
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "prefill_common.cuh"
 
 namespace mpfa {
 namespace {
 
 constexpr int KSTAGES = 4;
 constexpr int VSTAGES = 3;
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM clock: far beyond any legitimate wait
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;       // drain path only
 constexpr int NTHREADS = 512;
 // setmaxnreg only moves registers inside the pool the CTA got at launch (512 threads x the 128 registers of the
 // launch bound); a request beyond the pool would block forever, so the split is checked here.
@@ -122,75 +121,6 @@ constexpr uint32_t TM_S = 0, TM_O0 = 128, TM_O1 = 256, TM_P0 = 384, TM_P1 = 416,
                    TM_SFK0 = 464, TM_SFK1 = 472;
 constexpr uint32_t TMEM_COLS = 512;
 
-struct PrefillParams {
-  const uint8_t *q_sf;
-  const uint8_t *k_sf;
-  const __nv_bfloat16 *delta;  // may be null
-  const float *q_gscale;
-  const float *k_gscale;
-  __nv_bfloat16 *out;
-  float *out_f32;  // may be null
-  int32_t *status;
-  int B, N_q, N_kv, H_q, H_kv, nq_tiles, nk_tiles, n_items;
-  int causal;
-  float softmax_scale, v_scale;
-};
-
-// K, V and Delta_S read from the paged cache instead of contiguous tensors: 64-token pages whose
-// (page, kv head) slabs are stored as halves of this kernel's operand tiles (same swizzles), K scales
-// row-major [token][8] and Delta_S [page][q head][64] with its 16-byte groups XOR-ed by (q head mod G).
-struct PagedSrc {
-  const uint8_t *k_codes, *k_sf, *v_fp8;
-  const __nv_bfloat16 *delta;   // may be null
-  const int32_t *page_table;    // [B, max_pages]
-  const int32_t *seq_lens;      // [B] keys of each request (the last q_lens[b] of them are the queries' own)
-  const int32_t *q_lens;        // [B] queries of each request, <= N_q; null: N_q for all
-  int max_pages, num_pages;
-};
-
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-// Packed FP32 pairs (one issue slot for two IEEE operations; each half rounds like the scalar form).
-__device__ __forceinline__ void fma2(float &d0, float &d1, float a0, float a1, float b, float c) {
-  asm("{.reg .b64 ra, rb, rc, rd;\n\t"
-      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
-      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;}"
-      : "=f"(d0), "=f"(d1)
-      : "f"(a0), "f"(a1), "f"(b), "f"(c));
-}
-__device__ __forceinline__ void mul2(float &d0, float &d1, float a0, float a1, float b) {
-  asm("{.reg .b64 ra, rb, rd;\n\t"
-      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\t"
-      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;}"
-      : "=f"(d0), "=f"(d1)
-      : "f"(a0), "f"(a1), "f"(b));
-}
-__device__ __forceinline__ void acc2(float &d0, float &d1, float a0, float a1) {
-  asm("{.reg .b64 ra, rd;\n\t"
-      "mov.b64 ra, {%2, %3};\n\tmov.b64 rd, {%0, %1};\n\t"
-      "add.rn.f32x2 rd, rd, ra;\n\tmov.b64 {%0, %1}, rd;}"
-      : "+f"(d0), "+f"(d1)
-      : "f"(a0), "f"(a1));
-}
-
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-template <int N>
-__device__ __forceinline__ void setmaxnreg_inc() {
-  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
-}
-template <int N>
-__device__ __forceinline__ void setmaxnreg_dec() {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
-}
-
 // Optional timeline capture for tuning (compiled in only with -DMPFA_TRACE): one CTA records
 // clock64() at fixed points of every role, [role][block][event].
 #ifdef MPFA_TRACE
@@ -205,69 +135,6 @@ __device__ int g_trace_cta = 0;
 #define TR_INIT() do {} while (0)
 #define TR(role, t, ev) do {} while (0)
 #endif
-
-// One arrival per warp: every lane's earlier shared-memory writes and tensor-memory accesses are
-// ordered before it by the warp-level barrier.
-__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
-  __syncwarp();
-  if (lane == 0) mbar_arrive(bar);
-}
-
-struct Ctx {
-  uint32_t bars;      // shared address of barrier 0
-  volatile int *abort_flag;
-  int32_t *status;
-  __device__ __forceinline__ uint32_t bar(int i) const { return bars + 8u * (uint32_t)i; }
-  __device__ __forceinline__ bool probe(int i, uint32_t parity) const { return mbar_try_wait(bar(i), parity); }
-  // Bounded wait.  try_wait may itself suspend the thread for a system-dependent interval, so
-  // the bound is on elapsed SM clock cycles (about 2 s), checked once per 32 polls to keep the
-  // hand-off latency at the cost of a poll.  Also gives up as soon as another role has failed.
-  __device__ __forceinline__ bool wait(int i, uint32_t parity) const {
-    const uint32_t a = bar(i);
-    if (mbar_try_wait(a, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-      for (int k = 0; k < 32; ++k) {
-        if (mbar_try_wait_hint(a, parity, 1000u)) return true;   // the hardware may park the thread meanwhile
-      }
-      if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
-    }
-    *abort_flag = 1;
-    atomicOr(status, MPFA_DEV_TIMEOUT);
-    return false;
-  }
-};
-
-// Paged source: the two physical pages of KV block jb (t-th block of the traversal) of an item.  Every 16 blocks
-// the warp reads 32 page ids with one coalesced load (lane l: page index 2 jb + 1 - l); in between the ids come
-// from the lanes' registers.  A page past the end of the context (all its keys are masked) or with an id outside
-// the pool (reported in *status) is replaced by the block's other page, so operand tiles always hold finite bytes.
-struct PageLookup {
-  int ids;
-  __device__ __forceinline__ void get(const PagedSrc &pg, int32_t *status, int b, int nkv, int t, int jb, int lane,
-                                      int &page_lo, int &page_hi) {
-    if ((t & 15) == 0) {
-      const int n_pg = (nkv + 63) >> 6;
-      const int pi = 2 * jb + 1 - lane;
-      int id = -1;
-      if (pi >= 0 && pi < n_pg) {
-        id = pg.page_table[(size_t)b * pg.max_pages + pi];
-        if (id < 0 || id >= pg.num_pages) {
-          atomicOr(status, MPFA_DEV_BAD_PAGE);
-          id = -1;
-        }
-      }
-      ids = id;
-    }
-    page_hi = __shfl_sync(0xffffffffu, ids, (t & 15) * 2);
-    page_lo = __shfl_sync(0xffffffffu, ids, (t & 15) * 2 + 1);
-    if (page_hi < 0) page_hi = page_lo;
-    if (page_lo < 0) page_lo = page_hi < 0 ? 0 : page_hi;
-    if (page_hi < 0) page_hi = 0;
-  }
-};
 
 // One work item: a 128-row query tile of one q head.
 struct Tile {
@@ -743,7 +610,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         TR(2 + grp, c, 4);
         const float a_own = (m_t == m_own) ? 1.0f : ex2_approx(__fmul_rn(m_own - m_t, lam));
         // P = 2^(lam S - lam m) (Eq. 4)
-        const float cc = (m_t == -INFINITY) ? 0.0f : -__fmul_rn(m_t, lam);
+        // the factor 448 of the E4M3 operand is folded into the exponent: q = 448 P = 2^(lam S - lam m + log2 448)
+        const float cc = (m_t == -INFINITY) ? 0.0f : __fsub_rn(8.8073549220576042f, __fmul_rn(m_t, lam));
         float sum0 = 0.0f, sum1 = 0.0f, sum2 = 0.0f, sum3 = 0.0f;
 #ifdef MPFA_ABLATE_NO_SOFTMAX
         sum0 = __uint_as_float(s[5]);
@@ -762,11 +630,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             uint32_t packed[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-              float x0, x1, x2, x3, q0, q1, q2, q3;
+              float x0, x1, x2, x3;
               fma2(x0, x1, __uint_as_float(s[c0 + 4 * i]), __uint_as_float(s[c0 + 4 * i + 1]), lam, cc);
               fma2(x2, x3, __uint_as_float(s[c0 + 4 * i + 2]), __uint_as_float(s[c0 + 4 * i + 3]), lam, cc);
-              mul2(q0, q1, EX2_(x0), EX2_(x1), 448.0f);
-              mul2(q2, q3, EX2_(x2), EX2_(x3), 448.0f);
+              const float q0 = EX2_(x0), q1 = EX2_(x1), q2 = EX2_(x2), q3 = EX2_(x3);
               acc2(sum0, sum1, q0, q1);
               acc2(sum2, sum3, q2, q3);
               // two conversions written into the halves of one register (no separate merge instruction)
@@ -933,40 +800,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   if (warp == 2) tmem_dealloc(tm, TMEM_COLS);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// The driver entry point is looked up through the runtime so the library does not link libcuda.
-mpfa_status get_encoder(EncodeTiledFn *fn) {
-  static EncodeTiledFn cached = nullptr;
-  if (!cached) {
-    void *ptr = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    MPFA_CUDA_OK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q));
-    if (q != cudaDriverEntryPointSuccess || !ptr) return cuda_fail(cudaErrorNotSupported);
-    cached = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  *fn = cached;
-  return MPFA_OK;
-}
-
-// 2D byte tensor [rows][row_bytes], box = 128 rows x row_bytes, hardware swizzle = row_bytes.
-mpfa_status make_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, uint64_t rows, uint32_t row_bytes) {
-  cuuint64_t dims[2] = {row_bytes, rows};
-  cuuint64_t strides[1] = {row_bytes};
-  cuuint32_t box[2] = {row_bytes, 128};
-  cuuint32_t es[2] = {1, 1};
-  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, es,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
-                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    g_last_cuda_error = (int)r;
-    return MPFA_ERR_CUDA;
-  }
-  return MPFA_OK;
-}
-
 }  // namespace
 }  // namespace mpfa
 
@@ -979,6 +812,15 @@ extern "C" int mpfa_debug_set_trace(long long *buf, int cta) {
   return 0;
 }
 #endif
+
+// 0: one query tile per CTA, two softmax groups alternating over KV blocks (the faster one on B200, see
+// prefill_pair.cu's header for the measured comparison); 1: two query tiles per CTA (prefill_pair.cu)
+static int g_arrangement = 0;
+extern "C" int mpfa_set_prefill_arrangement(int a) {
+  if (a != 0 && a != 1) return MPFA_ERR_INVALID_ARG;
+  g_arrangement = a;
+  return MPFA_OK;
+}
 
 extern "C" mpfa_status mpfa_prefill(const mpfa_fp4_tensor *q, const mpfa_fp4_tensor *k, const uint8_t *v_fp8,
                                     const void *delta_s_bf16, const mpfa_stats *st, float v_scale, int causal,
@@ -1009,13 +851,6 @@ extern "C" mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *q, const mpfa
   if (n_cta >= (1ull << 31)) return MPFA_ERR_UNSUPPORTED;
   mpfa_status rc = check_arch();
   if (rc != MPFA_OK) return rc;
-  EncodeTiledFn enc;
-  rc = get_encoder(&enc);
-  if (rc != MPFA_OK) return rc;
-  CUtensorMap tq, tk, tv;
-  if ((rc = make_map(enc, &tq, q->codes, q_rows, 64)) != MPFA_OK) return rc;
-  if ((rc = make_map(enc, &tk, k->codes, k_rows, 64)) != MPFA_OK) return rc;
-  if ((rc = make_map(enc, &tv, v_fp8, k_rows, 128)) != MPFA_OK) return rc;
   PrefillParams p;
   p.q_sf = q->sf;
   p.k_sf = k->sf;
@@ -1036,6 +871,14 @@ extern "C" mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *q, const mpfa
   p.softmax_scale = softmax_scale;
   p.v_scale = v_scale;
   p.n_items = (int)n_cta;
+  if (g_arrangement == 1) return launch_prefill_pair(q, k, v_fp8, p, ew, static_cast<cudaStream_t>(stream));
+  EncodeTiledFn enc;
+  rc = get_encoder(&enc);
+  if (rc != MPFA_OK) return rc;
+  CUtensorMap tq, tk, tv;
+  if ((rc = make_map(enc, &tq, q->codes, q_rows, 64)) != MPFA_OK) return rc;
+  if ((rc = make_map(enc, &tk, k->codes, k_rows, 64)) != MPFA_OK) return rc;
+  if ((rc = make_map(enc, &tv, v_fp8, k_rows, 128)) != MPFA_OK) return rc;
   int dev = 0, n_sm = 0;
   MPFA_CUDA_OK(cudaGetDevice(&dev));
   MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
@@ -1072,11 +915,6 @@ extern "C" mpfa_status mpfa_prefill_paged(const mpfa_fp4_tensor *q, const mpfa_p
   const uint64_t n_cta = (uint64_t)q->B * q->H * nq_tiles;
   mpfa_status rc = check_arch();
   if (rc != MPFA_OK) return rc;
-  EncodeTiledFn enc;
-  rc = get_encoder(&enc);
-  if (rc != MPFA_OK) return rc;
-  CUtensorMap tq;
-  if ((rc = make_map(enc, &tq, q->codes, q_rows, 64)) != MPFA_OK) return rc;
   PrefillParams p;
   p.q_sf = q->sf;
   p.k_sf = nullptr;
@@ -1107,6 +945,12 @@ extern "C" mpfa_status mpfa_prefill_paged(const mpfa_fp4_tensor *q, const mpfa_p
   pg.q_lens = q_lens;
   pg.max_pages = max_pages_per_req;
   pg.num_pages = kv->num_pages;
+  if (g_arrangement == 1) return launch_prefill_pair_paged(q, p, pg, static_cast<cudaStream_t>(stream));
+  EncodeTiledFn enc;
+  rc = get_encoder(&enc);
+  if (rc != MPFA_OK) return rc;
+  CUtensorMap tq;
+  if ((rc = make_map(enc, &tq, q->codes, q_rows, 64)) != MPFA_OK) return rc;
   int dev = 0, n_sm = 0;
   MPFA_CUDA_OK(cudaGetDevice(&dev));
   MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));

@@ -192,3 +192,34 @@ def test_prefill_many_items_without_keys_per_cta():
         rows = rows[rows[:, 2] >= 8192 - 128]
         ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
         compare(o16n, o32n, rows, ref32, "empty items")
+
+
+@pytest.fixture
+def two_tile_arrangement():
+    from paper_2609_33135_b200 import binding
+    binding.mpfa_set_prefill_arrangement(1)
+    yield
+    binding.mpfa_set_prefill_arrangement(0)
+
+
+@pytest.mark.parametrize("name", ["cfg1b_qbias", "causal_384_gqa", "ragged_causal", "ragged_noncausal_nq_lt_nkv",
+                                  "causal_offset", "causal_nq_gt_nkv", "many_one_block_items", "many_short_items"])
+def test_two_tile_arrangement_matches_oracle(two_tile_arrangement, name):
+    """Section 5.1's arrangement (two query tiles per CTA, a softmax warpgroup and an accumulator each) is the same
+    arithmetic row by row: same oracle, same tolerance.  Odd tile counts leave one stage of the last pair idle."""
+    w = CASES[name]()
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+    rows = orc.all_rows(w.B, w.H_q, w.N_q)
+    ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, w.causal)
+    o16, o32 = run_gpu(w)
+    compare(o16, o32, rows, ref32, name)
+
+
+def test_two_tile_arrangement_sampled_rows_and_empty_items(two_tile_arrangement):
+    w = wl.prefill_workload("mid2", 62, 1, 4096 + 128, 8, 2, True, q_bias=True)   # odd number of query tiles
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+    rows = wl.sample_rows(62, w.B, w.H_q, w.N_q, 256).numpy()
+    ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
+    o16, o32 = run_gpu(w)
+    compare(o16, o32, rows, ref32, "4k+128, two tiles per CTA")
+    test_prefill_many_items_without_keys_per_cta()
