@@ -24,7 +24,8 @@
  *     shape and alignment errors are detected on the host before anything is launched.
  *     Errors found on the device (a bounded wait that gave up, a page index out of range)
  *     are OR-ed into *device_status, which the caller reads after synchronising.
- *   - Results are deterministic: the same inputs give bit-identical outputs.
+ *   - Results are deterministic: the same call (shapes, workspace size) on the same inputs gives bit-identical
+ *     outputs; no floating-point atomics are used anywhere.
  *
  * Physical layouts (all offsets in bytes, N_pad = N rounded up to a multiple of 128)
  *   NVFP4 tensor ("tile layout", mpfa_fp4_tensor):
@@ -127,10 +128,18 @@ typedef struct {
  *   k_bf16 [B, N_kv, H_kv, 128] or NULL (quantize Q only);
  *   q_out / k_out: tile-layout tensors with B, H, N filled in by the caller;
  *   delta_s_bf16 [B, H_q, N_kv_pad]: required iff MPFA_SMOOTH and k_bf16 != NULL;
- *   workspace: mpfa_quantize_workspace_bytes() bytes, 256-byte aligned; contents are
- *          scratch (column sums and maxima), overwritten by every call.
- * All arithmetic is specified bit by bit (FP64 column sums, one rounding to FP32, IEEE
- * divisions); outputs are reproducible to the bit. */
+ *   workspace: 256-byte aligned scratch, overwritten by every call (not needed with MPFA_STATS_FROZEN).
+ *          mpfa_quantize_workspace_bytes() is the size that lets the statistics pass cut the token axis into
+ *          its full 32 slices; any size down to mpfa_quantize_workspace_min_bytes() (one slice) is accepted and
+ *          only lowers the parallelism of that pass; less: MPFA_ERR_WORKSPACE.
+ * All arithmetic is specified step by step (FP64 column sums, one rounding to FP32, IEEE divisions).  The column
+ * sums are added in a fixed order (tokens ascending within a thread, then token lanes, then slices; the order is a
+ * function of the shapes, the workspace size and the device's SM count), so the outputs are reproducible bit for
+ * bit for any input.  They
+ * equal the single ascending FP64 sum of Eq. 7 - and every code and scale derived from it - bit for bit whenever
+ * each partial sum is exactly representable in FP64, which holds for BF16 inputs whose nonzero magnitudes in a
+ * column span fewer than about 40 binades over up to 2^17 tokens; outside that range the mean may differ from the
+ * sequential sum in its last FP32 bit. */
 mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, int B, int N_q, int N_kv, int H_q,
                              int H_kv, int flags, mpfa_stats *h_stats, mpfa_fp4_tensor *h_q_out,
                              mpfa_fp4_tensor *h_k_out, void *delta_s_bf16, void *workspace,
@@ -144,8 +153,9 @@ mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, int B, int 
  * Arguments and results are exactly those of mpfa_quantize_qk without the workspace pair.
  * The column sums and maxima live in a fixed MPFA_STATIC_SCRATCH_BYTES buffer that is
  * part of the library image: every GPU that loads the library carries it until the
- * process exits.  Shapes whose statistics need more (mpfa_quantize_workspace_bytes(B, H_q,
- * H_kv) > MPFA_STATIC_SCRATCH_BYTES, i.e. roughly B * (H_q + H_kv) > 250) are rejected
+ * process exits (the statistics pass uses as many token slices as fit in it).  Shapes whose
+ * statistics need more (mpfa_quantize_workspace_min_bytes(B, H_q, H_kv) >
+ * MPFA_STATIC_SCRATCH_BYTES, i.e. roughly B * (H_q + H_kv) > 250) are rejected
  * with MPFA_ERR_WORKSPACE and nothing is launched; with MPFA_STATS_FROZEN no statistics are
  * accumulated, the buffer is not used and no limit applies.  The call allocates nothing and frees
  * nothing.  The first call on each device looks up the buffer's device address (with that
@@ -286,6 +296,7 @@ double mpfa_bench_mma_flops(int kind, int n_cols, int iters);
 
 /* ---- sizes, layout maps, diagnostics (host only, no CUDA calls) ----------------------- */
 size_t mpfa_quantize_workspace_bytes(int B, int H_q, int H_kv);
+size_t mpfa_quantize_workspace_min_bytes(int B, int H_q, int H_kv);
 size_t mpfa_decode_workspace_bytes(int B, int H_q, int H_kv, int max_pages_per_req);
 size_t mpfa_fp4_codes_bytes(int B, int H, int N);
 size_t mpfa_fp4_sf_bytes(int B, int H, int N);

@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         sz, i, f, vp = ctypes.c_size_t, ctypes.c_int, ctypes.c_float, ctypes.c_void_p
         L.mpfa_quantize_workspace_bytes.restype = sz
         L.mpfa_quantize_workspace_bytes.argtypes = [i, i, i]
+        L.mpfa_quantize_workspace_min_bytes.restype = sz
+        L.mpfa_quantize_workspace_min_bytes.argtypes = [i, i, i]
         L.mpfa_decode_workspace_bytes.restype = sz
         L.mpfa_decode_workspace_bytes.argtypes = [i, i, i, i]
         for name in ("mpfa_fp4_codes_bytes", "mpfa_fp4_sf_bytes", "mpfa_delta_s_bytes", "mpfa_v_fp8_bytes"):

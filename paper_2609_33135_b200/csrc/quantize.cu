@@ -40,58 +40,71 @@ __device__ __forceinline__ void unpack8(const uint4 &u, float (&f)[8]) {
 }
 
 // One pass over a tensor [B, N, cols] gives, per column, everything the statistics need:
-//   the sum in FP64 (Eq. 7) - for BF16 inputs whose nonzero magnitudes are >= 2^-14 every partial sum
-//   of up to 2^17 tokens is exactly representable, so the accumulation order cannot change the result;
+//   the sum in FP64 (Eq. 7);
 //   max x and max (-x) - rounding is monotonic and symmetric, so
 //   max_t |fl(x_t - mu)| = max(fl(max x - mu), fl(mu - min x)) and no second pass over the tensor is
 //   needed for the per-tensor scale.
-// A CTA covers 256 columns x COLSTAT_TOKENS tokens: thread = (token lane 0..7, 8 columns), a warp
-// reads 512 contiguous bytes of one token row, four independent 16-byte loads in flight per thread;
-// the eight token lanes are folded in shared memory, then one atomic per column and statistic.
-// Maxima are stored as order-preserving unsigned keys so that a zeroed workspace is the identity.
+// The token axis is cut into S contiguous slices.  A CTA covers 256 columns x one slice: thread = (token lane
+// 0..7, 8 columns), a warp reads 512 contiguous bytes of one token row, four independent 16-byte loads in
+// flight per thread; each thread adds its tokens in ascending order, the eight token lanes are folded in lane
+// order in shared memory, and the slice's partial result goes to the workspace.  The finalize kernel adds the S
+// partial sums in slice order.  Every addition order is fixed by (N, S), so the result is reproducible bit for
+// bit for any input; it equals the oracle's single ascending FP64 sum whenever all these sums are exact (always
+// true for BF16 inputs whose exponents span fewer than about 40 binades per column).
 constexpr int COLSTAT_COLS = 256;
-constexpr int COLSTAT_TOKENS = 256;
-
-__device__ __forceinline__ unsigned int ordered_key(float f) {   // monotonic float -> unsigned, key(-inf) > 0
-  const unsigned int b = __float_as_uint(f);
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
-__device__ __forceinline__ float from_ordered_key(unsigned int k) {
-  return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
-}
+constexpr int STAT_MAX_SLICES = 32;
 
 // One launch covers up to two tensors (Q and K): blockIdx.y runs over the 256-column groups of the first, then
-// of the second; blocks past a tensor's last token tile leave at once.
+// of the second; blocks past a tensor's last slice leave at once.  The block that finishes a column group last
+// (a counter per group, zeroed by a memory-set node before the launch) adds the slices' partial sums in slice order
+// - which block does it cannot change the result - and writes mean = fl(sum / N) (0 without smoothing) and the
+// group's max |x - mean| from the column extremes (an exact, order-free maximum); the block that finishes the
+// whole launch last turns the per-batch-element maxima into the tensor scales.
 struct ColTensor {
   const __nv_bfloat16 *x;   // null: tensor absent (ygroups = 0)
-  int N, cols, ygroups;
-  double *sums;
-  unsigned int *kmax, *knegmax;
+  int N, cols, ygroups, slices, slice_len;
+  double *psum;             // [B][slices][cols]
+  float *pmax, *pneg;       // [B][slices][cols]
+  unsigned int *amax;       // [B], zero at launch
+  float *mean, *gscale;
 };
 
-__device__ __forceinline__ void colstat_body(const __nv_bfloat16 *__restrict__ x, const int N, const int cols,
-                                             double *__restrict__ sums, unsigned int *__restrict__ kmax,
-                                             unsigned int *__restrict__ knegmax, const int yg) {
+__device__ __forceinline__ void colstat_body(const ColTensor &a, const int yg, unsigned int *group_counter,
+                                             unsigned int *launch_counter, const unsigned int n_groups, const int smooth,
+                                             const ColTensor &t0, const ColTensor &t1) {
   __shared__ double s_sum[8][COLSTAT_COLS];
   __shared__ float s_max[8][COLSTAT_COLS], s_neg[8][COLSTAT_COLS];
-  if ((int)blockIdx.x * COLSTAT_TOKENS >= N) return;
+  __shared__ bool s_last;
+  const int sl = blockIdx.x;
+  if (sl >= a.slices) return;
   const int b = blockIdx.z;
+  const int N = a.N, cols = a.cols;
+  const __nv_bfloat16 *__restrict__ x = a.x;
   const int tl = threadIdx.x >> 5, cg = threadIdx.x & 31;
   const int col = yg * COLSTAT_COLS + cg * 8;
-  const int t0 = blockIdx.x * COLSTAT_TOKENS;
-  const int t1 = min(N, t0 + COLSTAT_TOKENS);
+  const int t0i = sl * a.slice_len;
+  const int t1i = min(N, t0i + a.slice_len);
   double acc[8];
   float mx[8], ng[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.0, mx[i] = -INFINITY, ng[i] = -INFINITY;
   if (col < cols) {
-    const __nv_bfloat16 *p = x + ((size_t)b * N + t0 + tl) * cols + col;
+    const __nv_bfloat16 *p = x + ((size_t)b * N + t0i + tl) * cols + col;
     const size_t step = (size_t)8 * cols;
-    int t = t0 + tl;
-    for (; t + 24 < t1; t += 32, p += 4 * step) {
-      uint4 u[4];
+    int t = t0i + tl;
+    // four loads of the next round are in flight while the current four are added (tokens still ascending)
+    uint4 u[4], un[4];
+    bool have = t + 24 < t1i;
+    if (have) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) u[j] = *reinterpret_cast<const uint4 *>(p + j * step);
+      for (int j = 0; j < 4; ++j) u[j] = __ldcs(reinterpret_cast<const uint4 *>(p + j * step));
+    }
+    while (have) {
+      const bool more = t + 32 + 24 < t1i;
+      if (more) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) un[j] = __ldcs(reinterpret_cast<const uint4 *>(p + (4 + j) * step));
+      }
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         float f[8];
@@ -99,10 +112,15 @@ __device__ __forceinline__ void colstat_body(const __nv_bfloat16 *__restrict__ x
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] += (double)f[i], mx[i] = fmaxf(mx[i], f[i]), ng[i] = fmaxf(ng[i], -f[i]);
       }
+      t += 32;
+      p += 4 * step;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) u[j] = un[j];
+      have = more;
     }
-    for (; t < t1; t += 8, p += step) {
+    for (; t < t1i; t += 8, p += step) {
       float f[8];
-      unpack8(*reinterpret_cast<const uint4 *>(p), f);
+      unpack8(__ldcs(reinterpret_cast<const uint4 *>(p)), f);
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[i] += (double)f[i], mx[i] = fmaxf(mx[i], f[i]), ng[i] = fmaxf(ng[i], -f[i]);
     }
@@ -112,80 +130,87 @@ __device__ __forceinline__ void colstat_body(const __nv_bfloat16 *__restrict__ x
   __syncthreads();
   const int c = yg * COLSTAT_COLS + threadIdx.x;
   if (c < cols) {
-    double a = 0.0;
+    double sum = 0.0;
     float m = -INFINITY, g = -INFINITY;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) a += s_sum[j][threadIdx.x], m = fmaxf(m, s_max[j][threadIdx.x]), g = fmaxf(g, s_neg[j][threadIdx.x]);
-    const size_t o = (size_t)b * cols + c;
-    atomicAdd(&sums[o], a);
-    atomicMax(&kmax[o], ordered_key(m));
-    atomicMax(&knegmax[o], ordered_key(g));
+    for (int j = 0; j < 8; ++j) sum += s_sum[j][threadIdx.x], m = fmaxf(m, s_max[j][threadIdx.x]), g = fmaxf(g, s_neg[j][threadIdx.x]);
+    const size_t o = ((size_t)b * a.slices + sl) * cols + c;
+    a.psum[o] = sum;
+    a.pmax[o] = m;
+    a.pneg[o] = g;
   }
-}
-
-__global__ void __launch_bounds__(256) colstat_kernel(const ColTensor a0, const ColTensor a1) {
-  if ((int)blockIdx.y < a0.ygroups)
-    colstat_body(a0.x, a0.N, a0.cols, a0.sums, a0.kmax, a0.knegmax, (int)blockIdx.y);
-  else
-    colstat_body(a1.x, a1.N, a1.cols, a1.sums, a1.kmax, a1.knegmax, (int)blockIdx.y - a0.ygroups);
-}
-
-// Per column: mean = fl(sum / N) (0 without smoothing); per batch element: max |x - mean| from the
-// column extremes.  grid (ceil(cols / 256), B).
-struct FinTensor {
-  const double *sums;   // null: tensor absent
-  const unsigned int *kmax, *knegmax;
-  int cols, N;
-  float *mean;
-  unsigned int *amax;
-  float *gscale;
-};
-
-// grid (ceil(max cols / 256), B, 2): blockIdx.z selects the tensor.
-__global__ void __launch_bounds__(256) finalize_stats_kernel(const FinTensor a0, const FinTensor a1, int smooth) {
-  const bool second = blockIdx.z != 0;
-  const double *__restrict__ sums = second ? a1.sums : a0.sums;
-  if (!sums) return;
-  const unsigned int *__restrict__ kmax = second ? a1.kmax : a0.kmax;
-  const unsigned int *__restrict__ knegmax = second ? a1.knegmax : a0.knegmax;
-  const int cols = second ? a1.cols : a0.cols, N = second ? a1.N : a0.N;
-  float *__restrict__ mean = second ? a1.mean : a0.mean;
-  unsigned int *__restrict__ amax = second ? a1.amax : a0.amax;
-  if ((int)blockIdx.x * 256 >= cols) return;
-  const int b = blockIdx.y, c = blockIdx.x * 256 + threadIdx.x;
+  // ---- the last block of this column group folds the slices
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(group_counter, 1u) == (unsigned int)a.slices - 1u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
   float m = 0.0f;
   if (c < cols) {
-    const size_t o = (size_t)b * cols + c;
-    const float mu = smooth ? __double2float_rn(__ddiv_rn(sums[o], (double)N)) : 0.0f;
-    mean[o] = mu;
-    const float hi = from_ordered_key(kmax[o]), lo = -from_ordered_key(knegmax[o]);
-    m = fmaxf(__fsub_rn(hi, mu), __fsub_rn(mu, lo));   // non-negative: lo <= mu <= hi (or mu = 0 and the larger side wins)
+    double sum = 0.0;
+    float hi = -INFINITY, ng2 = -INFINITY;
+    const size_t o0 = (size_t)b * a.slices * cols + c;
+    for (int s0 = 0; s0 < a.slices; s0 += 4) {   // four slices' loads in flight; the additions stay in slice order
+      double ps[4];
+      float pm[4], pn[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bool in = s0 + j < a.slices;
+        const size_t o = o0 + (size_t)(s0 + j) * cols;
+        ps[j] = in ? __ldcg(a.psum + o) : 0.0;
+        pm[j] = in ? __ldcg(a.pmax + o) : -INFINITY;
+        pn[j] = in ? __ldcg(a.pneg + o) : -INFINITY;
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (s0 + j < a.slices) sum += ps[j];
+        hi = fmaxf(hi, pm[j]);
+        ng2 = fmaxf(ng2, pn[j]);
+      }
+    }
+    const float mu = smooth ? __double2float_rn(__ddiv_rn(sum, (double)N)) : 0.0f;
+    a.mean[(size_t)b * cols + c] = mu;
+    m = fmaxf(__fsub_rn(hi, mu), __fsub_rn(mu, -ng2));   // non-negative: lo <= mu <= hi (or mu = 0 and the larger side wins)
     m = fmaxf(m, 0.0f);
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  __shared__ float wmax[8];
+  float *wmax = &s_max[0][0];
+  __syncthreads();
   if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = m;
   __syncthreads();
   if (threadIdx.x == 0) {
 #pragma unroll
     for (int i = 1; i < 8; ++i) m = fmaxf(m, wmax[i]);
-    atomicMax(&amax[b], __float_as_uint(m));   // non-negative floats order like their bit patterns
+    atomicMax(&a.amax[b], __float_as_uint(m));   // non-negative floats order like their bit patterns
+    __threadfence();
+    s_last = atomicAdd(launch_counter, 1u) == n_groups - 1u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int i = threadIdx.x; i < (int)gridDim.z; i += 256) {
+    if (t0.x) {
+      const float v = __uint_as_float(__ldcg(t0.amax + i));
+      t0.gscale[i] = v > 0.0f ? __fdiv_rn(v, 2688.0f) : 1.0f;
+    }
+    if (t1.x) {
+      const float v = __uint_as_float(__ldcg(t1.amax + i));
+      t1.gscale[i] = v > 0.0f ? __fdiv_rn(v, 2688.0f) : 1.0f;
+    }
   }
 }
 
-__global__ void finalize_scale_kernel(const FinTensor a0, const FinTensor a1, int B) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < B) {
-    if (a0.sums) {
-      float a = __uint_as_float(a0.amax[i]);
-      a0.gscale[i] = a > 0.0f ? __fdiv_rn(a, 2688.0f) : 1.0f;
-    }
-    if (a1.sums) {
-      float a = __uint_as_float(a1.amax[i]);
-      a1.gscale[i] = a > 0.0f ? __fdiv_rn(a, 2688.0f) : 1.0f;
-    }
-  }
+// counters: [B][ygroups of both tensors] group counters, then one launch counter; all zero at launch
+__global__ void __launch_bounds__(256, 3) colstat_kernel(const ColTensor a0, const ColTensor a1, unsigned int *counters, int smooth) {
+  const unsigned int groups = (unsigned int)(a0.ygroups + a1.ygroups);
+  unsigned int *gc = counters + blockIdx.z * groups + blockIdx.y;
+  unsigned int *lc = counters + gridDim.z * groups;
+  if ((int)blockIdx.y < a0.ygroups)
+    colstat_body(a0, (int)blockIdx.y, gc, lc, groups * gridDim.z, smooth, a0, a1);
+  else
+    colstat_body(a1, (int)blockIdx.y - a0.ygroups, gc, lc, groups * gridDim.z, smooth, a0, a1);
 }
 
 // One NVFP4 block (Eq. 1): 16 centered values -> E4M3 scale code + 8 bytes of E2M1 codes.
@@ -230,15 +255,101 @@ struct QuantTensor {
 __device__ __forceinline__ void quantize_tile_body(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ mean,
                                                    const float *__restrict__ gscale, const int N, const int H,
                                                    const int tiles, uint8_t *__restrict__ codes,
-                                                   uint8_t *__restrict__ sf, const int h) {
+                                                   uint8_t *__restrict__ sf, const int h, const int tile) {
   __shared__ float mu[HEAD_DIM];
   __shared__ __align__(16) uint8_t sf_tile[1024];
-  const int tile = blockIdx.x, b = blockIdx.z;
+  const int b = blockIdx.z;
   if (tile >= tiles) return;
   const int n_pad = tiles * TILE;
   if (threadIdx.x < HEAD_DIM) mu[threadIdx.x] = mean[((size_t)b * H + h) * HEAD_DIM + threadIdx.x];
   __syncthreads();
   const float d = gscale[b];
+  // the thread's block index g = threadIdx.x & 7 is the same in all four iterations: its 16 means live in registers
+  // (read from shared memory per block they cost 4-way bank conflicts: the data pipe was the kernel's limiter)
+  float mreg[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) mreg[i] = mu[(threadIdx.x & 7) * 16 + i];
+  // all eight 16-byte loads of the thread's four blocks are issued before the first block is quantized
+  uint4 raw[4][2];
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int id = it * 256 + threadIdx.x;
+    const int r = id >> 3, g = id & 7;
+    const int t = tile * TILE + r;
+    raw[it][0] = raw[it][1] = make_uint4(0u, 0u, 0u, 0u);
+    if (t < N) {
+      const uint4 *src = reinterpret_cast<const uint4 *>(x + (((size_t)b * N + t) * H + h) * HEAD_DIM + g * 16);
+      raw[it][0] = __ldcs(src);
+      raw[it][1] = __ldcs(src + 1);
+    }
+  }
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int id = it * 256 + threadIdx.x;
+    const int r = id >> 3, g = id & 7;
+    const int t = tile * TILE + r;
+    uint2 c = make_uint2(0u, 0u);
+    uint8_t sc = 0;
+    if (t < N) {
+      float xc[16], f[8];
+      unpack8(raw[it][0], f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) xc[i] = __fsub_rn(f[i], mreg[i]);
+      unpack8(raw[it][1], f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) xc[8 + i] = __fsub_rn(f[i], mreg[8 + i]);
+      quantize_block16(xc, d, sc, c);
+    }
+    __stcs(reinterpret_cast<uint2 *>(codes + (((size_t)b * H + h) * n_pad + t) * 64 + g * 8), c);
+    sf_tile[(g >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (g & 3)] = sc;
+  }
+  __syncthreads();
+  uint32_t *dst = reinterpret_cast<uint32_t *>(sf + (((size_t)b * H + h) * tiles + tile) * 1024);
+  dst[threadIdx.x] = reinterpret_cast<const uint32_t *>(sf_tile)[threadIdx.x];
+}
+
+// K tile with the compensation vector (Eq. 9) in the same pass: the tile's rows are staged once in shared memory
+// (coalesced 16-byte loads; a row is 256 contiguous bytes, rows of one head are H_kv * 256 bytes apart; row pitch
+// 272 bytes so that the 16-byte reads of 8 consecutive threads fall into 8 different bank groups), quantized from
+// there exactly like a Q tile, and then every key's Delta_S[hq][t] = qmean[hq] . (k[t] - kmean) is accumulated in
+// FP64 with channels ascending by thread (key, part), part taking the heads g = part, part + 2, ... of the group as
+// independent sequential chains; the result is expressed in units of gscale_q * gscale_k and rounded once to BF16.
+struct DeltaArgs {
+  const float *q_mean;     // null: no Delta_S (direct variant or statistics-only call)
+  const float *q_gscale;
+  __nv_bfloat16 *delta;    // [B, H_q, N_pad]
+  int H_q;
+};
+
+constexpr int KROW_PITCH = 272;
+constexpr int KTILE_SMEM = TILE * KROW_PITCH + 8 * HEAD_DIM * 8;   // staged rows + FP64 query means of the group
+
+__device__ __forceinline__ void quantize_k_tile_delta_body(const QuantTensor &a, const DeltaArgs &da, const int h,
+                                                           const int tile, uint8_t *dyn) {
+  constexpr int MAXG = 8;
+  __shared__ float mu[HEAD_DIM];
+  __shared__ __align__(16) uint8_t sf_tile[1024];
+  uint8_t *rows = dyn;
+  double(*qmu)[HEAD_DIM] = reinterpret_cast<double(*)[HEAD_DIM]>(dyn + TILE * KROW_PITCH);
+  const int b = blockIdx.z;
+  if (tile >= a.tiles) return;
+  const int N = a.N, H = a.H, n_pad = a.tiles * TILE;
+  const int G = da.H_q / H;
+  if (threadIdx.x < HEAD_DIM) mu[threadIdx.x] = a.mean[((size_t)b * H + h) * HEAD_DIM + threadIdx.x];
+  for (int j = threadIdx.x; j < G * HEAD_DIM; j += 256)
+    qmu[j >> 7][j & 127] = (double)da.q_mean[((size_t)b * da.H_q + h * G + (j >> 7)) * HEAD_DIM + (j & 127)];
+  for (int i = threadIdx.x; i < TILE * 16; i += 256) {
+    const int r = i >> 4, ch = i & 15;
+    const int tt = tile * TILE + r;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (tt < N) v = __ldcs(reinterpret_cast<const uint4 *>(a.x + (((size_t)b * N + tt) * H + h) * HEAD_DIM + ch * 8));
+    *reinterpret_cast<uint4 *>(rows + r * KROW_PITCH + ch * 16) = v;
+  }
+  __syncthreads();
+  const float d = a.gscale[b];
+  float mreg[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) mreg[i] = mu[(threadIdx.x & 7) * 16 + i];
 #pragma unroll
   for (int it = 0; it < 4; ++it) {
     const int id = it * 256 + threadIdx.x;
@@ -248,23 +359,78 @@ __device__ __forceinline__ void quantize_tile_body(const __nv_bfloat16 *__restri
     uint8_t sc = 0;
     if (t < N) {
       float xc[16];
-      load_center16(x + (((size_t)b * N + t) * H + h) * HEAD_DIM + g * 16, mu + g * 16, xc);
+      load_center16(reinterpret_cast<const __nv_bfloat16 *>(rows + r * KROW_PITCH + g * 32), mreg, xc);
       quantize_block16(xc, d, sc, c);
     }
-    *reinterpret_cast<uint2 *>(codes + (((size_t)b * H + h) * n_pad + t) * 64 + g * 8) = c;
+    *reinterpret_cast<uint2 *>(a.codes + (((size_t)b * H + h) * n_pad + t) * 64 + g * 8) = c;
     sf_tile[(g >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (g & 3)] = sc;
   }
+  // Delta_S.  The FP64 pipe is the scarce unit here (measured: an eighth of the FP32 rate on this GPU); two threads
+  // per key, each with the chains of every other head of the group, keep enough independent chains in flight to
+  // cover its latency.
+  {
+    const int key = threadIdx.x & 127, part = threadIdx.x >> 7;
+    const int t = tile * TILE + key;
+    double acc[MAXG / 2];
+#pragma unroll
+    for (int u = 0; u < MAXG / 2; ++u) acc[u] = 0.0;
+    if (t < N) {
+      const uint8_t *row = rows + key * KROW_PITCH;
+      for (int c0 = 0; c0 < HEAD_DIM; c0 += 8) {
+        float f[8];
+        unpack8(*reinterpret_cast<const uint4 *>(row + c0 * 2), f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const double kc = (double)__fsub_rn(f[i], mu[c0 + i]);
+#pragma unroll
+          for (int u = 0; u < MAXG / 2; ++u)
+            if (2 * u + part < G) acc[u] = fma(qmu[2 * u + part][c0 + i], kc, acc[u]);
+        }
+      }
+    }
+    const double denom = (double)da.q_gscale[b] * (double)d;
+#pragma unroll
+    for (int u = 0; u < MAXG / 2; ++u) {
+      const int g = 2 * u + part;
+      if (g < G) {
+        const float v = (t < N) ? __double2float_rn(__ddiv_rn(acc[u], denom)) : 0.0f;
+        da.delta[((size_t)b * da.H_q + h * G + g) * n_pad + t] = __float2bfloat16_rn(v);
+      }
+    }
+  }
   __syncthreads();
-  uint32_t *dst = reinterpret_cast<uint32_t *>(sf + (((size_t)b * H + h) * tiles + tile) * 1024);
+  uint32_t *dst = reinterpret_cast<uint32_t *>(a.sf + (((size_t)b * H + h) * a.tiles + tile) * 1024);
   dst[threadIdx.x] = reinterpret_cast<const uint32_t *>(sf_tile)[threadIdx.x];
 }
 
-// grid (max tiles, H of the first + H of the second tensor, B); one 128-token tile of one head per block.
+// grid (max tiles * (H of the first + H of the second tensor), 1, B); one 128-token tile of one head per block,
+// blockIdx.x = tile * heads + head: the head index runs fastest, so the blocks resident at any time read whole token
+// rows of the [B, N, H, 128] input (contiguous DRAM) instead of 256-byte pieces 256 * H bytes apart.
 __global__ void __launch_bounds__(256) quantize_fp4_tile_kernel(const QuantTensor a0, const QuantTensor a1) {
-  if ((int)blockIdx.y < a0.H)
-    quantize_tile_body(a0.x, a0.mean, a0.gscale, a0.N, a0.H, a0.tiles, a0.codes, a0.sf, (int)blockIdx.y);
+  const int heads = a0.H + a1.H;
+  const int tile = (int)blockIdx.x / heads, y = (int)blockIdx.x % heads;
+  if (y < a0.H)
+    quantize_tile_body(a0.x, a0.mean, a0.gscale, a0.N, a0.H, a0.tiles, a0.codes, a0.sf, y, tile);
   else
-    quantize_tile_body(a1.x, a1.mean, a1.gscale, a1.N, a1.H, a1.tiles, a1.codes, a1.sf, (int)blockIdx.y - a0.H);
+    quantize_tile_body(a1.x, a1.mean, a1.gscale, a1.N, a1.H, a1.tiles, a1.codes, a1.sf, y - a0.H, tile);
+}
+
+// grid (tiles * (H_kv + H_q), 1, B), KTILE_SMEM bytes of dynamic shared memory: K tiles with Delta_S and, when
+// aq.H > 0, the Q tiles in the same launch (same block order: tile-major, K head of a group then its G query heads).
+__global__ void __launch_bounds__(256) quantize_k_delta_kernel(const QuantTensor a, const DeltaArgs da, const QuantTensor aq) {
+  extern __shared__ __align__(16) uint8_t dyn_smem[];
+  const int heads = a.H + aq.H;
+  const int tile = (int)blockIdx.x / heads, y = (int)blockIdx.x % heads;
+  if (aq.H == 0) {
+    quantize_k_tile_delta_body(a, da, y, tile, dyn_smem);
+    return;
+  }
+  const int G = aq.H / a.H;
+  const int grp = y / (G + 1), r = y % (G + 1);
+  if (r == 0)
+    quantize_k_tile_delta_body(a, da, grp, tile, dyn_smem);
+  else
+    quantize_tile_body(aq.x, aq.mean, aq.gscale, aq.N, aq.H, aq.tiles, aq.codes, aq.sf, grp * G + r - 1, tile);
 }
 
 // Eq. 9: Delta_S[hq][t] = qmean[hq] . (k[t] - kmean), FP64 accumulation with channels ascending,
@@ -516,33 +682,49 @@ __global__ void __launch_bounds__(256) append_kv_kernel(const __nv_bfloat16 *__r
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
+// Workspace of the statistics pass: for each tensor S slices of per-column partial results (FP64 sum, maximum,
+// maximum of the negated values), then the per-batch-element maxima and one counter word.  S is the largest
+// slice count <= STAT_MAX_SLICES that fits the bytes the caller gave (at least 1).
 struct StatsWorkspace {
-  double *sums_q, *sums_k;
-  unsigned int *max_q, *neg_q, *max_k, *neg_k;   // per-column extremes as ordered keys
-  unsigned int *amax_q, *amax_k;
+  double *psum_q, *psum_k;
+  float *pmax_q, *pneg_q, *pmax_k, *pneg_k;
+  unsigned int *amax_q, *amax_k, *counter;
+  uint8_t *fixed;
+  size_t fixed_bytes;
+  int slices;
   size_t bytes;
 };
 
-StatsWorkspace carve(void *ws, int B, int H_q, int H_kv) {
-  StatsWorkspace w;
+// amax words of both tensors, a counter per (batch element, 256-column group) and the launch counter
+size_t stats_fixed_bytes(int B, int H_q, int H_kv) {
+  return align256(((size_t)2 * B + (size_t)B * ((H_q + 1) / 2 + (H_kv + 1) / 2) + 1) * sizeof(unsigned int));
+}
+size_t stats_slice_bytes(int B, int H_q, int H_kv) {   // one slice of both tensors
+  return align256((size_t)B * H_q * HEAD_DIM * 8) + 2 * align256((size_t)B * H_q * HEAD_DIM * 4) +
+         align256((size_t)B * H_kv * HEAD_DIM * 8) + 2 * align256((size_t)B * H_kv * HEAD_DIM * 4);
+}
+
+StatsWorkspace carve(void *ws, size_t ws_bytes, int B, int H_q, int H_kv) {
+  StatsWorkspace w{};
+  const size_t fixed = stats_fixed_bytes(B, H_q, H_kv), per = stats_slice_bytes(B, H_q, H_kv);
+  size_t S = ws_bytes > fixed ? (ws_bytes - fixed) / per : 0;
+  if (S > (size_t)STAT_MAX_SLICES) S = STAT_MAX_SLICES;
+  w.slices = (int)S;
   size_t o = 0;
   uint8_t *base = static_cast<uint8_t *>(ws);
-  w.sums_q = reinterpret_cast<double *>(base + o);
-  o += align256((size_t)B * H_q * HEAD_DIM * sizeof(double));
-  w.sums_k = reinterpret_cast<double *>(base + o);
-  o += align256((size_t)B * H_kv * HEAD_DIM * sizeof(double));
-  w.max_q = reinterpret_cast<unsigned int *>(base + o);
-  o += align256((size_t)B * H_q * HEAD_DIM * sizeof(unsigned int));
-  w.neg_q = reinterpret_cast<unsigned int *>(base + o);
-  o += align256((size_t)B * H_q * HEAD_DIM * sizeof(unsigned int));
-  w.max_k = reinterpret_cast<unsigned int *>(base + o);
-  o += align256((size_t)B * H_kv * HEAD_DIM * sizeof(unsigned int));
-  w.neg_k = reinterpret_cast<unsigned int *>(base + o);
-  o += align256((size_t)B * H_kv * HEAD_DIM * sizeof(unsigned int));
+  const size_t nq = (size_t)B * H_q * HEAD_DIM, nk = (size_t)B * H_kv * HEAD_DIM;
+  w.psum_q = reinterpret_cast<double *>(base + o);  o += S * align256(nq * 8);
+  w.psum_k = reinterpret_cast<double *>(base + o);  o += S * align256(nk * 8);
+  w.pmax_q = reinterpret_cast<float *>(base + o);   o += S * align256(nq * 4);
+  w.pneg_q = reinterpret_cast<float *>(base + o);   o += S * align256(nq * 4);
+  w.pmax_k = reinterpret_cast<float *>(base + o);   o += S * align256(nk * 4);
+  w.pneg_k = reinterpret_cast<float *>(base + o);   o += S * align256(nk * 4);
+  w.fixed = base + o;                                      // zeroed before every statistics launch
+  w.fixed_bytes = fixed;
   w.amax_q = reinterpret_cast<unsigned int *>(base + o);
-  o += align256((size_t)B * sizeof(unsigned int));
-  w.amax_k = reinterpret_cast<unsigned int *>(base + o);
-  o += align256((size_t)B * sizeof(unsigned int));
+  w.amax_k = w.amax_q + B;
+  w.counter = w.amax_k + B;
+  o += fixed;
   w.bytes = o;
   return w;
 }
@@ -551,33 +733,41 @@ StatsWorkspace carve(void *ws, int B, int H_q, int H_kv) {
 struct StatsJob {
   const __nv_bfloat16 *x;
   int N, H;
-  double *sums;
-  unsigned int *kmax, *knegmax, *amax;
+  double *psum;
+  float *pmax, *pneg;
+  unsigned int *amax;
   float *mean, *gscale;
 };
 
-// Means and per-tensor scales of up to two tensors: one pass over the data, three launches in all.
-mpfa_status tensor_stats(const StatsJob &j0, const StatsJob &j1, int B, bool smooth, cudaStream_t st) {
+// Means and per-tensor scales of up to two tensors: one pass over the data, one memory-set node (the amax words
+// and counters) and one launch.
+mpfa_status tensor_stats(const StatsJob &j0, const StatsJob &j1, int B, const StatsWorkspace &w, bool smooth, cudaStream_t st) {
   ColTensor c[2];
-  FinTensor f[2];
-  int tiles = 0, colgroups = 0;
+  int slices_x = 0;
   const StatsJob *jobs[2] = {&j0, &j1};
+  // as many slices as keep the whole launch resident at once (three 256-thread blocks per SM), within what the
+  // workspace holds
+  int dev = 0, n_sm = 0;
+  MPFA_CUDA_OK(cudaGetDevice(&dev));
+  MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  int groups = 0;
+  for (int i = 0; i < 2; ++i)
+    if (jobs[i]->x) groups += (jobs[i]->H * HEAD_DIM + COLSTAT_COLS - 1) / COLSTAT_COLS;
+  if (groups == 0) return MPFA_OK;
+  const int max_slices = std::min(w.slices, std::max(1, 3 * n_sm / (groups * B)));
   for (int i = 0; i < 2; ++i) {
     const StatsJob &j = *jobs[i];
     const int cols = j.H * HEAD_DIM;
-    c[i] = ColTensor{j.x, j.x ? j.N : 0, cols, j.x ? (cols + COLSTAT_COLS - 1) / COLSTAT_COLS : 0, j.sums, j.kmax, j.knegmax};
-    f[i] = FinTensor{j.x ? j.sums : nullptr, j.kmax, j.knegmax, cols, j.N, j.mean, j.amax, j.gscale};
-    if (j.x) {
-      tiles = std::max(tiles, (j.N + COLSTAT_TOKENS - 1) / COLSTAT_TOKENS);
-      colgroups = std::max(colgroups, (cols + 255) / 256);
-    }
+    // slices of at least 256 tokens, a multiple of 8 tokens long (the eight token lanes of a CTA)
+    int S = j.x ? std::min(max_slices, std::max(1, (j.N + 255) / 256)) : 0;
+    const int len = j.x ? ((j.N + S - 1) / S + 7) / 8 * 8 : 0;
+    if (j.x) S = (j.N + len - 1) / len;
+    c[i] = ColTensor{j.x, j.x ? j.N : 0, cols, j.x ? (cols + COLSTAT_COLS - 1) / COLSTAT_COLS : 0, S, len, j.psum, j.pmax,
+                     j.pneg, j.amax, j.mean, j.gscale};
+    if (j.x) slices_x = std::max(slices_x, S);
   }
-  if (c[0].ygroups + c[1].ygroups == 0) return MPFA_OK;
-  colstat_kernel<<<dim3(tiles, c[0].ygroups + c[1].ygroups, B), 256, 0, st>>>(c[0], c[1]);
-  MPFA_LAUNCH_OK();
-  finalize_stats_kernel<<<dim3(colgroups, B, 2), 256, 0, st>>>(f[0], f[1], smooth ? 1 : 0);
-  MPFA_LAUNCH_OK();
-  finalize_scale_kernel<<<(B + 127) / 128, 128, 0, st>>>(f[0], f[1], B);
+  MPFA_CUDA_OK(cudaMemsetAsync(w.fixed, 0, w.fixed_bytes, st));
+  colstat_kernel<<<dim3(slices_x, c[0].ygroups + c[1].ygroups, B), 256, 0, st>>>(c[0], c[1], w.counter, smooth ? 1 : 0);
   MPFA_LAUNCH_OK();
   return MPFA_OK;
 }
@@ -589,7 +779,12 @@ using namespace mpfa;
 
 extern "C" size_t mpfa_quantize_workspace_bytes(int B, int H_q, int H_kv) {
   if (B <= 0 || H_q <= 0 || H_kv <= 0) return 0;
-  return carve(nullptr, B, H_q, H_kv).bytes;
+  return stats_fixed_bytes(B, H_q, H_kv) + (size_t)STAT_MAX_SLICES * stats_slice_bytes(B, H_q, H_kv);
+}
+
+extern "C" size_t mpfa_quantize_workspace_min_bytes(int B, int H_q, int H_kv) {
+  if (B <= 0 || H_q <= 0 || H_kv <= 0) return 0;
+  return stats_fixed_bytes(B, H_q, H_kv) + stats_slice_bytes(B, H_q, H_kv);
 }
 
 extern "C" mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, int B, int N_q, int N_kv, int H_q,
@@ -615,8 +810,8 @@ extern "C" mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, 
   if (!frozen) {
     if (!workspace) return MPFA_ERR_INVALID_ARG;
     if (!aligned(workspace, 256)) return MPFA_ERR_ALIGNMENT;
-    w = carve(workspace, B, H_q, H_kv);
-    if (workspace_bytes < w.bytes) return MPFA_ERR_WORKSPACE;
+    w = carve(workspace, workspace_bytes, B, H_q, H_kv);
+    if (w.slices < 1) return MPFA_ERR_WORKSPACE;
   }
   mpfa_status rc = check_arch();
   if (rc != MPFA_OK) return rc;
@@ -624,9 +819,8 @@ extern "C" mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, 
   const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(q_bf16);
   const __nv_bfloat16 *k = static_cast<const __nv_bfloat16 *>(k_bf16);
   if (!frozen) {
-    MPFA_CUDA_OK(cudaMemsetAsync(workspace, 0, w.bytes, s));
-    rc = tensor_stats(StatsJob{q, N_q, H_q, w.sums_q, w.max_q, w.neg_q, w.amax_q, st->q_mean, st->q_gscale},
-                      StatsJob{k, N_kv, H_kv, w.sums_k, w.max_k, w.neg_k, w.amax_k, st->k_mean, st->k_gscale}, B, smooth, s);
+    rc = tensor_stats(StatsJob{q, N_q, H_q, w.psum_q, w.pmax_q, w.pneg_q, w.amax_q, st->q_mean, st->q_gscale},
+                      StatsJob{k, N_kv, H_kv, w.psum_k, w.pmax_k, w.pneg_k, w.amax_k, st->k_mean, st->k_gscale}, B, w, smooth, s);
     if (rc != MPFA_OK) return rc;
   }
   {
@@ -635,14 +829,23 @@ extern "C" mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, 
                    q ? q_out->sf : nullptr};
     QuantTensor tk{k, st->k_mean, st->k_gscale, N_kv, k ? H_kv : 0, k ? pad128(N_kv) / TILE : 0,
                    k ? k_out->codes : nullptr, k ? k_out->sf : nullptr};
-    quantize_fp4_tile_kernel<<<dim3(std::max(tq.tiles, tk.tiles), tq.H + tk.H, B), 256, 0, s>>>(tq, tk);
-    MPFA_LAUNCH_OK();
-  }
-  if (k) {
-    dim3 grid(pad128(N_kv) / TILE, H_kv, B);
-    if (smooth) {
-      delta_s_kernel<false><<<grid, 256, 0, s>>>(k, st->q_mean, st->k_mean, st->q_gscale, st->k_gscale, N_kv, H_q,
-                                                 H_kv, static_cast<__nv_bfloat16 *>(delta_s_bf16), nullptr, 0);
+    // with smoothing the K tiles also produce Delta_S (Eq. 9) from the rows they have staged (no third pass over
+    // K), in a launch of their own
+    const bool with_delta = k && smooth;
+    if (with_delta) {
+      DeltaArgs da{st->q_mean, st->q_gscale, static_cast<__nv_bfloat16 *>(delta_s_bf16), H_q};
+      MPFA_CUDA_OK(cudaFuncSetAttribute(quantize_k_delta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KTILE_SMEM));
+      const bool both = false;      // measured: in one launch the two kinds only compete for block slots (98 us against 40 + 37)
+      QuantTensor none{};
+      quantize_k_delta_kernel<<<dim3(std::max(tk.tiles, both ? tq.tiles : 0) * (tk.H + (both ? tq.H : 0)), 1, B), 256, KTILE_SMEM,
+                                s>>>(tk, da, both ? tq : none);
+      MPFA_LAUNCH_OK();
+      tk.H = 0;
+      tk.tiles = 0;
+      if (both) tq.H = 0, tq.tiles = 0;
+    }
+    if (tq.H + tk.H > 0) {
+      quantize_fp4_tile_kernel<<<dim3(std::max(tq.tiles, tk.tiles) * (tq.H + tk.H), 1, B), 256, 0, s>>>(tq, tk);
       MPFA_LAUNCH_OK();
     }
   }
@@ -683,8 +886,8 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
   if (!frozen) {
     if (!workspace) return MPFA_ERR_INVALID_ARG;
     if (!aligned(workspace, 256)) return MPFA_ERR_ALIGNMENT;
-    w = carve(workspace, 1, H_q, H_kv);
-    if (workspace_bytes < w.bytes) return MPFA_ERR_WORKSPACE;
+    w = carve(workspace, workspace_bytes, 1, H_q, H_kv);
+    if (w.slices < 1) return MPFA_ERR_WORKSPACE;
   }
   mpfa_status rc = check_arch();
   if (rc != MPFA_OK) return rc;
@@ -692,9 +895,8 @@ extern "C" mpfa_status mpfa_quantize_kv_paged(const void *k_bf16, const void *v_
   const __nv_bfloat16 *k = static_cast<const __nv_bfloat16 *>(k_bf16);
   const __nv_bfloat16 *v = static_cast<const __nv_bfloat16 *>(v_bf16);
   if (!frozen) {
-    MPFA_CUDA_OK(cudaMemsetAsync(workspace, 0, w.bytes, s));
-    rc = tensor_stats(StatsJob{k, N_tokens, H_kv, w.sums_k, w.max_k, w.neg_k, w.amax_k, st->k_mean, st->k_gscale},
-                      StatsJob{nullptr, 0, 0, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr}, 1, smooth, s);
+    rc = tensor_stats(StatsJob{k, N_tokens, H_kv, w.psum_k, w.pmax_k, w.pneg_k, w.amax_k, st->k_mean, st->k_gscale},
+                      StatsJob{nullptr, 0, 0, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr}, 1, w, smooth, s);
     if (rc != MPFA_OK) return rc;
   }
   if (first_token % PAGE != 0) {
@@ -792,7 +994,7 @@ extern "C" mpfa_status mpfa_quantize_qk_static(const void *q_bf16, const void *k
   if (flags & MPFA_STATS_FROZEN)
     return mpfa_quantize_qk(q_bf16, k_bf16, B, N_q, N_kv, H_q, H_kv, flags, st, q_out, k_out, delta_s_bf16, nullptr, 0,
                             stream);
-  if (carve(nullptr, B, H_q, H_kv).bytes > STATIC_SCRATCH_BYTES) return MPFA_ERR_WORKSPACE;
+  if (stats_fixed_bytes(B, H_q, H_kv) + stats_slice_bytes(B, H_q, H_kv) > STATIC_SCRATCH_BYTES) return MPFA_ERR_WORKSPACE;
   void *scratch = nullptr;
   mpfa_status rc = static_scratch_address(&scratch);
   if (rc != MPFA_OK) return rc;

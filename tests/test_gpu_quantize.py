@@ -138,3 +138,48 @@ def test_stage1_bit_exact_on_adversarial_values(kind):
     w = _adversarial(kind, 400 + len(kind))
     z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
     check_stage1(w, run_stage1_gpu(w), z)
+
+
+def test_means_are_deterministic_on_unflushed_inputs():
+    """Eq. 7 on inputs the seeded generator never produces: magnitudes from 2^-60 up to O(1) mixed in every column,
+    so the FP64 column sums are no longer exact and their value depends on the order of addition.  The kernels add
+    in a fixed order (no floating-point atomics): two runs must agree bit for bit in every output, and the means
+    must be within one FP32 ulp of the oracle's single ascending sum."""
+    from paper_2609_33135_b200 import binding
+    g = torch.Generator(device="cpu").manual_seed(77)
+    B, N, Hq, Hkv = 2, 3000, 4, 2
+    def draw(H):
+        x = torch.randn(B, N, H, 128, generator=g)
+        e = torch.randint(-60, 1, (B, N, H, 128), generator=g).float()
+        return (x * torch.exp2(e)).to(torch.bfloat16)
+    q, k, v = draw(Hq), draw(Hkv), draw(Hkv)
+    assert float(q.float().abs()[q.float().abs() > 0].min()) < 2.0 ** -55
+    runs = []
+    for _ in range(2):
+        s1 = binding.stage1(q.cuda(), k.cuda(), v.cuda())
+        torch.cuda.synchronize()
+        runs.append([t.clone() for t in (s1.stats.q_mean, s1.stats.k_mean, s1.stats.q_gscale, s1.stats.k_gscale, s1.q.codes,
+                                         s1.q.sf, s1.k.codes, s1.k.sf, s1.delta.view(torch.uint16))])
+    for a, b in zip(*runs):
+        assert torch.equal(a, b)
+    for got, x in ((runs[0][0], q), (runs[0][1], k)):
+        ref = orc.means(orc.bf16_bits(x))
+        got = got.cpu().numpy()
+        ulp = np.spacing(np.abs(ref).astype(np.float32))
+        assert np.all(np.abs(got.astype(np.float64) - ref.astype(np.float64)) <= ulp)
+        assert (got == ref).mean() > 0.99
+
+
+def test_stage1_with_a_one_slice_workspace_is_the_same_on_exact_inputs():
+    """The statistics pass takes as many token slices as the workspace holds; on the generator's inputs (exact
+    sums) the slice count cannot change a bit."""
+    from paper_2609_33135_b200 import binding
+    w = wl.prefill_workload("ws", 43, 1, 2500, 4, 2, True, q_bias=True)
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+    n_min = binding.lib().mpfa_quantize_workspace_min_bytes(1, 4, 2)
+    assert n_min < binding.lib().mpfa_quantize_workspace_bytes(1, 4, 2)
+    for nbytes in (n_min, 3 * n_min):
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        check_stage1(w, binding.stage1(w.q.cuda(), w.k.cuda(), w.v.cuda(), workspace=ws), z)
+    with pytest.raises(binding.MpfaError, match="workspace"):
+        binding.stage1(w.q.cuda(), w.k.cuda(), w.v.cuda(), workspace=torch.empty(n_min - 256, dtype=torch.uint8, device="cuda"))

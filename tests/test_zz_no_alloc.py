@@ -55,7 +55,7 @@ def test_static_scratch_rejects_oversized_shapes():
     from paper_2609_33135_b200 import binding
     limit = binding.lib().mpfa_static_scratch_bytes()
     B, Hq, Hkv = 16, 40, 8
-    assert binding.lib().mpfa_quantize_workspace_bytes(B, Hq, Hkv) > limit
+    assert binding.lib().mpfa_quantize_workspace_min_bytes(B, Hq, Hkv) > limit
     q = torch.zeros(B, 4, Hq, 128, dtype=torch.bfloat16, device="cuda")
     st = binding.Stats.empty(B, Hq, Hkv)
     q4 = binding.Fp4Tensor.empty(B, Hq, 4)
@@ -70,7 +70,7 @@ def test_static_scratch_frozen_statistics_have_no_size_limit_and_nothing_is_allo
     device allocator's books and the driver's free-memory figure do not move."""
     from paper_2609_33135_b200 import binding
     B, Hq, Hkv = 32, 32, 8
-    assert binding.lib().mpfa_quantize_workspace_bytes(B, Hq, Hkv) > binding.lib().mpfa_static_scratch_bytes()
+    assert binding.lib().mpfa_quantize_workspace_min_bytes(B, Hq, Hkv) > binding.lib().mpfa_static_scratch_bytes()
     g = torch.Generator(device="cpu").manual_seed(5)
     q = torch.randn(B, 1, Hq, 128, generator=g).to(torch.bfloat16).cuda()
     st = binding.Stats.empty(B, Hq, Hkv)
