@@ -33,11 +33,13 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 METRIC = "QK4PV8 prefill TFLOPS @16K-128K; decode KV GB/s vs HBM peak"
-KERNELS_PER_STEP = 7  # column statistics, mean+amax, scale, fp4 quantize (each one launch for Q and K), Delta_S, V quantize, prefill
+KERNELS_PER_STEP = 5  # column statistics (Q and K in one launch), K quantize + Delta_S, Q quantize, V quantize, prefill
 # Nominal dense tensor rates relative to BF16: FP4 4x, FP8 2x.  Per (query, key) pair the path does
 # 2d FP4 FLOP and 2d FP8 FLOP, so F attention FLOPs take (F/2)/(4P) + (F/2)/(2P) = 3F/(8P): the
 # mixed-precision bound in attention FLOP/s is 8/3 of the BF16 peak P.
 MIXED_OVER_BF16 = 8.0 / 3.0
+NOMINAL_MIXED_TFLOPS = 6000.0   # the same bound from the nominal dense peaks (9 PF/s FP4, 4.5 PF/s FP8)
+NOMINAL_HBM_GBS = 8000.0        # nominal HBM3e bandwidth the decode figure is also stated against
 KV_BYTES_PER_TOKEN_HEAD = 64 + 8 + 128 + 2 * 4  # K codes, K scales, V, Delta_S for a 4-head GQA group
 
 
@@ -147,8 +149,10 @@ def rank_seed(base_seed: int, rank: int) -> int:
 
 # ------------------------------------------------------------------------------------------
 def cpu_oracle_sample(w, steps: int, rows_per_head: int):
-    """The oracle, as it stands, on a bounded sample of the prefill workload: stage 1 on the full
-    tensors once, then `rows_per_head` evenly spaced query rows of every head against all their keys."""
+    """The oracle, as it stands, on a bounded sample of the prefill workload: stage 1 on the full tensors, then
+    `rows_per_head` evenly spaced query rows of every head against all their keys; the two parts are timed
+    separately so that the attention rate does not depend on how many rows share one stage-1 pass.
+    Returns (attention FLOPs of the sample, [(stage-1 seconds, attention seconds)] per step, description)."""
     from oracle import mpfa_oracle as orc
     import numpy as np
     q, k, v = orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v)
@@ -158,14 +162,22 @@ def cpu_oracle_sample(w, steps: int, rows_per_head: int):
                      np.tile(idx, w.H_q)], axis=1)
     pairs = float((idx.astype(np.int64) + 1 + (w.N_kv - w.N_q)).clip(0, w.N_kv).sum() * w.H_q)
     times = []
-    z = None
     for _ in range(steps):
         t0 = time.perf_counter()
         z = orc.stage1(q, k, v)
+        t1 = time.perf_counter()
         orc.prefill_rows(z, rows, w.softmax_scale, w.causal)
-        times.append(time.perf_counter() - t0)
-    return pairs * 4 * 128, times, f"stage 1 on the full tensors + {len(rows)} (head, query row) pairs " \
-                                  f"(every {stride}th row of each head) against all their keys"
+        times.append((t1 - t0, time.perf_counter() - t1))
+    return pairs * 4 * 128, times, f"{len(rows)} (head, query row) pairs (every {stride}th row of each head) against all " \
+                                  f"their keys; stage 1 on the full tensors timed separately"
+
+
+def cpu_baseline_record(flops, times, sample, cores):
+    """value = attention FLOPs of the sample / attention seconds (stage 1 excluded, as the kernel figures are)."""
+    s1 = sum(t[0] for t in times) / len(times)
+    att = sum(t[1] for t in times) / len(times)
+    return {"value": flops / att / 1e12, "unit": "TFLOPS", "cores": cores, "kind": "oracle", "sample": sample,
+            "attention_seconds": att, "seconds_per_query_key_pair": att / (flops / 512.0), "stage1_seconds_full_tensors": s1}
 
 
 def run_reference(args, rank):
@@ -175,16 +187,17 @@ def run_reference(args, rank):
     from paper_2609_33135_b200 import workloads as wl
     w = wl.config2_llama()
     cores = os.cpu_count() or 1
-    flops, times, sample = cpu_oracle_sample(w, args.warmup + args.steps, rows_per_head=256)
+    flops, times, sample = cpu_oracle_sample(w, args.warmup + args.steps, rows_per_head=args.ref_rows_per_head)
     times = times[args.warmup:]
-    ms = 1e3 * sum(times) / len(times)
-    val = flops / (ms * 1e-3) / 1e12
+    rec = cpu_baseline_record(flops, times, sample, cores)
+    ms = 1e3 * rec["attention_seconds"]
+    val = rec["value"]
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOPS", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "nvfp4/fp8 emulated in f32", "data": "synthetic",
-        "config": {"workload": w.name, "B": 1, "H_q": 32, "H_kv": 8, "head_dim": 128, "N": w.N_q, "causal": True},
-        "cpu_baseline": {"value": val, "unit": "TFLOPS", "cores": cores, "kind": "oracle", "sample": sample},
+        "config": {"workload": w.name, "B_per_gpu": 1, "H_q": 32, "H_kv": 8, "head_dim": 128, "N": w.N_q, "causal": True},
+        "cpu_baseline": rec,
         "e2e": {"value": val, "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
 
@@ -311,6 +324,92 @@ def bench_compensation_overhead(binding, s1, w, reps=5):
             "status": int(status.item())}
 
 
+def bench_mma_peaks(binding, dev):
+    """Tensor-core rates of this GPU for the three MMA kinds of the path (M = 128, N = 128, operands resident in
+    shared / tensor memory, one CTA per SM, a few milliseconds each, best of three): the measured counterpart of
+    the nominal 4x / 2x ratios.  The mixed bound takes equal FP4 and FP8 FLOPs per (query, key) pair."""
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    out = {}
+    for name, kind, iters in (("bf16_ss", 0, 20000), ("e4m3_ts", 2, 20000), ("nvfp4_ss", 3, 10000)):
+        best = 0.0
+        for _ in range(3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            flops = binding.mpfa_bench_mma_peak(kind, 128, iters, status)
+            b.record()
+            torch.cuda.synchronize()
+            best = max(best, flops / (a.elapsed_time(b) * 1e-3) / 1e12)
+        out[name] = best
+    out["mixed_fp4_fp8"] = 1.0 / (0.5 / out["nvfp4_ss"] + 0.5 / out["e4m3_ts"])
+    out["unit"] = "TFLOP/s"
+    out["status"] = int(status.item())
+    out["how"] = "mpfa_bench_mma_peak: back-to-back tcgen05.mma, M=128 N=128, CUDA events, best of 3 bursts"
+    return out
+
+
+def time_calls(fn, steps, warmup):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in evs]
+    return sum(ms) / len(ms), min(ms)
+
+
+def stage1_bytes(w):
+    """Algorithmic HBM bytes of stage 1: two passes over Q and K (statistics, quantize; Delta_S comes out of the K
+    quantize pass), packed codes + scales written (0.5625 B per element), Delta_S written, V read and written."""
+    nq, nk = w.q.numel(), w.k.numel()
+    return (2 * 2 + 0.5625) * (nq + nk) + 2.0 * w.B * w.N_kv * w.H_q + 3 * w.v.numel()
+
+
+def bench_prefill_config(binding, wl, name, seed, N, H_q, peaks, mma, local, with_compensation):
+    """One more prefill length of the metric (configs 3 and 4), inputs drawn on the device: attention kernel alone,
+    the whole step with stage 1, stage-1 GB/s, fractions of the bounds, clocks sampled during the timed steps."""
+    dev = torch.device("cuda", local)
+    w = wl.prefill_workload(name, seed, 1, N, H_q, 8, True, device=str(dev))
+    s1 = binding.stage1(w.q, w.k, w.v)
+    ws = binding.quantize_workspace(1, H_q, 8, dev)
+    out = torch.empty(1, N, H_q, 128, dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    steps = 5 if N <= 65536 else 3
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.2)
+    t0 = time.time()
+    k_ms, k_min = time_calls(lambda: binding.prefill(s1, True, w.softmax_scale, out=out, status=status), steps, 3)
+    q_ms, _ = time_calls(lambda: binding.stage1(w.q, w.k, w.v, workspace=ws, out=s1), steps, 2)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    tf = w.flops / (k_ms * 1e-3) / 1e12
+    rec = {"workload": w.name, "H_q": H_q, "H_kv": 8, "N": N, "kernel_ms": k_ms, "kernel_ms_min": k_min,
+           "prefill_kernel_tflops": tf, "step_tflops": w.flops / ((k_ms + q_ms) * 1e-3) / 1e12,
+           "frac_of_mixed_bound_from_bf16_peak": tf / (peaks["bf16"] * MIXED_OVER_BF16),
+           "frac_of_mixed_bound_from_measured_mma": tf / mma["mixed_fp4_fp8"] if mma else None,
+           "frac_of_nominal_mixed_bound": tf / NOMINAL_MIXED_TFLOPS,
+           "stage1_ms": q_ms, "stage1_gbs": stage1_bytes(w) / (q_ms * 1e-3) / 1e9,
+           "stage1_frac_of_hbm_peak": stage1_bytes(w) / (q_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+           "clocks": clocks, "data": "synthetic, drawn on the device", "status": int(status.item())}
+    if with_compensation:
+        rec["compensation_mma"] = bench_compensation_overhead(binding, s1, w, reps=2)
+    return rec
+
+
+def bench_two_tile_arrangement(binding, s1, w, out, status, steps):
+    """The same attention launch in the two-query-tile arrangement (Section 5.1's two stages), for the comparison."""
+    binding.mpfa_set_prefill_arrangement(1)
+    try:
+        ms, mn = time_calls(lambda: binding.prefill(s1, w.causal, w.softmax_scale, out=out, status=status), steps, 3)
+    finally:
+        binding.mpfa_set_prefill_arrangement(0)
+    return {"ms": ms, "ms_min": mn, "value": w.flops / (ms * 1e-3) / 1e12, "unit": "TFLOPS", "status": int(status.item())}
+
+
 def run_ours(args, rank, world, local):
     from paper_2609_33135_b200 import binding, workloads as wl
     binding.lib()  # fail loudly if the CUDA library is missing
@@ -423,6 +522,12 @@ def run_ours(args, rank, world, local):
 
     flops = w.flops
     value = whole_job_value(world, flops, ms_step)
+    mma = None
+    if rank == 0:
+        try:
+            mma = bench_mma_peaks(binding, dev)
+        except Exception as e:
+            mma = None
     long_run = total_ms > 2000.0
     bf16_peak = peaks["bf16_sustained"] if long_run else peaks["bf16"]
     peak = bf16_peak * MIXED_OVER_BF16
@@ -441,7 +546,13 @@ def run_ours(args, rank, world, local):
                 "h2d_bytes_per_step": (q.numel() + k.numel() + v.numel()) * 2, "d2h_bytes_per_step": out.numel() * 2},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": {"kernel": "prefill_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
-                     "unit": "TFLOP/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(N),
+                     "unit": "TFLOP/s", "frac": achieved / peak,
+                     "traffic": NCU_TRAFFIC_BYTES.get((w.H_q, N), {}).get("bytes"),
+                     "traffic_source": NCU_TRAFFIC_BYTES.get((w.H_q, N), {}).get("source"),
+                     "peak_measured": mma["mixed_fp4_fp8"] if mma else None,
+                     "frac_of_peak_measured": achieved / mma["mixed_fp4_fp8"] if mma else None,
+                     "peak_nominal": NOMINAL_MIXED_TFLOPS, "frac_of_peak_nominal": achieved / NOMINAL_MIXED_TFLOPS,
+                     "mma_rates_measured": mma,
                      "kernel_ms": kernel_ms,
                      "peak_note": f"{peaks['source']} bf16 {'sustained' if long_run else 'burst'} {bf16_peak} TF/s x 8/3 "
                                   "(nominal fp4 4x / fp8 2x of bf16; equal FP4 and FP8 FLOPs per pair)",
@@ -451,10 +562,8 @@ def run_ours(args, rank, world, local):
                                 "note": "attention kernel alone, quantization excluded (as the paper times it)"},
         "quantize_ms": ms_step - kernel_ms,
     }
-    # stage 1 against HBM: 2 passes over Q and K (statistics, quantize) + K once more for Delta_S + V once,
-    # packed codes, scales, Delta_S and FP8 V written
-    nq, nk = q.numel(), k.numel()
-    q_bytes = (2 * 2 + 0.5625) * (nq + nk) + 2 * nk + 2.0 * w.B * w.N_kv * w.H_q + 3 * v.numel()
+    # stage 1 against HBM (algorithmic bytes: see stage1_bytes)
+    q_bytes = stage1_bytes(w)
     result["quantize"] = {"ms": ms_step - kernel_ms, "algorithmic_bytes": q_bytes,
                           "value": q_bytes / ((ms_step - kernel_ms) * 1e-3) / 1e9, "unit": "GB/s",
                           "frac_of_hbm_peak": q_bytes / ((ms_step - kernel_ms) * 1e-3) / 1e9 / peaks["hbm_gbs"]}
@@ -477,17 +586,58 @@ def run_ours(args, rank, world, local):
                 result["prefill_paged"] = bench_prefill_paged(w, k, v, s1, out, max(3, args.steps // 2), 3)
             except Exception as e:
                 result["prefill_paged"] = {"error": repr(e)}
+        try:
+            result["prefill_two_tile_arrangement"] = bench_two_tile_arrangement(binding, s1, w, out, status, max(3, args.steps // 2))
+        except Exception as e:
+            result["prefill_two_tile_arrangement"] = {"error": repr(e)}
+        if world == 1 and not args.no_configs:
+            # the other lengths of the metric (configs 3 and 4), after the main buffers are released
+            del slots
+            torch.cuda.empty_cache()
+            by_cfg = {}
+            for key, name, seed, N2, hq2, comp in (("cfg3_32k", "cfg3_qwen14b_causal_32768", 1003, 32768, 40, False),
+                                                   ("cfg3_64k", "cfg3_qwen14b_causal_65536", 1003, 65536, 40, False),
+                                                   ("cfg4_128k", "cfg4_long_causal_131072", 1004, 131072, 32, True)):
+                try:
+                    by_cfg[key] = bench_prefill_config(binding, wl, name, seed, N2, hq2, peaks, mma, local, comp)
+                except Exception as e:
+                    by_cfg[key] = {"error": repr(e)}
+                torch.cuda.empty_cache()
+            result["prefill_by_config"] = by_cfg
+        if "decode" in result and "value" in result["decode"]:
+            result["decode"]["frac_of_nominal_hbm"] = result["decode"]["value"] / NOMINAL_HBM_GBS
+            result["decode"]["nominal_hbm_gbs"] = NOMINAL_HBM_GBS
         if world == 1 and not args.no_cpu:
             cores = os.cpu_count() or 1
             fl, times, sample = cpu_oracle_sample(w, 1, rows_per_head=args.cpu_rows_per_head)
-            result["cpu_baseline"] = {"value": fl / times[0] / 1e12, "unit": "TFLOPS", "cores": cores,
-                                      "kind": "oracle", "sample": sample, "seconds": times[0]}
+            result["cpu_baseline"] = cpu_baseline_record(fl, times, sample, cores)
         print(json.dumps(result))
 
 
-# DRAM bytes per prefill launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum);
-# from profiles/prefill_kernel_llama_shape.md (65,293,056 read + 80,688,640 written), keyed by sequence length.
-NCU_TRAFFIC_BYTES = {16384: 145981696}
+# DRAM bytes per prefill launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum), keyed by
+# (q heads, sequence length); lengths without a capture report no traffic figure.
+NCU_TRAFFIC_BYTES = {
+    (32, 16384): {"bytes": 145981696, "source": "profiles/prefill_kernel_llama_shape.md section 2 (65,293,056 read + 80,688,640 written)"},
+    (32, 131072): {"bytes": 44430000000, "source": "profiles/prefill_kernel_128k_and_paged_source.md section 1 (43.4 GB read + 1.03 GB written)"},
+}
+
+
+def _spawned_rank(rank, n, port, argv):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    sys.argv = argv
+    main()
+
+
+def spawn_ranks(n, fn=_spawned_rank):
+    """`python bench.py --gpus N` without a launcher: start the N ranks here (one process per GPU, rendezvous on
+    127.0.0.1), the same as `python -m torch.distributed.run --nproc-per-node N bench.py --gpus N ...`."""
+    import socket
+    import torch.multiprocessing as mp
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    mp.spawn(fn, args=(n, port, list(sys.argv)), nprocs=n, join=True)
 
 
 def main():
@@ -503,10 +653,16 @@ def main():
     ap.add_argument("--compensation", action="store_true", help="time the compensation placements even with --no-decode")
     ap.add_argument("--small-decode", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the 32K / 64K / 128K lines (prefill_by_config)")
     ap.add_argument("--cpu-rows-per-head", type=int, default=8192)
+    ap.add_argument("--ref-rows-per-head", type=int, default=512,
+                    help="reference arm: query rows per head in each step's sample")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args, int(os.environ.get("RANK", 0)))
+        return
+    if args.gpus > 1 and "RANK" not in os.environ:
+        spawn_ranks(args.gpus)
         return
     rank, world, local = dist_setup(args.gpus)
     try:

@@ -82,10 +82,25 @@ def k_structure(seed: int, H_kv: int, n_outlier: int):
 
 
 def make_qkv(seed: int, B: int, N_q: int, N_kv: int, H_q: int, H_kv: int,
-             n_outlier: Optional[int] = None, q_bias: bool = False):
-    """Draw Q [B,N_q,H_q,128], K, V [B,N_kv,H_kv,128] (BF16, CPU)."""
+             n_outlier: Optional[int] = None, q_bias: bool = False, device: str = "cpu"):
+    """Draw Q [B,N_q,H_q,128], K, V [B,N_kv,H_kv,128] (BF16).  On "cpu" the draw uses the CPU generator; on a CUDA
+    device it uses that device's generator with the same seeds (a different but equally reproducible stream),
+    which keeps the long benchmark shapes off the host."""
     if n_outlier is None:
         n_outlier = max(1, round(0.01 * H_kv * HEAD_DIM))
+    if device != "cpu":
+        def draw(sub, n, h):
+            g = torch.Generator(device=device)
+            g.manual_seed(seed * 16 + _SUB[sub])
+            return torch.randn(B, n, h, HEAD_DIM, generator=g, device=device)
+        q = draw("q", N_q, H_q)
+        if q_bias:
+            q = q + torch.empty(H_q, HEAD_DIM, dtype=torch.float32).normal_(
+                mean=0.0, std=math.sqrt(2.0), generator=_gen(seed, "qbias")).to(device)
+        bias, factor = k_structure(seed, H_kv, n_outlier)
+        k = draw("k", N_kv, H_kv) * factor.to(device) + bias.to(device)
+        v = draw("v", N_kv, H_kv)
+        return _finish(q), _finish(k), _finish(v)
     q = _randn_chunked((B * N_q, H_q, HEAD_DIM), _gen(seed, "q")).view(B, N_q, H_q, HEAD_DIM)
     if q_bias:
         qb = torch.empty(H_q, HEAD_DIM, dtype=torch.float32).normal_(
@@ -100,9 +115,9 @@ def make_qkv(seed: int, B: int, N_q: int, N_kv: int, H_q: int, H_kv: int,
 
 def prefill_workload(name: str, seed: int, B: int, N: int, H_q: int, H_kv: int, causal: bool,
                      n_outlier: Optional[int] = None, q_bias: bool = False,
-                     N_q: Optional[int] = None) -> PrefillWorkload:
+                     N_q: Optional[int] = None, device: str = "cpu") -> PrefillWorkload:
     N_q = N if N_q is None else N_q
-    q, k, v = make_qkv(seed, B, N_q, N, H_q, H_kv, n_outlier, q_bias)
+    q, k, v = make_qkv(seed, B, N_q, N, H_q, H_kv, n_outlier, q_bias, device)
     return PrefillWorkload(name, B, N_q, N, H_q, H_kv, causal, 1.0 / math.sqrt(HEAD_DIM), q, k, v)
 
 

@@ -69,3 +69,40 @@ def test_reference_arm_runs_on_rank_zero_only(capsys):
         gpus, steps, warmup = 2, 1, 0
     bench.run_reference(A, rank=1)        # other ranks exit without work or output
     assert capsys.readouterr().out == ""
+
+
+def _spawn_probe(rank, n, port, argv):
+    """Stands in for bench._spawned_rank: same arguments; sets the same environment through it but stops before
+    the CUDA part, then goes through the rendezvous on gloo."""
+    sys.path.insert(0, ROOT)
+    import bench
+    orig_main = bench.main
+    seen = {}
+    bench.main = lambda: seen.update(rank=os.environ["RANK"], world=os.environ["WORLD_SIZE"],
+                                     local=os.environ["LOCAL_RANK"], addr=os.environ["MASTER_ADDR"], argv=list(sys.argv))
+    try:
+        bench._spawned_rank(rank, n, port, argv)
+    finally:
+        bench.main = orig_main
+    assert seen == {"rank": str(rank), "world": str(n), "local": str(rank), "addr": "127.0.0.1", "argv": argv}
+    r, w, _ = bench.dist_setup(n, backend="gloo")
+    assert (r, w) == (rank, n)
+    assert bench.max_over_ranks(float(rank), w) == float(n - 1)
+    import torch.distributed as dist
+    dist.destroy_process_group()
+
+
+@pytest.mark.timeout(120)
+def test_plain_invocation_with_gpus_spawns_its_own_ranks(monkeypatch):
+    """`python bench.py --gpus 2` without a launcher (no RANK in the environment) must start the ranks itself."""
+    sys.path.insert(0, ROOT)
+    import bench
+    for k in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT"):
+        monkeypatch.delenv(k, raising=False)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "2", "--steps", "1"])
+    bench.spawn_ranks(2, fn=_spawn_probe)
+    # and main() takes that route when RANK is unset
+    called = {}
+    monkeypatch.setattr(bench, "spawn_ranks", lambda n: called.setdefault("n", n))
+    bench.main()
+    assert called == {"n": 2}
