@@ -52,9 +52,16 @@ def lib() -> ctypes.CDLL:
     """Load libmpfa.so (built by paper_2609_33135_b200.build).  Raises if it is missing."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise MpfaError(f"{LIB_PATH} not found: build it with `python -m paper_2609_33135_b200.build`")
-        L = ctypes.CDLL(LIB_PATH)
+        _lib = load_library(LIB_PATH)
+    return _lib
+
+
+def load_library(path: str) -> ctypes.CDLL:
+    """A build of the library with the C ABI's argument types declared."""
+    if True:
+        if not os.path.exists(path):
+            raise MpfaError(f"{path} not found: build it with `python -m paper_2609_33135_b200.build`")
+        L = ctypes.CDLL(path)
         sz, i, f, vp = ctypes.c_size_t, ctypes.c_int, ctypes.c_float, ctypes.c_void_p
         L.mpfa_quantize_workspace_bytes.restype = sz
         L.mpfa_quantize_workspace_bytes.argtypes = [i, i, i]
@@ -108,8 +115,7 @@ def lib() -> ctypes.CDLL:
         L.mpfa_bench_mma_peak.argtypes = [i, i, i, vp, vp]
         L.mpfa_bench_mma_flops.restype = ctypes.c_double
         L.mpfa_bench_mma_flops.argtypes = [i, i, i]
-        _lib = L
-    return _lib
+        return L
 
 
 def _check(rc: int, what: str) -> None:

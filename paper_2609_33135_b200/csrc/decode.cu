@@ -106,7 +106,12 @@ constexpr uint32_t TM_SFK = 400;   // D_NK x 8
 static_assert(TM_SFK + D_NK * 8 <= 512, "tensor memory");
 constexpr uint32_t TM_COLS = 512;
 
-constexpr long long D_WAIT_CYCLES = 4000000000ll;   // about two seconds
+#ifndef MPFA_WAIT_LIMIT_CYCLES
+#define MPFA_WAIT_LIMIT_CYCLES 4000000000ll   // about two seconds of SM clock
+#endif
+constexpr long long D_WAIT_CYCLES = MPFA_WAIT_LIMIT_CYCLES;
+// Test builds only (-DMPFA_TEST_DROP_V_COPY with a short limit): every CTA's V producer leaves out its first copy,
+// so the give-up path runs (status bit, roles leave, copies in flight awaited, tensor memory released).
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -453,6 +458,11 @@ __global__ void __launch_bounds__(D_THREADS, 1) decode_split_kernel(const Decode
             fence_proxy_async_smem();
             __syncwarp();
           }
+#ifdef MPFA_TEST_DROP_V_COPY
+          if (c == 0) {
+            // left out on purpose (work items are drawn dynamically: any CTA may be the one that gets work)
+          } else
+#endif
           if (elect_one()) {
             const uint32_t sdst = sbase + D_OFF_V + st * VST_BYTES;
             mbar_expect_tx(full, (id0 >= 0 ? 8192u : 0u) + (id1 >= 0 ? 8192u : 0u));

@@ -47,7 +47,19 @@ namespace {
 #define MPFA_WAIT_LIMIT_CYCLES 4000000000ll   // about 2 s of SM clock: far beyond any legitimate wait
 #endif
 constexpr long long WAIT_LIMIT_CYCLES = MPFA_WAIT_LIMIT_CYCLES;
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;       // drain path only
+#ifndef MPFA_DRAIN_LIMIT_NS
+#define MPFA_DRAIN_LIMIT_NS 2000000000ull
+#endif
+constexpr uint64_t WAIT_LIMIT_NS = MPFA_DRAIN_LIMIT_NS;   // drain path only
+// Test builds only (-DMPFA_TEST_DROP_V_COPY, together with short limits): the producer of CTA 0 leaves out the
+// first V copy of the launch, so the P V issuer's wait for it runs out and the whole give-up path executes -
+// status bit, every role leaving its loops, copies in flight drained, tensor memory released.  Never defined in
+// the product library.
+#ifdef MPFA_TEST_DROP_V_COPY
+#define MPFA_DROP_V(c) ((c) == 0u && blockIdx.x == 0)
+#else
+#define MPFA_DROP_V(c) false
+#endif
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;

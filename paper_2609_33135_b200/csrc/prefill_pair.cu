@@ -290,7 +290,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         nk_armed = c + 1;
         if (c >= (uint32_t)VSTAGES) ok = cx.wait(BAR_V_EMPTY + vs, (c / VSTAGES - 1) & 1u);
         if (!ok) break;
-        if (PAGED) {
+        if (MPFA_DROP_V(c)) {
+          // test build: this copy is left out on purpose
+        } else if (PAGED) {
           if (elect_one()) {
             const uint32_t bar = cx.bar(BAR_V_FULL + vs);
             mbar_expect_tx(bar, 16384);
@@ -301,7 +303,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           mbar_expect_tx(cx.bar(BAR_V_FULL + vs), 16384);
           tma_load_2d(sbase + OFF_V + vs * 16384, &tm_v, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
         }
-        nv_armed = c + 1;
+        if (!MPFA_DROP_V(c)) nv_armed = c + 1;
       }
       gb += it.Tmax;
       ++tq;
@@ -311,7 +313,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (uint32_t c = nk_armed - min(nk_armed, (uint32_t)KSTAGES); c < nk_armed; ++c)
         mbar_wait_ns(cx.bar(BAR_K_FULL + c % KSTAGES), (c / KSTAGES) & 1u, WAIT_LIMIT_NS);
       for (uint32_t c = nv_armed - min(nv_armed, (uint32_t)VSTAGES); c < nv_armed; ++c)
-        mbar_wait_ns(cx.bar(BAR_V_FULL + c % VSTAGES), (c / VSTAGES) & 1u, WAIT_LIMIT_NS);
+        if (!MPFA_DROP_V(c)) mbar_wait_ns(cx.bar(BAR_V_FULL + c % VSTAGES), (c / VSTAGES) & 1u, WAIT_LIMIT_NS);
       for (uint32_t i = nq_armed - min(nq_armed, 2u); i < nq_armed; ++i)
         mbar_wait_ns(cx.bar(BAR_Q_FULL + (i & 1)), (i >> 1) & 1u, WAIT_LIMIT_NS);
     }
