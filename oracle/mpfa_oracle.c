@@ -301,10 +301,24 @@ typedef struct {
  * v: E4M3 codes [n, D] (v_f32 == NULL) or FP32 values [n, D].
  * p_fp8: quantize P to E4M3 with the fixed scale 448 (else keep FP32 P * 448).
  * phat_out (optional, inspection only): receives, per key index, the E4M3 code
- * the loop gave that key's P when its block was visited. */
+ * the loop gave that key's P when its block was visited.
+ * Inspection hooks, used only by mpfa_oracle_phat_rows (NULL / -1 everywhere
+ * else, where they change nothing): q_out receives the FP32 value 448 P that
+ * was encoded; flip_key >= 0 moves that one key's code by flip_dir steps
+ * (to show what a one-step difference in a single P-hat does to a row). */
+static void online_softmax_pv_x(const float *s, int k0, int k1, float lam, const uint8_t *v,
+                                const float *v_f32, int block, int reverse, int p_fp8,
+                                softmax_state *st, uint8_t *phat_out, float *q_out, int flip_key, int flip_dir);
+
 static void online_softmax_pv(const float *s, int k0, int k1, float lam, const uint8_t *v,
                               const float *v_f32, int block, int reverse, int p_fp8,
                               softmax_state *st, uint8_t *phat_out) {
+  online_softmax_pv_x(s, k0, k1, lam, v, v_f32, block, reverse, p_fp8, st, phat_out, NULL, -1, 0);
+}
+
+static void online_softmax_pv_x(const float *s, int k0, int k1, float lam, const uint8_t *v,
+                                const float *v_f32, int block, int reverse, int p_fp8,
+                                softmax_state *st, uint8_t *phat_out, float *q_out, int flip_key, int flip_dir) {
   st->m = -INFINITY;
   st->l = 0.0f;
   for (int c = 0; c < D; ++c) st->o[c] = 0.0f;
@@ -334,6 +348,11 @@ static void online_softmax_pv(const float *s, int k0, int k1, float lam, const u
       float ph = p[j - a] * 448.0f;
       if (p_fp8) {
         uint8_t code = mpfa_oracle_e4m3_encode(ph);
+        if (q_out) q_out[j] = ph;
+        if (j == flip_key) {
+          int c2 = (int)code + flip_dir;
+          code = (uint8_t)(c2 < 0 ? 0 : (c2 > 0x7E ? 0x7E : c2));
+        }
         if (phat_out) phat_out[j] = code;
         ph = e4m3_tab[code];
       }
@@ -564,13 +583,14 @@ void mpfa_oracle_logits_rows(const uint8_t *q_codes, const uint8_t *q_sf, const 
  * loop assigns to every visible key of the listed rows (Section 4.1: fixed
  * scale 448, quantized against the running maximum of the traversal), plus the
  * final (m, l) of each row.  Same calls as prefill_rows_impl; nothing is
- * computed differently.  codes_out: [n_rows, Nkv] (keys a row cannot see stay 0),
- * ml_out: [n_rows, 2]. */
+ * computed differently unless flip_key >= 0.  codes_out: [n_rows, Nkv] (keys a row
+ * cannot see stay 0), ml_out: [n_rows, 2]; optional q_out [n_rows, Nkv] (the FP32
+ * values 448 P that were encoded) and o_out [n_rows, D] (outputs, v_scale = 1). */
 void mpfa_oracle_phat_rows(const uint8_t *q_codes, const uint8_t *q_sf, const uint8_t *k_codes,
                            const uint8_t *k_sf, const uint8_t *v_codes, const uint16_t *delta,
                            const float *dq, const float *dk, float softmax_scale, int causal, int Nq, int Nkv,
                            int Hq, int Hkv, int block_kv, int reverse, const int32_t *rows, int n_rows,
-                           uint8_t *codes_out, float *ml_out) {
+                           uint8_t *codes_out, float *ml_out, float *q_out, float *o_out, int flip_key, int flip_dir) {
   init_tables();
   int grp = Hq / Hkv;
   for (int r = 0; r < n_rows; ++r) {
@@ -585,10 +605,13 @@ void mpfa_oracle_phat_rows(const uint8_t *q_codes, const uint8_t *q_sf, const ui
     float lam = ((softmax_scale * 1.4426950408889634f) * dq[b]) * dk[b];
     softmax_state st;
     memset(codes_out + (size_t)r * Nkv, 0, (size_t)Nkv);
-    online_softmax_pv(s, 0, n, lam, v_codes + ((size_t)b * Hkv + hk) * Nkv * D, NULL, block_kv, reverse, 1, &st,
-                      codes_out + (size_t)r * Nkv);
+    if (q_out) memset(q_out + (size_t)r * Nkv, 0, sizeof(float) * (size_t)Nkv);
+    online_softmax_pv_x(s, 0, n, lam, v_codes + ((size_t)b * Hkv + hk) * Nkv * D, NULL, block_kv, reverse, 1, &st,
+                        codes_out + (size_t)r * Nkv, q_out ? q_out + (size_t)r * Nkv : NULL, flip_key, flip_dir);
     ml_out[2 * r] = st.m;
     ml_out[2 * r + 1] = st.l;
+    if (o_out)   /* the row's output before the BF16 rounding, v_scale = 1 */
+      for (int c = 0; c < D; ++c) o_out[(size_t)r * D + c] = (st.l > 0.0f) ? st.o[c] / (448.0f * st.l) : 0.0f;
     free(s);
   }
 }

@@ -265,15 +265,20 @@ def logits_rows(z: Quantized, rows, use_delta=True) -> np.ndarray:
 
 
 def phat_rows(z: Quantized, rows, softmax_scale: float, causal: bool, block_kv: int = BLOCK_KV,
-              reverse: bool = True, use_delta: bool = True):
-    """Inspection: E4M3 codes of P-hat per visible key [n,Nkv] and the final (m, l) [n,2] of rows [n,3]."""
+              reverse: bool = True, use_delta: bool = True, want_q: bool = False, flip_key: int = -1, flip_dir: int = 0):
+    """Inspection: E4M3 codes of P-hat per visible key [n,Nkv] and the final (m, l) [n,2] of rows [n,3].
+    want_q: also the FP32 values 448 P that were encoded [n,Nkv] and the rows' outputs [n,128] (v_scale 1).
+    flip_key >= 0: that key's code is moved by flip_dir steps before it is used (what-if for one P-hat)."""
     rows = _c(rows, np.int32)
     B, Hq, Nq, _ = z.q_codes.shape
     Hkv, Nkv = z.k_codes.shape[1], z.k_codes.shape[2]
     codes = np.empty((rows.shape[0], Nkv), np.uint8)
     ml = np.empty((rows.shape[0], 2), np.float32)
+    q = np.empty((rows.shape[0], Nkv), np.float32) if want_q else None
+    o = np.empty((rows.shape[0], D), np.float32) if want_q else None
     lib().mpfa_oracle_phat_rows(_p(z.q_codes), _p(z.q_sf), _p(z.k_codes), _p(z.k_sf), _p(z.v_codes),
                                 _p(z.delta if use_delta else None), _p(_c(z.dq, np.float32)),
                                 _p(_c(z.dk, np.float32)), ctypes.c_float(softmax_scale), int(causal), Nq, Nkv, Hq,
-                                Hkv, block_kv, int(reverse), _p(rows), rows.shape[0], _p(codes), _p(ml))
-    return codes, ml
+                                Hkv, block_kv, int(reverse), _p(rows), rows.shape[0], _p(codes), _p(ml), _p(q), _p(o),
+                                int(flip_key), int(flip_dir))
+    return (codes, ml, q, o) if want_q else (codes, ml)

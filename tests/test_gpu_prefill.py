@@ -155,20 +155,44 @@ def test_prefill_on_degenerate_inputs(kind):
     rows = orc.all_rows(w.B, w.H_q, w.N_q)
     ref32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
     o16, o32 = run_gpu(w)
-    # These tensors are plain N(0,1) draws without the workloads' structure.  The kernel takes 2^x from the hardware
-    # approximation (within 2 ulp), the oracle rounds it correctly; when 448 P falls within that distance of an E4M3
-    # rounding boundary the two pick neighbouring codes (a 6 % step of one P), which on a row with few dozen keys
-    # moves the output by a few 1e-3.  One such row in 2400 was seen here ("zeros", request 1, head 3, row 81:
-    # 4.5e-3), so isolated rows get the allowance of one such step; everything else is held to the usual bound.
+    # Both sides decide the E4M3 code of P-hat in FP32 from 448 P; the one input of that decision they do not share
+    # bit for bit is 2^x (hardware approximation within 2 ulp on the GPU, correctly rounded in the oracle).  A row may
+    # therefore exceed the bound only if that is demonstrably what happened: the oracle's own 448 P of one of its
+    # keys lies within 2e-6 (relative) of an E4M3 rounding boundary, and the oracle with exactly that key's code moved
+    # one step across that boundary reproduces the kernel's row within the usual bound.  On structured workloads no
+    # row needs this; on these structureless N(0,1) tensors one row in a few thousand does (few dozen keys, so one
+    # 6 % step of one P moves the output by a few 1e-3).
     g32 = o32[rows[:, 0], rows[:, 2], rows[:, 1]]
     d = np.abs(g32 - ref32)
     assert np.isfinite(g32).all()
-    row_max = d.max(axis=1)
-    assert (row_max > MAX_ABS).sum() <= max(1, len(rows) // 1000), (kind, int((row_max > MAX_ABS).sum()))
-    assert row_max.max() <= 3e-2 and d.mean() <= MEAN_ABS, (kind, float(row_max.max()), float(d.mean()))
-    keep = row_max <= MAX_ABS
+    assert d.mean() <= MEAN_ABS, (kind, float(d.mean()))
+    over = np.nonzero(d.max(axis=1) > MAX_ABS)[0]
+    assert len(over) <= max(1, len(rows) // 1000), (kind, len(over))
+    grid = np.array([orc.e4m3_decode(c) for c in range(0x7F)], np.float64)
+    bounds = (grid[1:] + grid[:-1]) / 2                      # rounding boundaries between adjacent codes
+    for r in over:
+        row = rows[r:r + 1]
+        codes, _, q, _ = orc.phat_rows(z, row, w.softmax_scale, True, want_q=True)
+        n_vis = int(row[0, 2]) + 1 + (w.N_kv - w.N_q)
+        qv = q[0, :n_vis].astype(np.float64)
+        nearest = np.abs(qv[:, None] - bounds[None, :])
+        j = nearest.argmin(axis=1)
+        rel = nearest[np.arange(n_vis), j] / np.maximum(bounds[j], 1e-30)
+        cands = np.nonzero(rel <= 2e-6)[0]
+        assert len(cands) >= 1, (kind, row, float(d[r].max()), float(rel.min()))
+        explained = False
+        for key in cands:
+            direction = 1 if codes[0, key] == j[key] else -1   # code below the boundary moves up, and the reverse
+            _, _, _, o_flip = orc.phat_rows(z, row, w.softmax_scale, True, want_q=True, flip_key=int(key), flip_dir=direction)
+            if np.abs(g32[r] - o_flip[0]).max() <= MAX_ABS:
+                explained = True
+                print(f"{kind}: row {row[0].tolist()} differs by {d[r].max():.2e}: key {key} has 448 P = {qv[key]:.9g}, "
+                      f"{rel[key]:.1e} from the boundary {bounds[j[key]]:.9g} between codes {j[key]:#x} and {j[key] + 1:#x}; "
+                      f"with that code moved one step the oracle is within {np.abs(g32[r] - o_flip[0]).max():.1e}")
+                break
+        assert explained, (kind, row, float(d[r].max()))
+    keep = d.max(axis=1) <= MAX_ABS
     compare(o16, o32, rows[keep], ref32[keep], kind)
-
 
 def test_prefill_many_items_without_keys_per_cta():
     """Causal, far more queries than keys (N_q = 8192, N_kv = 128, 32 heads): 63 of the 64 query tiles see no key at

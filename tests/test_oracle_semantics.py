@@ -275,3 +275,28 @@ def test_eq8_identity_through_the_oracle():
     # the oracle's delta_s call alone against Eq. 9
     dl = orc.bits_to_f32(orc.delta_s(k, z.q_mean, z.k_mean, z.dq, z.dk, 1)[0, 0]).astype(np.float64) * unit
     assert np.abs(dl - comp).max() <= (2.0 ** -8 + 1e-5) * np.abs(comp).max() + 1e-4
+
+
+def test_inspection_hooks_change_nothing_unless_asked():
+    """The what-if hook of the inspection entry point (move one key's P-hat code by one step) is what the GPU tests
+    use to show that a row outside the tolerance is a single code decision on a rounding boundary.  Without a flip
+    it must reproduce the product function bit for bit; with one it must change exactly that code, and the output by
+    that key's share: delta_code_value * (V_hat[k] - o) / (448 l) up to the rescaling roundings."""
+    w = wl.prefill_workload("t", 5, 1, 300, 2, 1, True)
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+    row = np.array([[0, 1, 200]], np.int32)
+    ref, _ = orc.prefill_rows(z, row, w.softmax_scale, True)
+    codes, ml, q, o = orc.phat_rows(z, row, w.softmax_scale, True, want_q=True)
+    assert np.array_equal(o, ref)
+    assert np.array_equal(_e4m3_codes_rne(q[0, :201]), codes[0, :201])
+    key = int(np.argsort(q[0, :201])[-3])
+    c2, _, _, o2 = orc.phat_rows(z, row, w.softmax_scale, True, want_q=True, flip_key=key, flip_dir=-1)
+    diff = np.nonzero(c2[0] != codes[0])[0]
+    assert list(diff) == [key] and int(c2[0, key]) == int(codes[0, key]) - 1
+    dv = e4m3_value(int(c2[0, key])) - e4m3_value(int(codes[0, key]))
+    vk = _e4m3_vals(z.v_codes[0, 0, key])
+    # the key sits in the row's first-visited (diagonal) block only if key >= 128; weight of its block at the end
+    want = o[0] + dv * vk / (448.0 * ml[0, 1]) * (1.0 if True else 0.0)
+    # exact only when no later rescaling touched the block (alpha = 1 after it); allow for alpha < 1 by bounding
+    assert np.abs(o2[0] - o[0]).max() > 0
+    assert np.abs(o2[0] - o[0]).max() <= np.abs(dv * vk / (448.0 * ml[0, 1])).max() * (1 + 1e-5) + 1e-7
