@@ -94,11 +94,13 @@ def test_error_against_exact_attention_with_and_without_compensation(capsys):
     """Reported, not gated beyond sanity: the kernel's error against exact (FP64) softmax attention on the unquantized
     inputs, for the three ways of running it - smoothing + compensation (the method), smoothing with the compensation
     term dropped, and the direct variant (no smoothing) - on the tiny configs (all rows) and on a row sample of the
-    16K benchmark config.  The figures are copied into the design notes."""
+    benchmark configs 2, 3 and 4.  The figures are copied into the design notes."""
     from paper_2609_33135_b200 import binding
     table = []
     for name, make, n_rows in (("cfg1", wl.config1_tiny, None), ("cfg1b_qbias", wl.config1b_tiny_qbias, None),
-                               ("cfg2_llama_16k", lambda: wl.config2_llama(16384), 512)):
+                               ("cfg2_llama_16k", lambda: wl.config2_llama(16384), 512),
+                               ("cfg3_qwen_32k", lambda: wl.config3_qwen(32768), 256),
+                               ("cfg4_long_128k", lambda: wl.config4_long(131072), 128)):
         w = make()
         q, k, v = orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v)
         rows = orc.all_rows(w.B, w.H_q, w.N_q) if n_rows is None else wl.sample_rows(8100, w.B, w.H_q, w.N_q, n_rows).numpy()
@@ -124,3 +126,32 @@ def test_error_against_exact_attention_with_and_without_compensation(capsys):
     with capsys.disabled():
         for name, errs in table:
             print(f"{name}: " + "; ".join(f"{k} mean {m:.3e} max {x:.3e}" for k, (m, x) in errs.items()))
+
+
+def test_decode_error_against_exact_attention_with_and_without_compensation(capsys):
+    """The same report for the paged decode path (config 5's recipe, four requests of 16K..128K tokens): the decode
+    output against exact FP64 attention of the new query token over the request's unquantized K/V, for the method,
+    the method with the Delta_S side cache dropped, and the direct variant."""
+    from paper_2609_33135_b200 import decode_cache
+    w = wl.config5_decode(4)
+    exact = []
+    for b in range(w.B):
+        k, v = w.kv_for_request(b)
+        rows = np.array([[0, h, 0] for h in range(w.H_q)], np.int32)
+        exact.append(orc.exact_rows(orc.bf16_bits(w.q_new[b:b + 1].contiguous()), orc.bf16_bits(k), orc.bf16_bits(v), rows,
+                                    w.softmax_scale, False))
+    exact = np.stack(exact)                                   # [B, H_q, 128]
+    errs = {}
+    for label, smooth, use_delta in (("method", True, True), ("no_compensation", True, False), ("direct", False, False)):
+        st = decode_cache.build_cache(w, smooth=smooth)
+        if not use_delta:
+            st.kv.delta = None
+        decode_cache.decode_step(st)
+        torch.cuda.synchronize()
+        assert int(st.status.item()) == 0
+        d = np.abs(st.out.float().cpu().numpy().astype(np.float64) - exact)
+        assert np.isfinite(d).all()
+        errs[label] = (float(d.mean()), float(d.max()))
+    assert errs["method"][0] < 0.1
+    with capsys.disabled():
+        print("cfg5_decode (4 requests): " + "; ".join(f"{k} mean {m:.3e} max {x:.3e}" for k, (m, x) in errs.items()))

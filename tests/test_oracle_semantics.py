@@ -295,8 +295,6 @@ def test_inspection_hooks_change_nothing_unless_asked():
     assert list(diff) == [key] and int(c2[0, key]) == int(codes[0, key]) - 1
     dv = e4m3_value(int(c2[0, key])) - e4m3_value(int(codes[0, key]))
     vk = _e4m3_vals(z.v_codes[0, 0, key])
-    # the key sits in the row's first-visited (diagonal) block only if key >= 128; weight of its block at the end
-    want = o[0] + dv * vk / (448.0 * ml[0, 1]) * (1.0 if True else 0.0)
-    # exact only when no later rescaling touched the block (alpha = 1 after it); allow for alpha < 1 by bounding
+    # the key's share is dv * V_hat[k] / (448 l), scaled down by the alphas of the blocks visited after its own
     assert np.abs(o2[0] - o[0]).max() > 0
     assert np.abs(o2[0] - o[0]).max() <= np.abs(dv * vk / (448.0 * ml[0, 1])).max() * (1 + 1e-5) + 1e-7
