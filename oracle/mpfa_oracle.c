@@ -615,3 +615,66 @@ void mpfa_oracle_phat_rows(const uint8_t *q_codes, const uint8_t *q_sf, const ui
     free(s);
   }
 }
+
+/* ------------------------------------------------------------------------- */
+/* precision-assignment variant: NVFP4 Q K^T with BF16 P V (Section 3.1)      */
+/* ------------------------------------------------------------------------- */
+
+/* One of the paper's four precision assignments (Section 3.1, Section 7.2): the logits are the same
+ * NVFP4 + rank-one logits as in the method, but P is carried to the second MMA in BF16 and V stays in
+ * BF16 (the unquantized input).  Per KV block (reverse order, as in the method):
+ *   m_new = max(m, rowmax);  P = 2^(lam S - lam m_new) in FP32;  l = alpha l + sum P (FP32 P);
+ *   P_b = BF16_RNE(P);  O = alpha O + sum_k P_b[k] V[k] (FP32, k ascending);  out = O / l.
+ * No scale 448 is involved (BF16 has the range); reading taken: P is rounded once, to nearest even.
+ * v: BF16 [B, Nkv, Hkv, D] as given to stage 1. */
+void mpfa_oracle_prefill_rows_pv_bf16(const uint8_t *q_codes, const uint8_t *q_sf, const uint8_t *k_codes,
+                                      const uint8_t *k_sf, const uint16_t *v, const uint16_t *delta, const float *dq,
+                                      const float *dk, float softmax_scale, int causal, int Nq, int Nkv, int Hq, int Hkv,
+                                      int block_kv, const int32_t *rows, int n_rows, float *out_f32, uint16_t *out_bf16) {
+  init_tables();
+  int grp = Hq / Hkv;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int r = 0; r < n_rows; ++r) {
+    int b = rows[3 * r], hq = rows[3 * r + 1], i = rows[3 * r + 2];
+    int hk = hq / grp;
+    int n = visible_keys(i, Nq, Nkv, causal);
+    float *s = (float *)malloc(sizeof(float) * (size_t)(n > 0 ? n : 1));
+    float *p = (float *)malloc(sizeof(float) * (size_t)block_kv);
+    logits_row_q4(q_codes + (((size_t)b * Hq + hq) * Nq + i) * (D / 2), q_sf + (((size_t)b * Hq + hq) * Nq + i) * NBLK,
+                  k_codes + ((size_t)b * Hkv + hk) * Nkv * (D / 2), k_sf + ((size_t)b * Hkv + hk) * Nkv * NBLK,
+                  delta ? delta + ((size_t)b * Hq + hq) * Nkv : NULL, n, s);
+    float lam = ((softmax_scale * 1.4426950408889634f) * dq[b]) * dk[b];
+    float m = -INFINITY, l = 0.0f, o[D];
+    for (int c = 0; c < D; ++c) o[c] = 0.0f;
+    for (int jb = n > 0 ? (n - 1) / block_kv : -1; jb >= 0; --jb) {
+      int a = jb * block_kv, e = (jb + 1) * block_kv > n ? n : (jb + 1) * block_kv;
+      float rowmax = -INFINITY;
+      for (int j = a; j < e; ++j)
+        if (s[j] > rowmax) rowmax = s[j];
+      float m_new = m > rowmax ? m : rowmax;
+      if (m_new == -INFINITY) continue;
+      float mlam = m_new * lam;
+      float alpha = (m == -INFINITY) ? 0.0f : exp2_f32((m - m_new) * lam);
+      float rowsum = 0.0f;
+      for (int j = a; j < e; ++j) {
+        p[j - a] = exp2_f32(fmaf(s[j], lam, -mlam));
+        rowsum += p[j - a];
+      }
+      l = alpha * l + rowsum;
+      for (int c = 0; c < D; ++c) o[c] = alpha * o[c];
+      for (int j = a; j < e; ++j) {
+        float pb = mpfa_oracle_bf16_to_f32(mpfa_oracle_f32_to_bf16(p[j - a]));
+        const uint16_t *vr = v + (((size_t)b * Nkv + j) * Hkv + hk) * D;
+        for (int c = 0; c < D; ++c) o[c] += pb * mpfa_oracle_bf16_to_f32(vr[c]);
+      }
+      m = m_new;
+    }
+    for (int c = 0; c < D; ++c) {
+      float x = (l > 0.0f) ? o[c] / l : 0.0f;
+      out_f32[(size_t)r * D + c] = x;
+      out_bf16[(size_t)r * D + c] = mpfa_oracle_f32_to_bf16(x);
+    }
+    free(p);
+    free(s);
+  }
+}

@@ -282,3 +282,20 @@ def phat_rows(z: Quantized, rows, softmax_scale: float, causal: bool, block_kv: 
                                 Hkv, block_kv, int(reverse), _p(rows), rows.shape[0], _p(codes), _p(ml), _p(q), _p(o),
                                 int(flip_key), int(flip_dir))
     return (codes, ml, q, o) if want_q else (codes, ml)
+
+
+def prefill_rows_pv_bf16(z: Quantized, v_bits: np.ndarray, rows, softmax_scale: float, causal: bool,
+                         block_kv: int = BLOCK_KV, use_delta: bool = True):
+    """Precision-assignment variant of Section 3.1: NVFP4 logits as in the method, P rounded to BF16, V = the BF16
+    input [B,Nkv,Hkv,128] (uint16 bits), FP32 accumulation.  -> (FP32 [n,128], BF16 bits [n,128])."""
+    rows = _c(rows, np.int32)
+    B, Hq, Nq, _ = z.q_codes.shape
+    Hkv, Nkv = z.k_codes.shape[1], z.k_codes.shape[2]
+    n = rows.shape[0]
+    o32 = np.empty((n, D), np.float32)
+    o16 = np.empty((n, D), np.uint16)
+    lib().mpfa_oracle_prefill_rows_pv_bf16(_p(z.q_codes), _p(z.q_sf), _p(z.k_codes), _p(z.k_sf), _p(_c(v_bits, np.uint16)),
+                                           _p(z.delta if use_delta else None), _p(_c(z.dq, np.float32)),
+                                           _p(_c(z.dk, np.float32)), ctypes.c_float(softmax_scale), int(causal), Nq, Nkv,
+                                           Hq, Hkv, block_kv, _p(rows), n, _p(o32), _p(o16))
+    return o32, o16

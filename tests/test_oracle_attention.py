@@ -210,3 +210,35 @@ def test_elementwise_placement_adds_the_same_term_after_the_products():
     a, _ = orc.prefill_rows(z, all_rows, w.softmax_scale, True, use_delta=False)
     b, _ = orc.prefill_rows(z, all_rows, w.softmax_scale, True, use_delta=False, elementwise=True)
     assert np.array_equal(a, b)
+
+
+def test_bf16_pv_variant_against_fp64_recomputation():
+    """Section 3.1's NVFP4 + BF16 assignment: same logits as the method, P in BF16, V unquantized BF16.  Pinned
+    against an FP64 softmax over the oracle's own logits with the BF16 inputs of V (what is left is the BF16 rounding
+    of P: 2^-9 relative per term, and FP32 summation), on GQA heads with visibly different V, and against the method:
+    the two differ (FP8 P and FP8 V against BF16) but track each other."""
+    from test_oracle_stage1 import _dequant
+    w = wl.prefill_workload("t", 36, 1, 300, 4, 2, True, q_bias=True)
+    v = w.v.clone().float()
+    v[:, :, 1] = v[:, :, 1] * 0.5 + 3.0
+    w.v = wl._finish(v)
+    q, k, vb = orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v)
+    z = orc.stage1(q, k, vb)
+    rows = np.array([[0, h, i] for h in range(4) for i in (0, 127, 128, 299)], np.int32)
+    o32, o16 = orc.prefill_rows_pv_bf16(z, vb, rows, w.softmax_scale, True)
+    s = orc.logits_rows(z, rows).astype(np.float64)
+    lam = float(np.float32(w.softmax_scale)) * float(z.dq[0]) * float(z.dk[0])
+    vf = orc.bits_to_f32(vb).astype(np.float64)
+    for r, (_, h, i) in enumerate(rows):
+        x = s[r, :i + 1] * lam
+        p = np.exp(x - x.max())
+        ref = (p / p.sum()) @ vf[0, :i + 1, h // 2]
+        assert np.abs(o32[r] - ref).max() <= 2.0 ** -8 * np.abs(ref).max() + 1e-5, (h, i)
+        wrong = (p / p.sum()) @ vf[0, :i + 1, 1 - h // 2]
+        assert np.abs(o32[r] - wrong).max() > 0.5
+    assert np.array_equal(o16, torch.from_numpy(o32).to(torch.bfloat16).view(torch.uint16).numpy())
+    m32, _ = orc.prefill_rows(z, rows, w.softmax_scale, True)
+    d = np.abs(m32 - o32)
+    assert 1e-4 < d.mean() < 0.1
+    # single-key rows return V itself (P = 1 up to the rounding of lam * m inside the fused multiply-add)
+    assert np.abs(o32[0] - vf[0, 0, 0]).max() <= 1e-5
