@@ -368,7 +368,7 @@ def stage1_bytes(w):
     return (2 * 2 + 0.5625) * (nq + nk) + 2.0 * w.B * w.N_kv * w.H_q + 3 * w.v.numel()
 
 
-def bench_prefill_config(binding, wl, name, seed, N, H_q, peaks, mma, local, with_compensation):
+def bench_prefill_config(binding, wl, name, seed, N, H_q, peaks, mma, local, with_compensation, with_variants=False):
     """One more prefill length of the metric (configs 3 and 4), inputs drawn on the device: attention kernel alone,
     the whole step with stage 1, stage-1 GB/s, fractions of the bounds, clocks sampled during the timed steps."""
     dev = torch.device("cuda", local)
@@ -397,6 +397,18 @@ def bench_prefill_config(binding, wl, name, seed, N, H_q, peaks, mma, local, wit
            "clocks": clocks, "data": "synthetic, drawn on the device", "status": int(status.item())}
     if with_compensation:
         rec["compensation_mma"] = bench_compensation_overhead(binding, s1, w, reps=2)
+    if with_variants:
+        # Section 3.1's precision assignments on the same quantized Q and K: NVFP4 + FP8 (the product path) against
+        # NVFP4 + BF16 (P in BF16, V unquantized, second MMA kind::f16), attention kernel alone
+        vt = binding.mpfa_pack_v_bf16(w.v)
+        run = lambda: binding.mpfa_prefill_variant(s1.q, s1.k, vt, s1.delta, s1.stats, 1.0, True, w.softmax_scale,
+                                                   binding.MPFA_VARIANT_PV_BF16, out, None, status)
+        b_ms, b_min = time_calls(run, steps, 2)
+        rec["precision_variants"] = {"nvfp4_qk_fp8_pv_ms": k_ms, "nvfp4_qk_bf16_pv_ms": b_ms,
+                                     "nvfp4_qk_bf16_pv_tflops": w.flops / (b_ms * 1e-3) / 1e12,
+                                     "fp8_pv_speedup_over_bf16_pv": b_ms / k_ms, "status": int(status.item()),
+                                     "note": "NVFP4 + NVFP4 not built"}
+        del vt
     return rec
 
 
@@ -599,7 +611,7 @@ def run_ours(args, rank, world, local):
                                                    ("cfg3_64k", "cfg3_qwen14b_causal_65536", 1003, 65536, 40, False),
                                                    ("cfg4_128k", "cfg4_long_causal_131072", 1004, 131072, 32, True)):
                 try:
-                    by_cfg[key] = bench_prefill_config(binding, wl, name, seed, N2, hq2, peaks, mma, local, comp)
+                    by_cfg[key] = bench_prefill_config(binding, wl, name, seed, N2, hq2, peaks, mma, local, comp, with_variants=(N2 == 65536))
                 except Exception as e:
                     by_cfg[key] = {"error": repr(e)}
                 torch.cuda.empty_cache()

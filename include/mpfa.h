@@ -176,6 +176,10 @@ size_t mpfa_static_scratch_bytes(void);
 mpfa_status mpfa_quantize_v(const void *v_bf16, int B, int N_kv, int H_kv, float v_scale, uint8_t *v_fp8,
                             void *stream);
 
+/* For MPFA_VARIANT_PV_BF16 only (Section 3.1's NVFP4 + BF16 assignment): V unchanged, re-tiled from
+ * [B, N_kv, H_kv, 128] to [B, H_kv, N_kv_pad, 128] BF16 (pad rows zero; 1024-byte aligned, 2 * mpfa_v_fp8_bytes()). */
+mpfa_status mpfa_pack_v_bf16(const void *v_bf16, int B, int N_kv, int H_kv, void *v_tiles_bf16, void *stream);
+
 /* The same arithmetic for ONE request, written through its page-table row into the paged
  * cache (Section 6: low-bit K/V cache writes fused with quantization and compensation
  * generation).  k_bf16, v_bf16 [N_tokens, H_kv, 128] are the tokens at positions
@@ -229,8 +233,15 @@ mpfa_status mpfa_prefill(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tensor *h_k,
  *                                         running maximum.  Same term, one FP32 rounding placed differently; it
  *                                         exists to measure what the rank-one MMA saves.  With delta_s_bf16 == NULL
  *                                         it is the same as variant 0.
+ *   MPFA_VARIANT_PV_BF16                  the NVFP4 + BF16 precision assignment of Section 3.1 / Section 7.2: Q K^T as in
+ *                                         the product path (block-scaled FP4 MMA + rank-one seed), but P = 2^(lam S -
+ *                                         lam m) is rounded to BF16 (no scale 448) and the second MMA is BF16 x BF16 on
+ *                                         the UNQUANTIZED V.  For this variant the v_fp8 argument points at the BF16
+ *                                         tile tensor [B, H_kv, N_kv_pad, 128] written by mpfa_pack_v_bf16 (1024-byte
+ *                                         aligned) and v_scale must be 1.  It exists to measure what FP8 for P V buys
+ *                                         (always in the one-query-tile arrangement).
  * Any other value: MPFA_ERR_INVALID_ARG. */
-enum { MPFA_VARIANT_COMP_ELEMENTWISE = 1 };
+enum { MPFA_VARIANT_COMP_ELEMENTWISE = 1, MPFA_VARIANT_PV_BF16 = 2 };
 mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tensor *h_k, const uint8_t *v_fp8,
                                  const void *delta_s_bf16, const mpfa_stats *h_stats, float v_scale, int causal,
                                  float softmax_scale, int variant, void *out_bf16, float *out_f32,

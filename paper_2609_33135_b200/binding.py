@@ -21,6 +21,7 @@ MPFA_STATS_FROZEN = 2
 MPFA_DEV_TIMEOUT = 1
 MPFA_DEV_BAD_PAGE = 2
 MPFA_VARIANT_COMP_ELEMENTWISE = 1
+MPFA_VARIANT_PV_BF16 = 2
 HEAD_DIM = 128
 PAGE = 64
 
@@ -91,6 +92,8 @@ def load_library(path: str) -> ctypes.CDLL:
         L.mpfa_static_scratch_bytes.restype = sz
         L.mpfa_quantize_v.restype = i
         L.mpfa_quantize_v.argtypes = [vp, i, i, i, f, vp, vp]
+        L.mpfa_pack_v_bf16.restype = i
+        L.mpfa_pack_v_bf16.argtypes = [vp, i, i, i, vp, vp]
         L.mpfa_quantize_kv_paged.restype = i
         L.mpfa_quantize_kv_paged.argtypes = [vp, vp, i, i, i, i, i, ctypes.POINTER(_Stats), f,
                                              ctypes.POINTER(_PagedKV), vp, vp, sz, vp]
@@ -399,3 +402,12 @@ def mpfa_bench_mma_peak(kind: int, n_cols: int, iters: int, status: torch.Tensor
 def mpfa_set_prefill_arrangement(arrangement: int) -> None:
     """0 (default): one query tile per CTA; 1: two query tiles per CTA.  Same arithmetic row by row."""
     _check(lib().mpfa_set_prefill_arrangement(arrangement), "mpfa_set_prefill_arrangement")
+
+
+def mpfa_pack_v_bf16(v: torch.Tensor) -> torch.Tensor:
+    """V [B,N,H,128] bf16 -> the BF16 tile tensor [B,H,N_pad,128] the MPFA_VARIANT_PV_BF16 prefill reads."""
+    assert v.is_cuda and v.dtype == torch.bfloat16 and v.is_contiguous()
+    B, N, H, _ = v.shape
+    out = aligned_empty(2 * lib().mpfa_v_fp8_bytes(B, H, N), v.device).view(torch.bfloat16).view(B, H, _pad128(N), HEAD_DIM)
+    _check(lib().mpfa_pack_v_bf16(_ptr(v), B, N, H, _ptr(out), _stream()), "mpfa_pack_v_bf16")
+    return out

@@ -74,17 +74,6 @@ static_assert(REGS_UTIL<false> <= 128 && REGS_UTIL<true> <= 128 && REGS_CORR<fal
 static_assert(REGS_SOFTMAX % 8 == 0 && REGS_UTIL<false> % 8 == 0 && REGS_CORR<false> % 8 == 0 && REGS_UTIL<true> % 8 == 0 &&
               REGS_CORR<true> % 8 == 0, "setmaxnreg granularity");
 
-constexpr uint32_t OFF_Q = 0;                               // 2 tiles (the next tile's queries are prefetched)
-constexpr uint32_t OFF_K = OFF_Q + 2 * 8192;
-constexpr uint32_t OFF_V = OFF_K + KSTAGES * 8192;
-constexpr uint32_t OFF_DELTA = OFF_V + VSTAGES * 16384;
-constexpr uint32_t OFF_ONES = OFF_DELTA + KSTAGES * 4096;
-constexpr uint32_t OFF_SFQ = OFF_ONES + 4096;
-constexpr uint32_t OFF_SFK = OFF_SFQ + 2 * 1024;
-constexpr uint32_t OFF_ALPHA = OFF_SFK + KSTAGES * 1024;   // alpha[2][128]
-constexpr uint32_t OFF_M = OFF_ALPHA + 2 * 128 * 4;        // running maximum after block t, [t & 1][128]
-constexpr uint32_t OFF_L = OFF_M + 2 * 128 * 4;            // final (l, m) of the two softmax groups, [item & 3][2][2][128]
-constexpr uint32_t OFF_BAR = OFF_L + 4 * 4 * 128 * 4;
 enum {
   BAR_Q_FULL = 0,                       // [2] query tile of work item i in buffer i & 1
   BAR_Q_EMPTY = 2,                      // [2] every Q K^T MMA of that work item has completed
@@ -110,12 +99,35 @@ enum {
   BAR_SF_READY = BAR_O_FREE + 1,        // [KSTAGES] paged source only: scales and Delta_S of the stage re-tiled
   NUM_BARS = BAR_SF_READY + KSTAGES
 };
-constexpr uint32_t OFF_MISC = OFF_BAR + NUM_BARS * 8;   // tmem base, abort flag
-// paged source only: per K stage the two pages' scale bytes (2 x 512) and Delta_S rows (2 x 128) as stored
-constexpr uint32_t RAW_STAGE = 1280;
-constexpr uint32_t OFF_RAW = (OFF_MISC + 16 + 127) & ~127u;
-constexpr uint32_t SMEM_BYTES = OFF_MISC + 16 + 1024;                          // + slack for the 1024-byte alignment
-constexpr uint32_t SMEM_BYTES_PAGED = OFF_RAW + KSTAGES * RAW_STAGE + 1024;
+static_assert(NUM_BARS <= 64, "barrier table");
+// Shared-memory layout.  PVB = the NVFP4 + BF16 precision assignment (mpfa_prefill_variant): V tiles are BF16
+// (32 KB, two stages), P is handed to the second MMA through shared memory as a K-major BF16 A operand (2 x 32 KB),
+// and the K ring has three stages to make room.
+template <bool PVB>
+struct Lay {
+  static constexpr int KST = PVB ? 3 : KSTAGES;
+  static constexpr int VST = PVB ? 2 : VSTAGES;
+  static constexpr uint32_t V_BYTES = PVB ? 32768u : 16384u;
+  static constexpr uint32_t OFF_Q = 0;                               // 2 tiles (the next tile's queries are prefetched)
+  static constexpr uint32_t OFF_K = OFF_Q + 2 * 8192;
+  static constexpr uint32_t OFF_V = OFF_K + KST * 8192;
+  static constexpr uint32_t OFF_DELTA = OFF_V + VST * V_BYTES;
+  static constexpr uint32_t OFF_ONES = OFF_DELTA + KST * 4096;
+  static constexpr uint32_t OFF_SFQ = OFF_ONES + 4096;
+  static constexpr uint32_t OFF_SFK = OFF_SFQ + 2 * 1024;
+  static constexpr uint32_t OFF_ALPHA = OFF_SFK + KST * 1024;   // alpha[2][128]
+  static constexpr uint32_t OFF_M = OFF_ALPHA + 2 * 128 * 4;        // running maximum after block t, [t & 1][128]
+  static constexpr uint32_t OFF_L = OFF_M + 2 * 128 * 4;            // final (l, m) of the two softmax groups, [item & 3][2][2][128]
+  static constexpr uint32_t OFF_BAR = OFF_L + 4 * 4 * 128 * 4;
+  static constexpr uint32_t OFF_MISC = OFF_BAR + 64 * 8;            // tmem base, abort flag (NUM_BARS <= 64)
+  // paged source only: per K stage the two pages' scale bytes (2 x 512) and Delta_S rows (2 x 128) as stored
+  static constexpr uint32_t RAW_STAGE = 1280;
+  static constexpr uint32_t OFF_RAW = (OFF_MISC + 16 + 127) & ~127u;
+  static constexpr uint32_t OFF_PS = (OFF_MISC + 16 + 1023) & ~1023u;   // PVB only: P of the two softmax groups
+  static constexpr uint32_t SMEM_BYTES = (PVB ? OFF_PS + 2 * 32768 : OFF_MISC + 16) + 1024;   // + slack for the 1024-byte alignment
+  static constexpr uint32_t SMEM_BYTES_PAGED = OFF_RAW + KST * RAW_STAGE + 1024;
+};
+static_assert(Lay<true>::SMEM_BYTES <= 227 * 1024 && Lay<false>::SMEM_BYTES_PAGED <= 227 * 1024, "shared memory");
 
 constexpr uint32_t TM_S = 0, TM_O0 = 128, TM_O1 = 256, TM_P0 = 384, TM_P1 = 416, TM_SFQ = 448 /* 2 x 8 */,
                    TM_SFK0 = 464, TM_SFK1 = 472;
@@ -176,10 +188,21 @@ struct TileWalk {
 
 // EW: ablation variant of Section 7.4 (compensation placement): Delta_S is not seeded by the BF16 MMA but
 // loaded by the softmax warps and added to the scores element by element in FP32, before masking and the maximum.
-template <bool PAGED, bool EW>
+// PVB: precision-assignment variant of Section 3.1 (NVFP4 Q K^T, BF16 P V): P = 2^(lam S - lam m) is rounded to BF16
+// and handed to the second MMA through shared memory (K-major A operand), V is the BF16 input in the tile layout
+// written by mpfa_pack_v_bf16, the second MMA is kind::f16 (eight K = 16 steps per block).
+template <bool PAGED, bool EW, bool PVB = false>
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const PrefillParams p, const PagedSrc pg) {
+  static_assert(!(PVB && (PAGED || EW)), "the BF16 variant exists for contiguous operands with the seed MMA only");
+  using L = Lay<PVB>;
+  constexpr int KST = L::KST, VST = L::VST;
+  constexpr uint32_t OFF_Q = L::OFF_Q, OFF_K = L::OFF_K, OFF_V = L::OFF_V, OFF_DELTA = L::OFF_DELTA, OFF_ONES = L::OFF_ONES,
+                     OFF_SFQ = L::OFF_SFQ, OFF_SFK = L::OFF_SFK, OFF_M = L::OFF_M, OFF_L = L::OFF_L, OFF_BAR = L::OFF_BAR,
+                     OFF_MISC = L::OFF_MISC, OFF_RAW = L::OFF_RAW, RAW_STAGE = L::RAW_STAGE, OFF_PS = L::OFF_PS,
+                     V_BYTES = L::V_BYTES;
+  (void)OFF_PS; (void)OFF_RAW; (void)RAW_STAGE;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -222,7 +245,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   }
   // rank-one operands: MN-major, 128B swizzle, K = 16.  Row k = 0 of each 64-element half
   // holds the data (ones / Delta_S), every other row stays zero for the CTA's lifetime.
-  for (int i = tid; i < (KSTAGES * 4096 + 4096) / 16; i += NTHREADS)
+  for (int i = tid; i < (KST * 4096 + 4096) / 16; i += NTHREADS)
     reinterpret_cast<uint4 *>(smem + OFF_DELTA)[i] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
   if (tid < 128) reinterpret_cast<uint16_t *>(smem + OFF_ONES)[(tid >> 6) * 1024 + (tid & 63)] = 0x3F80;  // 1.0
@@ -274,10 +297,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       for (int t = 0; t < tl.T && ok; ++t) {
         const uint32_t c = gb + t;
         const int jb = tl.T - 1 - t;
-        const uint32_t ks = c % KSTAGES, vs = c % VSTAGES;
+        const uint32_t ks = c % KST, vs = c % VST;
         int page_lo = 0, page_hi = 0;
         if (PAGED) look.get(pg, p.status, tl.b, tl.nkv, t, jb, lane, page_lo, page_hi);
-        if (c >= (uint32_t)KSTAGES) ok = cx.wait(BAR_K_EMPTY + ks, (c / KSTAGES - 1) & 1u);
+        if (c >= (uint32_t)KST) ok = cx.wait(BAR_K_EMPTY + ks, (c / KST - 1) & 1u);
         if (!ok) break;
         TR(0, c, 0);
         if (PAGED) {
@@ -306,7 +329,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
         }
         nk_armed = c + 1;
-        if (c >= (uint32_t)VSTAGES) ok = cx.wait(BAR_V_EMPTY + vs, (c / VSTAGES - 1) & 1u);
+        if (c >= (uint32_t)VST) ok = cx.wait(BAR_V_EMPTY + vs, (c / VST - 1) & 1u);
         if (!ok) break;
         TR(0, c, 1);
         if (MPFA_DROP_V(c)) {
@@ -319,18 +342,20 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             bulk_load(sbase + OFF_V + vs * 16384 + 8192, pg.v_fp8 + ((size_t)page_hi * p.H_kv + tl.hk) * 8192, 8192, bar);
           }
         } else if (elect_one()) {
-          mbar_expect_tx(cx.bar(BAR_V_FULL + vs), 16384);
-          tma_load_2d(sbase + OFF_V + vs * 16384, &tm_v, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
+          mbar_expect_tx(cx.bar(BAR_V_FULL + vs), V_BYTES);
+          tma_load_2d(sbase + OFF_V + vs * V_BYTES, &tm_v, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
+          if (PVB)   // BF16 rows are 256 bytes: the second 64-channel half is a box of its own
+            tma_load_2d(sbase + OFF_V + vs * V_BYTES + 16384, &tm_v, 128, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
         }
         if (!MPFA_DROP_V(c)) nv_armed = c + 1;
       }
     }
     if (*cx.abort_flag) {
       // Drain: copies still in flight must land before the CTA's shared memory is released.
-      for (uint32_t c = nk_armed - min(nk_armed, (uint32_t)KSTAGES); c < nk_armed; ++c)
-        mbar_wait_ns(cx.bar(BAR_K_FULL + c % KSTAGES), (c / KSTAGES) & 1u, WAIT_LIMIT_NS);
-      for (uint32_t c = nv_armed - min(nv_armed, (uint32_t)VSTAGES); c < nv_armed; ++c)
-        if (!MPFA_DROP_V(c)) mbar_wait_ns(cx.bar(BAR_V_FULL + c % VSTAGES), (c / VSTAGES) & 1u, WAIT_LIMIT_NS);
+      for (uint32_t c = nk_armed - min(nk_armed, (uint32_t)KST); c < nk_armed; ++c)
+        mbar_wait_ns(cx.bar(BAR_K_FULL + c % KST), (c / KST) & 1u, WAIT_LIMIT_NS);
+      for (uint32_t c = nv_armed - min(nv_armed, (uint32_t)VST); c < nv_armed; ++c)
+        if (!MPFA_DROP_V(c)) mbar_wait_ns(cx.bar(BAR_V_FULL + c % VST), (c / VST) & 1u, WAIT_LIMIT_NS);
       for (uint32_t i = nq_armed - min(nq_armed, 2u); i < nq_armed; ++i)
         mbar_wait_ns(cx.bar(BAR_Q_FULL + (i & 1)), (i >> 1) & 1u, WAIT_LIMIT_NS);
     }
@@ -365,10 +390,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       for (int t = 0; t < tl.T && ok; ++t) {
         const uint32_t c = gb + t;
-        const uint32_t ks = c % KSTAGES, sb = c & 1;
+        const uint32_t ks = c % KST, sb = c & 1;
         TR(5, c, 0);
-        ok = cx.wait(BAR_K_FULL + ks, (c / KSTAGES) & 1u);
-        if (PAGED) ok = ok && cx.wait(BAR_SF_READY + ks, (c / KSTAGES) & 1u);
+        ok = cx.wait(BAR_K_FULL + ks, (c / KST) & 1u);
+        if (PAGED) ok = ok && cx.wait(BAR_SF_READY + ks, (c / KST) & 1u);
         if (!ok) break;
         const uint32_t tSFK = tm + (sb ? TM_SFK1 : TM_SFK0);
         const uint64_t d_sfk = d_sfk0 + (uint64_t)((ks * 1024) >> 4);
@@ -409,8 +434,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int rsw = tl.hq % G;
       for (int t = 0; t < tl.T && ok; ++t) {
         const uint32_t c = gb + t;
-        const uint32_t ks = c % KSTAGES;
-        ok = cx.wait(BAR_K_FULL + ks, (c / KSTAGES) & 1u);
+        const uint32_t ks = c % KST;
+        ok = cx.wait(BAR_K_FULL + ks, (c / KST) & 1u);
         if (!ok) break;
         const uint8_t *raw = smem + OFF_RAW + ks * RAW_STAGE;
         // scales: row-major [key][8] -> the 32x128b tile layout tcgen05.cp expects (lane = key mod 32)
@@ -433,7 +458,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   } else if (warp == 3) {
     // =========================== P V issuer ===========================
     const uint32_t id_fp8 = idesc_e4m3(128, 128, 0, 1);
-    const uint64_t d_v0 = smem_desc(sbase + OFF_V, 16, 1024, SWZ_128B);
+    const uint32_t id_bf16_pv = idesc_bf16(128, 128, 0, 1);
+    const uint64_t d_v0 = smem_desc(sbase + OFF_V, PVB ? 16384 : 16, 1024, SWZ_128B);
+    const uint64_t d_p0 = smem_desc(sbase + OFF_PS, 16, 1024, SWZ_128B);
+    (void)id_fp8; (void)id_bf16_pv; (void)d_p0;
     bool ok = true;
     uint32_t n_used = 0;   // items so far that used the accumulators (T > 0)
     for (; ok && walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
@@ -444,8 +472,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       for (int t = 0; t < tl.T && ok; ++t) {
         const uint32_t c = gb + t;
         TR(1, c, 0);
-        const uint32_t sb = c & 1, vs = c % VSTAGES;
-        ok = cx.wait(BAR_V_FULL + vs, (c / VSTAGES) & 1u);
+        const uint32_t sb = c & 1, vs = c % VST;
+        ok = cx.wait(BAR_V_FULL + vs, (c / VST) & 1u);
         TR(1, c, 1);
         ok = ok && cx.wait(BAR_O_READY + sb, (c >> 1) & 1u);
         TR(1, c, 2);
@@ -455,14 +483,24 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         tc_fence_after();
         const uint32_t tP = tm + (sb ? TM_P1 : TM_P0);
         const uint32_t tOacc = tm + (sb ? TM_O1 : TM_O0);
-        const uint64_t d_v = d_v0 + (uint64_t)((vs * 16384) >> 4);
+        const uint64_t d_v = d_v0 + (uint64_t)((vs * V_BYTES) >> 4);
         if (elect_one()) {
+          if constexpr (PVB) {
+            // BF16: A = P of this group from shared memory (K-major, two 64-key halves of 16 KB), B = V (MN-major,
+            // two 64-channel halves of 16 KB, 16 keys = 2 KB per K step)
+            const uint64_t d_p = d_p0 + (uint64_t)((sb * 32768) >> 4);
+#pragma unroll
+            for (int k16 = 0; k16 < 8; ++k16)
+              mma_bf16_ss(tOacc, d_p + (uint64_t)(((k16 >> 2) * 16384 + (k16 & 3) * 32) >> 4), d_v + (uint64_t)((2048 * k16) >> 4),
+                          id_bf16_pv, (t >= 2 || k16 > 0) ? 1u : 0u);
+          } else {
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
 #ifdef MPFA_ABLATE_NO_PV
             if (k4 > 100)
 #endif
             mma_e4m3_ts(tOacc, tP + 8 * k4, d_v + (uint64_t)((4096 * k4) >> 4), id_fp8, (t >= 2 || k4 > 0) ? 1u : 0u);
+          }
           mma_commit(cx.bar(BAR_O_FULL + sb));
           mma_commit(cx.bar(BAR_P_EMPTY + sb));
           mma_commit(cx.bar(BAR_V_EMPTY + vs));
@@ -480,6 +518,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     float *s_m = reinterpret_cast<float *>(smem + OFF_M);
     const uint32_t tS = tm + TM_S + lane_off;
     const uint32_t tP = tm + (grp ? TM_P1 : TM_P0) + lane_off;
+    uint8_t *const ps_row = smem + OFF_PS + grp * 32768 + row * 128;   // PVB: this thread's row of the group's P operand
+    (void)tP; (void)ps_row;
     bool ok = true;
     uint32_t n_used = 0;   // items so far with T > 0: only those go through the row-sum ring
     for (; ok && walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
@@ -613,7 +653,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const float a_own = (m_t == m_own) ? 1.0f : ex2_approx(__fmul_rn(m_own - m_t, lam));
         // P = 2^(lam S - lam m) (Eq. 4)
         // the factor 448 of the E4M3 operand is folded into the exponent: q = 448 P = 2^(lam S - lam m + log2 448)
-        const float cc = (m_t == -INFINITY) ? 0.0f : __fsub_rn(8.8073549220576042f, __fmul_rn(m_t, lam));
+        const float cc = (m_t == -INFINITY) ? 0.0f : __fsub_rn(PVB ? 0.0f : 8.8073549220576042f, __fmul_rn(m_t, lam));
         float sum0 = 0.0f, sum1 = 0.0f, sum2 = 0.0f, sum3 = 0.0f;
 #ifdef MPFA_ABLATE_NO_SOFTMAX
         sum0 = __uint_as_float(s[5]);
@@ -630,6 +670,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
           for (int c0 = 0; c0 < 128; c0 += 32) {
             uint32_t packed[8];
+            uint32_t pbf[4];
+            (void)packed; (void)pbf;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               float x0, x1, x2, x3;
@@ -638,6 +680,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
               const float q0 = EX2_(x0), q1 = EX2_(x1), q2 = EX2_(x2), q3 = EX2_(x3);
               acc2(sum0, sum1, q0, q1);
               acc2(sum2, sum3, q2, q3);
+              if constexpr (PVB) {
+                // BF16 pairs (first operand of the conversion goes to the upper half)
+                asm("cvt.rn.bf16x2.f32 %0, %2, %1;" : "=r"(pbf[2 * (i & 1)]) : "f"(q0), "f"(q1));
+                asm("cvt.rn.bf16x2.f32 %0, %2, %1;" : "=r"(pbf[2 * (i & 1) + 1]) : "f"(q2), "f"(q3));
+                if (i & 1) {
+                  // eight keys = one 16-byte chunk of the row in the K-major, 128B-swizzled A operand
+                  const int ch = (c0 >> 3) + (i >> 1);
+                  *reinterpret_cast<uint4 *>(ps_row + (ch >> 3) * 16384 + (((ch & 7) ^ (row & 7)) << 4)) =
+                      make_uint4(pbf[0], pbf[1], pbf[2], pbf[3]);
+                }
+              } else {
               // two conversions written into the halves of one register (no separate merge instruction)
               asm("{.reg .b16 lo, hi;\n\t"
                   "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
@@ -645,18 +698,25 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                   "mov.b32 %0, {lo, hi};}"
                   : "=r"(packed[i])
                   : "f"(q0), "f"(q1), "f"(q2), "f"(q3));
+              }
             }
+            if constexpr (!PVB) {
 #ifndef MPFA_ABLATE_NO_PST
             tmem_st8(tP + (c0 >> 2), packed);
 #else
             if (packed[0] == 0x12345u && packed[7] == 77u) tmem_st8(tP + (c0 >> 2), packed);
 #endif
+            }
           }
         }
         l_own = __fadd_rn(__fmul_rn(a_own, l_own), (sum0 + sum1) + (sum2 + sum3));
         m_own = m_t;
         TR(2 + grp, c, 5);
-        tmem_st_wait();
+        if constexpr (PVB) {
+          fence_proxy_async_smem();   // the P rows were written through the generic proxy, the MMA reads them through the async one
+        } else {
+          tmem_st_wait();
+        }
         tc_fence_before();
         warp_arrive(cx.bar(BAR_P_FULL + grp), lane);
         TR(2 + grp, c, 6);
@@ -836,8 +896,9 @@ extern "C" mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *q, const mpfa
                                             const void *delta_s_bf16, const mpfa_stats *st, float v_scale, int causal,
                                             float softmax_scale, int variant, void *out_bf16, float *out_f32,
                                             int32_t *device_status, void *stream) {
-  if (variant != 0 && variant != MPFA_VARIANT_COMP_ELEMENTWISE) return MPFA_ERR_INVALID_ARG;
+  if (variant != 0 && variant != MPFA_VARIANT_COMP_ELEMENTWISE && variant != MPFA_VARIANT_PV_BF16) return MPFA_ERR_INVALID_ARG;
   const bool ew = variant == MPFA_VARIANT_COMP_ELEMENTWISE && delta_s_bf16 != nullptr;
+  const bool pvb = variant == MPFA_VARIANT_PV_BF16;   // v_fp8 then points at the BF16 tile tensor of mpfa_pack_v_bf16
   if (!q || !k || !v_fp8 || !st || !out_bf16 || !device_status) return MPFA_ERR_INVALID_ARG;
   if (!q->codes || !q->sf || !k->codes || !k->sf || !st->q_gscale || !st->k_gscale) return MPFA_ERR_INVALID_ARG;
   if (q->B <= 0 || q->B != k->B || q->H <= 0 || k->H <= 0 || q->N <= 0 || k->N <= 0) return MPFA_ERR_INVALID_ARG;
@@ -873,24 +934,27 @@ extern "C" mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *q, const mpfa
   p.softmax_scale = softmax_scale;
   p.v_scale = v_scale;
   p.n_items = (int)n_cta;
-  if (g_arrangement == 1) return launch_prefill_pair(q, k, v_fp8, p, ew, static_cast<cudaStream_t>(stream));
+  if (g_arrangement == 1 && !pvb) return launch_prefill_pair(q, k, v_fp8, p, ew, static_cast<cudaStream_t>(stream));
   EncodeTiledFn enc;
   rc = get_encoder(&enc);
   if (rc != MPFA_OK) return rc;
   CUtensorMap tq, tk, tv;
   if ((rc = make_map(enc, &tq, q->codes, q_rows, 64)) != MPFA_OK) return rc;
   if ((rc = make_map(enc, &tk, k->codes, k_rows, 64)) != MPFA_OK) return rc;
-  if ((rc = make_map(enc, &tv, v_fp8, k_rows, 128)) != MPFA_OK) return rc;
+  if ((rc = pvb ? make_map(enc, &tv, v_fp8, k_rows, 256, 128) : make_map(enc, &tv, v_fp8, k_rows, 128)) != MPFA_OK) return rc;
   int dev = 0, n_sm = 0;
   MPFA_CUDA_OK(cudaGetDevice(&dev));
   MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
   const unsigned grid = (unsigned)(n_cta < (uint64_t)n_sm ? n_cta : (uint64_t)n_sm);   // one persistent CTA per SM
-  if (ew) {
-    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-    prefill_kernel<false, true><<<grid, NTHREADS, SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+  if (pvb) {
+    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<true>::SMEM_BYTES));
+    prefill_kernel<false, false, true><<<grid, NTHREADS, Lay<true>::SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+  } else if (ew) {
+    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::SMEM_BYTES));
+    prefill_kernel<false, true><<<grid, NTHREADS, Lay<false>::SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
   } else {
-    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-    prefill_kernel<false, false><<<grid, NTHREADS, SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::SMEM_BYTES));
+    prefill_kernel<false, false><<<grid, NTHREADS, Lay<false>::SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
   }
   MPFA_LAUNCH_OK();
   return MPFA_OK;
@@ -957,8 +1021,8 @@ extern "C" mpfa_status mpfa_prefill_paged(const mpfa_fp4_tensor *q, const mpfa_p
   MPFA_CUDA_OK(cudaGetDevice(&dev));
   MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
   const unsigned grid = (unsigned)(n_cta < (uint64_t)n_sm ? n_cta : (uint64_t)n_sm);
-  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES_PAGED));
-  prefill_kernel<true, false><<<grid, NTHREADS, SMEM_BYTES_PAGED, static_cast<cudaStream_t>(stream)>>>(tq, tq, tq, p, pg);
+  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::SMEM_BYTES_PAGED));
+  prefill_kernel<true, false><<<grid, NTHREADS, Lay<false>::SMEM_BYTES_PAGED, static_cast<cudaStream_t>(stream)>>>(tq, tq, tq, p, pg);
   MPFA_LAUNCH_OK();
   return MPFA_OK;
 }

@@ -185,14 +185,16 @@ mpfa_status get_encoder(EncodeTiledFn *fn) {
   return MPFA_OK;
 }
 
-// 2D byte tensor [rows][row_bytes], box = 128 rows x row_bytes, hardware swizzle = row_bytes.
-mpfa_status make_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, uint64_t rows, uint32_t row_bytes) {
+// 2D byte tensor [rows][row_bytes], box = 128 rows x box_bytes (default: the whole row), hardware swizzle = box_bytes.
+inline mpfa_status make_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, uint64_t rows, uint32_t row_bytes,
+                            uint32_t box_bytes = 0) {
+  if (box_bytes == 0) box_bytes = row_bytes;
   cuuint64_t dims[2] = {row_bytes, rows};
   cuuint64_t strides[1] = {row_bytes};
-  cuuint32_t box[2] = {row_bytes, 128};
+  cuuint32_t box[2] = {box_bytes, 128};
   cuuint32_t es[2] = {1, 1};
   CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, es,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     g_last_cuda_error = (int)r;

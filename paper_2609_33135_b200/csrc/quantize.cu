@@ -548,6 +548,23 @@ __global__ void __launch_bounds__(256) quantize_v_tile_kernel(const __nv_bfloat1
   }
 }
 
+// grid (N_pad/128, H, B): V tile -> [B, H, N_pad, 128] BF16, unchanged values (the NVFP4 + BF16 precision assignment
+// of Section 3.1 reads V in BF16); pad rows zero.
+__global__ void __launch_bounds__(256) pack_v_bf16_kernel(const __nv_bfloat16 *__restrict__ v, int N, int H,
+                                                          __nv_bfloat16 *__restrict__ out) {
+  const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int n_pad = gridDim.x * TILE;
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int id = it * 256 + threadIdx.x;
+    const int r = id >> 4, seg = id & 15;
+    const int t = tile * TILE + r;
+    uint4 c = make_uint4(0u, 0u, 0u, 0u);
+    if (t < N) c = *reinterpret_cast<const uint4 *>(v + (((size_t)b * N + t) * H + h) * HEAD_DIM + seg * 8);
+    *reinterpret_cast<uint4 *>(out + (((size_t)b * H + h) * n_pad + t) * HEAD_DIM + seg * 8) = c;
+  }
+}
+
 // Paged cache write for one request: grid (pages, H_kv).  K and V of one (page, head) are
 // quantized into shared memory in the byte order of the decode kernel's shared-memory operand
 // tiles (so that decode fills a tile with one bulk copy) and copied out with 16-byte stores.
@@ -861,6 +878,17 @@ extern "C" mpfa_status mpfa_quantize_v(const void *v_bf16, int B, int N_kv, int 
   dim3 grid(pad128(N_kv) / TILE, H_kv, B);
   quantize_v_tile_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16 *>(v_bf16), N_kv, H_kv, 1.0f / v_scale, v_fp8);
+  MPFA_LAUNCH_OK();
+  return MPFA_OK;
+}
+
+extern "C" mpfa_status mpfa_pack_v_bf16(const void *v_bf16, int B, int N_kv, int H_kv, void *v_tiles_bf16, void *stream) {
+  if (!v_bf16 || !v_tiles_bf16 || B <= 0 || N_kv <= 0 || H_kv <= 0) return MPFA_ERR_INVALID_ARG;
+  if (!aligned(v_bf16, 16) || !aligned(v_tiles_bf16, 1024)) return MPFA_ERR_ALIGNMENT;
+  mpfa_status rc = check_arch();
+  if (rc != MPFA_OK) return rc;
+  pack_v_bf16_kernel<<<dim3(pad128(N_kv) / TILE, H_kv, B), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16 *>(v_bf16), N_kv, H_kv, static_cast<__nv_bfloat16 *>(v_tiles_bf16));
   MPFA_LAUNCH_OK();
   return MPFA_OK;
 }

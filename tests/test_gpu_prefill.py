@@ -247,3 +247,47 @@ def test_two_tile_arrangement_sampled_rows_and_empty_items(two_tile_arrangement)
     o16, o32 = run_gpu(w)
     compare(o16, o32, rows, ref32, "4k+128, two tiles per CTA")
     test_prefill_many_items_without_keys_per_cta()
+
+
+@pytest.mark.parametrize("name", ["cfg1b_qbias", "causal_384_gqa", "ragged_causal", "ragged_noncausal_nq_lt_nkv",
+                                  "causal_offset", "many_short_items"])
+def test_prefill_bf16_pv_variant_matches_its_oracle(name):
+    """Section 3.1's NVFP4 + BF16 precision assignment (mpfa_prefill_variant, MPFA_VARIANT_PV_BF16): the same logits,
+    P in BF16, V unquantized.  Held to the same tolerance against the oracle's statement of that assignment; a BF16
+    rounding of P is a 2^-9 step, and 2^x within 2 ulp cannot move it except on a boundary, as for the FP8 codes."""
+    from paper_2609_33135_b200 import binding as B_
+    w = CASES[name]()
+    s1 = B_.stage1(w.q.cuda(), w.k.cuda(), w.v.cuda())
+    vt = B_.mpfa_pack_v_bf16(w.v.cuda())
+    out = torch.empty(w.B, w.N_q, w.H_q, 128, dtype=torch.bfloat16, device="cuda")
+    o32 = torch.empty(w.B, w.N_q, w.H_q, 128, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B_.mpfa_prefill_variant(s1.q, s1.k, vt, s1.delta, s1.stats, 1.0, w.causal, w.softmax_scale, B_.MPFA_VARIANT_PV_BF16,
+                            out, o32, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+    rows = orc.all_rows(w.B, w.H_q, w.N_q)
+    ref32, _ = orc.prefill_rows_pv_bf16(z, orc.bf16_bits(w.v), rows, w.softmax_scale, w.causal)
+    compare(out.view(torch.uint16).cpu().numpy(), o32.cpu().numpy(), rows, ref32, name + " (BF16 P V)")
+    # and it is a different function from the product path
+    m32, _ = orc.prefill_rows(z, rows, w.softmax_scale, w.causal)
+    assert np.abs(m32 - ref32).mean() > 1e-4
+
+
+def test_prefill_bf16_pv_variant_sampled_rows_4k():
+    from paper_2609_33135_b200 import binding as B_
+    w = wl.prefill_workload("mid3", 63, 1, 4096, 8, 2, True, q_bias=True)
+    s1 = B_.stage1(w.q.cuda(), w.k.cuda(), w.v.cuda())
+    vt = B_.mpfa_pack_v_bf16(w.v.cuda())
+    out = torch.empty(w.B, w.N_q, w.H_q, 128, dtype=torch.bfloat16, device="cuda")
+    o32 = torch.empty(w.B, w.N_q, w.H_q, 128, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B_.mpfa_prefill_variant(s1.q, s1.k, vt, s1.delta, s1.stats, 1.0, True, w.softmax_scale, B_.MPFA_VARIANT_PV_BF16, out, o32,
+                            status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    z = orc.stage1(orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v))
+    rows = wl.sample_rows(63, w.B, w.H_q, w.N_q, 256).numpy()
+    ref32, _ = orc.prefill_rows_pv_bf16(z, orc.bf16_bits(w.v), rows, w.softmax_scale, True)
+    compare(out.view(torch.uint16).cpu().numpy(), o32.cpu().numpy(), rows, ref32, "4k (BF16 P V)")
