@@ -25,6 +25,12 @@
 //                (Eq. 6), and at the end of an item O_r / (448 l) * v_scale -> BF16 (Algorithm 1 line 17).
 // Tensor memory (496 of 512 columns): S [0,128), O_0 [128,256), O_1 [256,384), P_hat_0 [384,416), P_hat_1 [416,448),
 // scale factors of 2 x 2 query tiles [448,480) and of two K blocks [480,496).
+// Measured on B200 against the one-query-tile kernel of prefill.cu (same arithmetic row by row): 1046 against 1273
+// TFLOPS at 16K, 1142 against 1397 at 64K, although this kernel executes 12 % fewer instructions per block.  With the
+// rescaling of O compiled out both take the same time; with it, one accumulator per tile puts the rescale between two
+// dependent P V MMAs of that tile (the other kernel alternates two accumulators), and at these lengths some row of a
+// warp moves its maximum in most blocks.  This arrangement is therefore not the default
+// (mpfa_set_prefill_arrangement).
 // Template parameter EW: the compensation-placement ablation (no seed MMA, Delta_S added element by element by the
 // softmax threads).  Every mbarrier wait is bounded; on expiry the CTA raises MPFA_DEV_TIMEOUT in *device_status,
 // all roles leave their loops, outstanding TMA copies are drained and tensor memory is released.
