@@ -415,29 +415,20 @@ __global__ void __launch_bounds__(256) quantize_fp4_tile_kernel(const QuantTenso
     quantize_tile_body(a1.x, a1.mean, a1.gscale, a1.N, a1.H, a1.tiles, a1.codes, a1.sf, y - a0.H, tile);
 }
 
-// grid (tiles * (H_kv + H_q), 1, B), KTILE_SMEM bytes of dynamic shared memory: K tiles with Delta_S and, when
-// aq.H > 0, the Q tiles in the same launch (same block order: tile-major, K head of a group then its G query heads).
-__global__ void __launch_bounds__(256) quantize_k_delta_kernel(const QuantTensor a, const DeltaArgs da, const QuantTensor aq) {
+// grid (tiles * H_kv, 1, B), KTILE_SMEM bytes of dynamic shared memory: K tiles with Delta_S, blockIdx.x = tile * H_kv +
+// head.  A launch of its own: these blocks are bound by the FP64 pipe, the Q tiles by memory, and in one launch
+// (kinds interleaved) they only competed for block slots (98 us against 42 + 38 at 16K).
+__global__ void __launch_bounds__(256) quantize_k_delta_kernel(const QuantTensor a, const DeltaArgs da) {
   extern __shared__ __align__(16) uint8_t dyn_smem[];
-  const int heads = a.H + aq.H;
-  const int tile = (int)blockIdx.x / heads, y = (int)blockIdx.x % heads;
-  if (aq.H == 0) {
-    quantize_k_tile_delta_body(a, da, y, tile, dyn_smem);
-    return;
-  }
-  const int G = aq.H / a.H;
-  const int grp = y / (G + 1), r = y % (G + 1);
-  if (r == 0)
-    quantize_k_tile_delta_body(a, da, grp, tile, dyn_smem);
-  else
-    quantize_tile_body(aq.x, aq.mean, aq.gscale, aq.N, aq.H, aq.tiles, aq.codes, aq.sf, grp * G + r - 1, tile);
+  quantize_k_tile_delta_body(a, da, (int)blockIdx.x % a.H, (int)blockIdx.x / a.H, dyn_smem);
 }
 
 // Eq. 9: Delta_S[hq][t] = qmean[hq] . (k[t] - kmean), FP64 accumulation with channels ascending,
 // expressed in units of gscale_q * gscale_k and rounded once to BF16.  Two threads per key token
 // (256 threads per 128-token tile): thread (key, part) takes the heads g = part, part + 2, ... of the
-// group, each as its own sequential chain.  grid (N_pad/128, H_kv, B).  dst_stride / dst_base let the same
-// kernel write the dense [B, H_q, N_pad] vector or one page of the paged side cache.
+// group, each as its own sequential chain.  grid (N_pad/128, H_kv, B).  Used for the paged side cache (PAGED: the
+// entries go to their page through the page-table row); the dense vector of mpfa_quantize_qk comes out of
+// quantize_k_delta_kernel, which runs the same chains on rows it has already staged.
 template <bool PAGED>
 __global__ void __launch_bounds__(256) delta_s_kernel(const __nv_bfloat16 *__restrict__ k,
                                                       const float *__restrict__ q_mean,
@@ -852,14 +843,10 @@ extern "C" mpfa_status mpfa_quantize_qk(const void *q_bf16, const void *k_bf16, 
     if (with_delta) {
       DeltaArgs da{st->q_mean, st->q_gscale, static_cast<__nv_bfloat16 *>(delta_s_bf16), H_q};
       MPFA_CUDA_OK(cudaFuncSetAttribute(quantize_k_delta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KTILE_SMEM));
-      const bool both = false;      // measured: in one launch the two kinds only compete for block slots (98 us against 40 + 37)
-      QuantTensor none{};
-      quantize_k_delta_kernel<<<dim3(std::max(tk.tiles, both ? tq.tiles : 0) * (tk.H + (both ? tq.H : 0)), 1, B), 256, KTILE_SMEM,
-                                s>>>(tk, da, both ? tq : none);
+      quantize_k_delta_kernel<<<dim3(tk.tiles * tk.H, 1, B), 256, KTILE_SMEM, s>>>(tk, da);
       MPFA_LAUNCH_OK();
       tk.H = 0;
       tk.tiles = 0;
-      if (both) tq.H = 0, tq.tiles = 0;
     }
     if (tq.H + tk.H > 0) {
       quantize_fp4_tile_kernel<<<dim3(std::max(tq.tiles, tk.tiles) * (tq.H + tk.H), 1, B), 256, 0, s>>>(tq, tk);
