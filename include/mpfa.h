@@ -128,7 +128,9 @@ typedef struct {
  *   k_bf16 [B, N_kv, H_kv, 128] or NULL (quantize Q only);
  *   q_out / k_out: tile-layout tensors with B, H, N filled in by the caller;
  *   delta_s_bf16 [B, H_q, N_kv_pad]: required iff MPFA_SMOOTH and k_bf16 != NULL;
- *   workspace: 256-byte aligned scratch, overwritten by every call (not needed with MPFA_STATS_FROZEN).
+ *   workspace: 256-byte aligned scratch, overwritten by every call (not needed with MPFA_STATS_FROZEN).  The call
+ *          enqueues one memory-set node over its first few hundred bytes (maxima and block counters) and four
+ *          kernels; two calls that overlap on the GPU need separate workspaces.
  *          mpfa_quantize_workspace_bytes() is the size that lets the statistics pass cut the token axis into
  *          its full 32 slices; any size down to mpfa_quantize_workspace_min_bytes() (one slice) is accepted and
  *          only lowers the parallelism of that pass; less: MPFA_ERR_WORKSPACE.
