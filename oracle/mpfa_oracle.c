@@ -18,7 +18,8 @@
  * attention, softmax rows summing to one, traversal-order invariance in FP64;
  * the reverse block order, the fixed scale 448 of P-hat (codes of a worked row,
  * subnormal codes included) and the GQA head mapping against NumPy statements
- * of the same steps on operands built code by code.
+ * of the same steps on operands built code by code; the NVFP4 + NVFP4 assignment
+ * (token-axis V quantizer, block-scaled P) against NumPy statements of its steps.
  * Parity unpinned (the paper prints no worked example for them, they are
  * readings fixed by this file): the per-tensor scale recipe, reciprocal-multiply
  * element scaling, the unit in which the compensation vector is stored, FP32
@@ -675,6 +676,141 @@ void mpfa_oracle_prefill_rows_pv_bf16(const uint8_t *q_codes, const uint8_t *q_s
       out_bf16[(size_t)r * D + c] = mpfa_oracle_f32_to_bf16(x);
     }
     free(p);
+    free(s);
+  }
+}
+
+/* ------------------------------------------------------------------------- */
+/* precision-assignment variant: NVFP4 Q K^T with NVFP4 P V (Section 3.1)     */
+/* ------------------------------------------------------------------------- */
+
+/* V for a block-scaled second MMA: the contraction runs over the keys, so the 16-element blocks of
+ * Eq. 1 lie along the token axis (tokens 16 g .. 16 g + 15 of one channel; tokens past N count as zero).
+ * Same recipe as the Q/K quantizer with the caller's tensor scale d in place of a statistic and no
+ * centering:  r = amax / (6 d);  sc = E4M3(r);  s = decode(sc) d;  code = E2M1(x (1 / s)).
+ * v: BF16 [B, N, H, D];  codes: [B, H, D, NB, 8] (NB = ceil(N / 16); two E2M1 codes per byte, the even
+ * token of the block in the low nibble);  sf: [B, H, D, NB]. */
+void mpfa_oracle_quantize_v_fp4(const uint16_t *v, int B, int N, int H, float d, uint8_t *codes, uint8_t *sf) {
+  int NB = (N + G - 1) / G;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int b = 0; b < B; ++b)
+    for (int h = 0; h < H; ++h)
+      for (int c = 0; c < D; ++c)
+        for (int g = 0; g < NB; ++g) {
+          float x[G];
+          float a = 0.0f;
+          for (int i = 0; i < G; ++i) {
+            int t = g * G + i;
+            x[i] = t < N ? mpfa_oracle_bf16_to_f32(v[(((size_t)b * N + t) * H + h) * D + c]) : 0.0f;
+            if (fabsf(x[i]) > a) a = fabsf(x[i]);
+          }
+          float e = 6.0f * d;
+          float r = a / e;
+          uint8_t sc = mpfa_oracle_e4m3_encode(r);
+          float s = mpfa_oracle_e4m3_decode(sc) * d;
+          float inv = 1.0f / s;
+          if (!(s > 0.0f) || isinf(inv)) inv = 0.0f;
+          size_t blk = (((size_t)b * H + h) * D + c) * NB + g;
+          sf[blk] = sc;
+          for (int i = 0; i < G; i += 2) {
+            uint8_t lo = mpfa_oracle_e2m1_encode(x[i] * inv);
+            uint8_t hi = mpfa_oracle_e2m1_encode(x[i + 1] * inv);
+            codes[blk * (G / 2) + i / 2] = (uint8_t)(lo | (hi << 4));
+          }
+        }
+}
+
+/* The fourth precision assignment of Section 3.1 / 7.2: logits as in the method; P and V both enter the
+ * second MMA as NVFP4 operands.  The paper gives no arithmetic for it; reading taken, per KV block
+ * (reverse order) and row:
+ *   m_new, alpha, P = 2^(lam S - lam m_new), l = alpha l + sum P           as in the method;
+ *   q = 448 P (P <= 1, so the tensor scale of P is fixed at 1 / (6 * 448) and needs no statistic, like the
+ *   fixed 448 of the FP8 path: a block's scale amax_P / (6 d_P) is then 448 amax_P = max q <= 448);
+ *   per 16 keys (blocks aligned to multiples of 16; keys the row cannot see count as 0):
+ *     sc = E4M3(max q);  s = decode(sc);  code_j = E2M1(q_j (6 / s))     (6 / s = 0 when s = 0);
+ *   O = alpha O + sum over the 16-key blocks of (s s_V[c]) * sum_j code_j vcode_j[c]
+ *       (the block-scaled MMA: exact 16-term dot product, one scale product per block, FP32 adds, blocks
+ *       ascending);
+ *   out = O / (6 * 448 * l) * d_V.
+ * v_codes / v_sf: as written by mpfa_oracle_quantize_v_fp4 for the same N = Nkv.
+ * Inspection outputs (optional): pcodes_out [n_rows, Nkv] E2M1 codes of P, psf_out [n_rows, ceil(Nkv/16)]. */
+void mpfa_oracle_prefill_rows_pv_fp4(const uint8_t *q_codes, const uint8_t *q_sf, const uint8_t *k_codes,
+                                     const uint8_t *k_sf, const uint8_t *v_codes, const uint8_t *v_sf,
+                                     const uint16_t *delta, const float *dq, const float *dk, float v_gscale,
+                                     float softmax_scale, int causal, int Nq, int Nkv, int Hq, int Hkv, int block_kv,
+                                     const int32_t *rows, int n_rows, float *out_f32, uint16_t *out_bf16,
+                                     uint8_t *pcodes_out, uint8_t *psf_out) {
+  init_tables();
+  int grp = Hq / Hkv;
+  int NB = (Nkv + G - 1) / G;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int r = 0; r < n_rows; ++r) {
+    int b = rows[3 * r], hq = rows[3 * r + 1], i = rows[3 * r + 2];
+    int hk = hq / grp;
+    int n = visible_keys(i, Nq, Nkv, causal);
+    float *s = (float *)malloc(sizeof(float) * (size_t)(n > 0 ? n : 1));
+    float *q = (float *)malloc(sizeof(float) * (size_t)(block_kv + G));
+    logits_row_q4(q_codes + (((size_t)b * Hq + hq) * Nq + i) * (D / 2), q_sf + (((size_t)b * Hq + hq) * Nq + i) * NBLK,
+                  k_codes + ((size_t)b * Hkv + hk) * Nkv * (D / 2), k_sf + ((size_t)b * Hkv + hk) * Nkv * NBLK,
+                  delta ? delta + ((size_t)b * Hq + hq) * Nkv : NULL, n, s);
+    if (pcodes_out) memset(pcodes_out + (size_t)r * Nkv, 0, (size_t)Nkv);
+    if (psf_out) memset(psf_out + (size_t)r * NB, 0, (size_t)NB);
+    float lam = ((softmax_scale * 1.4426950408889634f) * dq[b]) * dk[b];
+    float m = -INFINITY, l = 0.0f, o[D];
+    for (int c = 0; c < D; ++c) o[c] = 0.0f;
+    const uint8_t *vc = v_codes + ((size_t)b * Hkv + hk) * D * NB * (G / 2);
+    const uint8_t *vs = v_sf + ((size_t)b * Hkv + hk) * D * NB;
+    for (int jb = n > 0 ? (n - 1) / block_kv : -1; jb >= 0; --jb) {
+      int a = jb * block_kv, e = (jb + 1) * block_kv > n ? n : (jb + 1) * block_kv;
+      float rowmax = -INFINITY;
+      for (int j = a; j < e; ++j)
+        if (s[j] > rowmax) rowmax = s[j];
+      float m_new = m > rowmax ? m : rowmax;
+      if (m_new == -INFINITY) continue;
+      float mlam = m_new * lam;
+      float alpha = (m == -INFINITY) ? 0.0f : exp2_f32((m - m_new) * lam);
+      float rowsum = 0.0f;
+      for (int j = a; j < e; ++j) {
+        float p = exp2_f32(fmaf(s[j], lam, -mlam));
+        rowsum += p;
+        q[j - a] = p * 448.0f;
+      }
+      for (int j = e; j < a + block_kv + G; ++j) q[j - a] = 0.0f;   /* keys the row cannot see */
+      l = alpha * l + rowsum;
+      for (int c = 0; c < D; ++c) o[c] = alpha * o[c];
+      for (int g0 = a; g0 < e; g0 += G) {                         /* a is a multiple of 16 */
+        float amax = 0.0f;
+        for (int j = 0; j < G; ++j)
+          if (q[g0 - a + j] > amax) amax = q[g0 - a + j];
+        uint8_t sc = mpfa_oracle_e4m3_encode(amax);
+        float sp = e4m3_tab[sc];
+        float inv = sp > 0.0f ? 6.0f / sp : 0.0f;
+        float pv[G];
+        for (int j = 0; j < G; ++j) {
+          uint8_t code = mpfa_oracle_e2m1_encode(q[g0 - a + j] * inv);
+          pv[j] = mpfa_oracle_e2m1_decode(code);
+          if (pcodes_out && g0 + j < Nkv) pcodes_out[(size_t)r * Nkv + g0 + j] = code;
+        }
+        if (psf_out) psf_out[(size_t)r * NB + g0 / G] = sc;
+        int gi = g0 / G;
+        for (int c = 0; c < D; ++c) {
+          const uint8_t *vb = vc + ((size_t)c * NB + gi) * (G / 2);
+          float dot = 0.0f;
+          for (int j = 0; j < G / 2; ++j) {
+            dot += pv[2 * j] * e2m1_pair_lo[vb[j]];
+            dot += pv[2 * j + 1] * e2m1_pair_hi[vb[j]];
+          }
+          o[c] += (sp * e4m3_tab[vs[(size_t)c * NB + gi]]) * dot;
+        }
+      }
+      m = m_new;
+    }
+    for (int c = 0; c < D; ++c) {
+      float x = (l > 0.0f) ? o[c] / (2688.0f * l) * v_gscale : 0.0f;
+      out_f32[(size_t)r * D + c] = x;
+      out_bf16[(size_t)r * D + c] = mpfa_oracle_f32_to_bf16(x);
+    }
+    free(q);
     free(s);
   }
 }

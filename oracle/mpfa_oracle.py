@@ -299,3 +299,35 @@ def prefill_rows_pv_bf16(z: Quantized, v_bits: np.ndarray, rows, softmax_scale: 
                                            _p(_c(z.dk, np.float32)), ctypes.c_float(softmax_scale), int(causal), Nq, Nkv,
                                            Hq, Hkv, block_kv, _p(rows), n, _p(o32), _p(o16))
     return o32, o16
+
+
+def quantize_v_fp4(v: np.ndarray, d: float):
+    """V for the NVFP4 + NVFP4 assignment (Section 3.1): 16-token blocks along the key axis, tensor scale d.
+    -> (codes uint8 [B,H,128,NB,8], sf uint8 [B,H,128,NB]), NB = ceil(N/16)."""
+    B, N, H, _ = v.shape
+    NB = (N + 15) // 16
+    codes = np.empty((B, H, D, NB, 8), np.uint8)
+    sf = np.empty((B, H, D, NB), np.uint8)
+    lib().mpfa_oracle_quantize_v_fp4(_p(v), B, N, H, ctypes.c_float(d), _p(codes), _p(sf))
+    return codes, sf
+
+
+def prefill_rows_pv_fp4(z: Quantized, v_codes: np.ndarray, v_sf: np.ndarray, v_gscale: float, rows, softmax_scale: float,
+                        causal: bool, block_kv: int = BLOCK_KV, use_delta: bool = True, want_codes: bool = False):
+    """Precision-assignment variant of Section 3.1: NVFP4 logits as in the method, P and V as NVFP4 operands of the
+    second MMA.  -> (FP32 [n,128], BF16 bits [n,128]) and, with want_codes, the E2M1 codes [n,Nkv] and E4M3 block
+    scales [n,ceil(Nkv/16)] of P."""
+    rows = _c(rows, np.int32)
+    B, Hq, Nq, _ = z.q_codes.shape
+    Hkv, Nkv = z.k_codes.shape[1], z.k_codes.shape[2]
+    n = rows.shape[0]
+    o32 = np.empty((n, D), np.float32)
+    o16 = np.empty((n, D), np.uint16)
+    pc = np.empty((n, Nkv), np.uint8) if want_codes else None
+    ps = np.empty((n, (Nkv + 15) // 16), np.uint8) if want_codes else None
+    lib().mpfa_oracle_prefill_rows_pv_fp4(_p(z.q_codes), _p(z.q_sf), _p(z.k_codes), _p(z.k_sf), _p(_c(v_codes, np.uint8)),
+                                          _p(_c(v_sf, np.uint8)), _p(z.delta if use_delta else None),
+                                          _p(_c(z.dq, np.float32)), _p(_c(z.dk, np.float32)), ctypes.c_float(v_gscale),
+                                          ctypes.c_float(softmax_scale), int(causal), Nq, Nkv, Hq, Hkv, block_kv, _p(rows), n,
+                                          _p(o32), _p(o16), _p(pc), _p(ps))
+    return (o32, o16, pc, ps) if want_codes else (o32, o16)
