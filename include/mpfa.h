@@ -182,6 +182,18 @@ mpfa_status mpfa_quantize_v(const void *v_bf16, int B, int N_kv, int H_kv, float
  * [B, N_kv, H_kv, 128] to [B, H_kv, N_kv_pad, 128] BF16 (pad rows zero; 1024-byte aligned, 2 * mpfa_v_fp8_bytes()). */
 mpfa_status mpfa_pack_v_bf16(const void *v_bf16, int B, int N_kv, int H_kv, void *v_tiles_bf16, void *stream);
 
+/* For MPFA_VARIANT_PV_FP4 only (Section 3.1's NVFP4 + NVFP4 assignment): V as the block-scaled FP4 operand of the
+ * second MMA.  That MMA contracts over the keys, so the 16-element blocks of Eq. 1 lie along the TOKEN axis (tokens
+ * 16 g .. 16 g + 15 of one channel; tokens past N_kv count as zero).  Recipe of the Q/K quantizer with the caller's
+ * tensor scale in place of a statistic and no centering: block scale = E4M3(amax / (6 v_gscale)), code =
+ * E2M1(v * (1 / (decode(scale) * v_gscale))); v_gscale = max|V| / (6 * 448) uses the whole range.
+ * v_fp4 (1024-byte aligned, mpfa_v_fp4_bytes()): codes [B, H_kv, N_kv_pad/128, 128 channels, 64 bytes] (two keys per
+ * byte, the even key in the low nibble) followed by the block scales, two 512-byte atoms per (b, h, tile) in the
+ * tcgen05.cp order (atom = 64 keys; byte (channel mod 32) * 16 + (channel / 32) * 4 + block mod 4). */
+size_t mpfa_v_fp4_bytes(int B, int H_kv, int N_kv);
+mpfa_status mpfa_quantize_v_fp4(const void *v_bf16, int B, int N_kv, int H_kv, float v_gscale, uint8_t *v_fp4,
+                                void *stream);
+
 /* The same arithmetic for ONE request, written through its page-table row into the paged
  * cache (Section 6: low-bit K/V cache writes fused with quantization and compensation
  * generation).  k_bf16, v_bf16 [N_tokens, H_kv, 128] are the tokens at positions
@@ -242,8 +254,16 @@ mpfa_status mpfa_prefill(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tensor *h_k,
  *                                         tile tensor [B, H_kv, N_kv_pad, 128] written by mpfa_pack_v_bf16 (1024-byte
  *                                         aligned) and v_scale must be 1.  It exists to measure what FP8 for P V buys
  *                                         (always in the one-query-tile arrangement).
+ *   MPFA_VARIANT_PV_FP4                   the NVFP4 + NVFP4 precision assignment of Section 3.1 / Section 7.2: Q K^T as in
+ *                                         the product path; q = 448 P is quantized per row and 16 keys (block scale
+ *                                         E4M3(max q), codes E2M1(q * (6 / scale)): the tensor scale of P is fixed at
+ *                                         1 / (6 * 448)), written to shared memory as a K-major operand with its scale
+ *                                         factors, and the second MMA is block-scaled FP4 x FP4 on the V operand written
+ *                                         by mpfa_quantize_v_fp4 (passed as the v_fp8 argument; v_scale = the v_gscale
+ *                                         given there).  It exists to reproduce the paper's observation that this
+ *                                         assignment is slower than FP8 for P V (always in the one-query-tile arrangement).
  * Any other value: MPFA_ERR_INVALID_ARG. */
-enum { MPFA_VARIANT_COMP_ELEMENTWISE = 1, MPFA_VARIANT_PV_BF16 = 2 };
+enum { MPFA_VARIANT_COMP_ELEMENTWISE = 1, MPFA_VARIANT_PV_BF16 = 2, MPFA_VARIANT_PV_FP4 = 3 };
 mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *h_q, const mpfa_fp4_tensor *h_k, const uint8_t *v_fp8,
                                  const void *delta_s_bf16, const mpfa_stats *h_stats, float v_scale, int causal,
                                  float softmax_scale, int variant, void *out_bf16, float *out_f32,

@@ -733,13 +733,19 @@ void mpfa_oracle_quantize_v_fp4(const uint16_t *v, int B, int N, int H, float d,
  *       ascending);
  *   out = O / (6 * 448 * l) * d_V.
  * v_codes / v_sf: as written by mpfa_oracle_quantize_v_fp4 for the same N = Nkv.
- * Inspection outputs (optional): pcodes_out [n_rows, Nkv] E2M1 codes of P, psf_out [n_rows, ceil(Nkv/16)]. */
+ * Inspection outputs (optional): pcodes_out [n_rows, Nkv] E2M1 codes of P, psf_out [n_rows, ceil(Nkv/16)] block
+ * scale codes, y_out [n_rows, Nkv] the FP32 values q (6 / s) that were encoded, amax_out [n_rows, ceil(Nkv/16)] the
+ * FP32 block maxima that were encoded.  Inspection switches (-1 everywhere else, where they change nothing):
+ * flip_key >= 0 moves that key's E2M1 code by flip_dir steps; flip_blk >= 0 moves that block's scale code by
+ * flip_blk_dir steps before its codes are made (to show what a one-step difference in a single decision does to a
+ * row). */
 void mpfa_oracle_prefill_rows_pv_fp4(const uint8_t *q_codes, const uint8_t *q_sf, const uint8_t *k_codes,
                                      const uint8_t *k_sf, const uint8_t *v_codes, const uint8_t *v_sf,
                                      const uint16_t *delta, const float *dq, const float *dk, float v_gscale,
                                      float softmax_scale, int causal, int Nq, int Nkv, int Hq, int Hkv, int block_kv,
                                      const int32_t *rows, int n_rows, float *out_f32, uint16_t *out_bf16,
-                                     uint8_t *pcodes_out, uint8_t *psf_out) {
+                                     uint8_t *pcodes_out, uint8_t *psf_out, float *y_out, float *amax_out,
+                                     int flip_key, int flip_dir, int flip_blk, int flip_blk_dir) {
   init_tables();
   int grp = Hq / Hkv;
   int NB = (Nkv + G - 1) / G;
@@ -755,6 +761,8 @@ void mpfa_oracle_prefill_rows_pv_fp4(const uint8_t *q_codes, const uint8_t *q_sf
                   delta ? delta + ((size_t)b * Hq + hq) * Nkv : NULL, n, s);
     if (pcodes_out) memset(pcodes_out + (size_t)r * Nkv, 0, (size_t)Nkv);
     if (psf_out) memset(psf_out + (size_t)r * NB, 0, (size_t)NB);
+    if (y_out) memset(y_out + (size_t)r * Nkv, 0, sizeof(float) * (size_t)Nkv);
+    if (amax_out) memset(amax_out + (size_t)r * NB, 0, sizeof(float) * (size_t)NB);
     float lam = ((softmax_scale * 1.4426950408889634f) * dq[b]) * dk[b];
     float m = -INFINITY, l = 0.0f, o[D];
     for (int c = 0; c < D; ++c) o[c] = 0.0f;
@@ -783,11 +791,21 @@ void mpfa_oracle_prefill_rows_pv_fp4(const uint8_t *q_codes, const uint8_t *q_sf
         for (int j = 0; j < G; ++j)
           if (q[g0 - a + j] > amax) amax = q[g0 - a + j];
         uint8_t sc = mpfa_oracle_e4m3_encode(amax);
+        if (amax_out) amax_out[(size_t)r * NB + g0 / G] = amax;
+        if (g0 / G == flip_blk) {
+          int c2 = (int)sc + flip_blk_dir;
+          sc = (uint8_t)(c2 < 0 ? 0 : (c2 > 0x7E ? 0x7E : c2));
+        }
         float sp = e4m3_tab[sc];
         float inv = sp > 0.0f ? 6.0f / sp : 0.0f;
         float pv[G];
         for (int j = 0; j < G; ++j) {
           uint8_t code = mpfa_oracle_e2m1_encode(q[g0 - a + j] * inv);
+          if (y_out && g0 + j < Nkv) y_out[(size_t)r * Nkv + g0 + j] = q[g0 - a + j] * inv;
+          if (g0 + j == flip_key) {
+            int c2 = (int)code + flip_dir;
+            code = (uint8_t)(c2 < 0 ? 0 : (c2 > 7 ? 7 : c2));
+          }
           pv[j] = mpfa_oracle_e2m1_decode(code);
           if (pcodes_out && g0 + j < Nkv) pcodes_out[(size_t)r * Nkv + g0 + j] = code;
         }

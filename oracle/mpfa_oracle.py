@@ -313,10 +313,12 @@ def quantize_v_fp4(v: np.ndarray, d: float):
 
 
 def prefill_rows_pv_fp4(z: Quantized, v_codes: np.ndarray, v_sf: np.ndarray, v_gscale: float, rows, softmax_scale: float,
-                        causal: bool, block_kv: int = BLOCK_KV, use_delta: bool = True, want_codes: bool = False):
+                        causal: bool, block_kv: int = BLOCK_KV, use_delta: bool = True, want_codes: bool = False,
+                        flip_key: int = -1, flip_dir: int = 0, flip_blk: int = -1, flip_blk_dir: int = 0):
     """Precision-assignment variant of Section 3.1: NVFP4 logits as in the method, P and V as NVFP4 operands of the
     second MMA.  -> (FP32 [n,128], BF16 bits [n,128]) and, with want_codes, the E2M1 codes [n,Nkv] and E4M3 block
-    scales [n,ceil(Nkv/16)] of P."""
+    scales [n,ceil(Nkv/16)] of P, the FP32 values [n,Nkv] the codes were made from and the FP32 block maxima
+    [n,ceil(Nkv/16)] the scales were made from.  flip_*: inspection switches (one decision moved by that many code steps)."""
     rows = _c(rows, np.int32)
     B, Hq, Nq, _ = z.q_codes.shape
     Hkv, Nkv = z.k_codes.shape[1], z.k_codes.shape[2]
@@ -325,9 +327,12 @@ def prefill_rows_pv_fp4(z: Quantized, v_codes: np.ndarray, v_sf: np.ndarray, v_g
     o16 = np.empty((n, D), np.uint16)
     pc = np.empty((n, Nkv), np.uint8) if want_codes else None
     ps = np.empty((n, (Nkv + 15) // 16), np.uint8) if want_codes else None
+    y = np.empty((n, Nkv), np.float32) if want_codes else None
+    am = np.empty((n, (Nkv + 15) // 16), np.float32) if want_codes else None
     lib().mpfa_oracle_prefill_rows_pv_fp4(_p(z.q_codes), _p(z.q_sf), _p(z.k_codes), _p(z.k_sf), _p(_c(v_codes, np.uint8)),
                                           _p(_c(v_sf, np.uint8)), _p(z.delta if use_delta else None),
                                           _p(_c(z.dq, np.float32)), _p(_c(z.dk, np.float32)), ctypes.c_float(v_gscale),
                                           ctypes.c_float(softmax_scale), int(causal), Nq, Nkv, Hq, Hkv, block_kv, _p(rows), n,
-                                          _p(o32), _p(o16), _p(pc), _p(ps))
-    return (o32, o16, pc, ps) if want_codes else (o32, o16)
+                                          _p(o32), _p(o16), _p(pc), _p(ps), _p(y), _p(am), int(flip_key), int(flip_dir),
+                                          int(flip_blk), int(flip_blk_dir))
+    return (o32, o16, pc, ps, y, am) if want_codes else (o32, o16)

@@ -22,6 +22,7 @@ MPFA_DEV_TIMEOUT = 1
 MPFA_DEV_BAD_PAGE = 2
 MPFA_VARIANT_COMP_ELEMENTWISE = 1
 MPFA_VARIANT_PV_BF16 = 2
+MPFA_VARIANT_PV_FP4 = 3
 HEAD_DIM = 128
 PAGE = 64
 
@@ -70,7 +71,7 @@ def load_library(path: str) -> ctypes.CDLL:
         L.mpfa_quantize_workspace_min_bytes.argtypes = [i, i, i]
         L.mpfa_decode_workspace_bytes.restype = sz
         L.mpfa_decode_workspace_bytes.argtypes = [i, i, i, i]
-        for name in ("mpfa_fp4_codes_bytes", "mpfa_fp4_sf_bytes", "mpfa_delta_s_bytes", "mpfa_v_fp8_bytes"):
+        for name in ("mpfa_fp4_codes_bytes", "mpfa_fp4_sf_bytes", "mpfa_delta_s_bytes", "mpfa_v_fp8_bytes", "mpfa_v_fp4_bytes"):
             getattr(L, name).restype = sz
             getattr(L, name).argtypes = [i, i, i]
         L.mpfa_sf_offset.restype = sz
@@ -92,6 +93,8 @@ def load_library(path: str) -> ctypes.CDLL:
         L.mpfa_static_scratch_bytes.restype = sz
         L.mpfa_quantize_v.restype = i
         L.mpfa_quantize_v.argtypes = [vp, i, i, i, f, vp, vp]
+        L.mpfa_quantize_v_fp4.restype = i
+        L.mpfa_quantize_v_fp4.argtypes = [vp, i, i, i, f, vp, vp]
         L.mpfa_pack_v_bf16.restype = i
         L.mpfa_pack_v_bf16.argtypes = [vp, i, i, i, vp, vp]
         L.mpfa_quantize_kv_paged.restype = i
@@ -410,4 +413,13 @@ def mpfa_pack_v_bf16(v: torch.Tensor) -> torch.Tensor:
     B, N, H, _ = v.shape
     out = aligned_empty(2 * lib().mpfa_v_fp8_bytes(B, H, N), v.device).view(torch.bfloat16).view(B, H, _pad128(N), HEAD_DIM)
     _check(lib().mpfa_pack_v_bf16(_ptr(v), B, N, H, _ptr(out), _stream()), "mpfa_pack_v_bf16")
+    return out
+
+
+def mpfa_quantize_v_fp4(v: torch.Tensor, v_gscale: float) -> torch.Tensor:
+    """V [B,N,H,128] bf16 -> the FP4 operand (codes of all tiles, then block scales) the MPFA_VARIANT_PV_FP4 prefill reads."""
+    assert v.is_cuda and v.dtype == torch.bfloat16 and v.is_contiguous()
+    B, N, H, _ = v.shape
+    out = aligned_empty(lib().mpfa_v_fp4_bytes(B, H, N), v.device)
+    _check(lib().mpfa_quantize_v_fp4(_ptr(v), B, N, H, v_gscale, _ptr(out), _stream()), "mpfa_quantize_v_fp4")
     return out

@@ -41,6 +41,7 @@
 // tensor memory is released.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp4.h>
 #include <cuda_fp8.h>
 
 #include "common.cuh"
@@ -100,14 +101,17 @@ enum {
   NUM_BARS = BAR_SF_READY + KSTAGES
 };
 static_assert(NUM_BARS <= 64, "barrier table");
-// Shared-memory layout.  PVB = the NVFP4 + BF16 precision assignment (mpfa_prefill_variant): V tiles are BF16
-// (32 KB, two stages), P is handed to the second MMA through shared memory as a K-major BF16 A operand (2 x 32 KB),
-// and the K ring has three stages to make room.
-template <bool PVB>
+// Shared-memory layout.  PVK selects the operands of the second MMA (mpfa_prefill_variant): 0 = the method (FP8);
+// 1 = the NVFP4 + BF16 precision assignment: V tiles are BF16 (32 KB, two stages), P is handed to the second MMA
+// through shared memory as a K-major BF16 A operand (2 x 32 KB), and the K ring has three stages to make room;
+// 2 = the NVFP4 + NVFP4 assignment: V tiles are channel-major FP4 (8 KB + 1 KB of block scales), P goes through
+// shared memory as a K-major FP4 A operand (2 x 8 KB) with its block scales (2 x 1 KB).
+template <int PVK>
 struct Lay {
+  static constexpr bool PVB = PVK == 1, PV4 = PVK == 2;
   static constexpr int KST = PVB ? 3 : KSTAGES;
   static constexpr int VST = PVB ? 2 : VSTAGES;
-  static constexpr uint32_t V_BYTES = PVB ? 32768u : 16384u;
+  static constexpr uint32_t V_BYTES = PVB ? 32768u : (PV4 ? 8192u : 16384u);
   static constexpr uint32_t OFF_Q = 0;                               // 2 tiles (the next tile's queries are prefetched)
   static constexpr uint32_t OFF_K = OFF_Q + 2 * 8192;
   static constexpr uint32_t OFF_V = OFF_K + KST * 8192;
@@ -123,14 +127,20 @@ struct Lay {
   // paged source only: per K stage the two pages' scale bytes (2 x 512) and Delta_S rows (2 x 128) as stored
   static constexpr uint32_t RAW_STAGE = 1280;
   static constexpr uint32_t OFF_RAW = (OFF_MISC + 16 + 127) & ~127u;
-  static constexpr uint32_t OFF_PS = (OFF_MISC + 16 + 1023) & ~1023u;   // PVB only: P of the two softmax groups
-  static constexpr uint32_t SMEM_BYTES = (PVB ? OFF_PS + 2 * 32768 : OFF_MISC + 16) + 1024;   // + slack for the 1024-byte alignment
+  static constexpr uint32_t OFF_PS = (OFF_MISC + 16 + 1023) & ~1023u;   // PVB / PV4 only: P of the two softmax groups
+  static constexpr uint32_t PS_BYTES = PVB ? 32768u : 8192u;
+  static constexpr uint32_t OFF_SFP = OFF_PS + 2 * PS_BYTES;            // PV4 only: block scales of P, [group][2 atoms]
+  static constexpr uint32_t OFF_SFV = OFF_SFP + 2 * 1024;               // PV4 only: block scales of V, [stage][2 atoms]
+  static constexpr uint32_t SMEM_BYTES =
+      (PVB ? OFF_PS + 2 * PS_BYTES : (PV4 ? OFF_SFV + VST * 1024 : OFF_MISC + 16)) + 1024;   // + slack for the 1024-byte alignment
   static constexpr uint32_t SMEM_BYTES_PAGED = OFF_RAW + KST * RAW_STAGE + 1024;
 };
-static_assert(Lay<true>::SMEM_BYTES <= 227 * 1024 && Lay<false>::SMEM_BYTES_PAGED <= 227 * 1024, "shared memory");
+static_assert(Lay<1>::SMEM_BYTES <= 227 * 1024 && Lay<2>::SMEM_BYTES <= 227 * 1024 && Lay<0>::SMEM_BYTES_PAGED <= 227 * 1024, "shared memory");
 
 constexpr uint32_t TM_S = 0, TM_O0 = 128, TM_O1 = 256, TM_P0 = 384, TM_P1 = 416, TM_SFQ = 448 /* 2 x 8 */,
                    TM_SFK0 = 464, TM_SFK1 = 472;
+// NVFP4 + NVFP4 variant only: block scales of P (per softmax group) and of V (per block parity)
+constexpr uint32_t TM_SFP0 = 480, TM_SFP1 = 488, TM_SFV0 = 496, TM_SFV1 = 504;
 constexpr uint32_t TMEM_COLS = 512;
 
 // Optional timeline capture for tuning (compiled in only with -DMPFA_TRACE): one CTA records
@@ -191,18 +201,22 @@ struct TileWalk {
 // PVB: precision-assignment variant of Section 3.1 (NVFP4 Q K^T, BF16 P V): P = 2^(lam S - lam m) is rounded to BF16
 // and handed to the second MMA through shared memory (K-major A operand), V is the BF16 input in the tile layout
 // written by mpfa_pack_v_bf16, the second MMA is kind::f16 (eight K = 16 steps per block).
-template <bool PAGED, bool EW, bool PVB = false>
+// PV4: the NVFP4 + NVFP4 assignment: q = 448 P is quantized per row and 16 keys (E4M3 block scale of max q, E2M1 codes
+// of q * (6 / scale)) and written with its scales to shared memory; V is the channel-major FP4 operand of
+// mpfa_quantize_v_fp4; the second MMA is kind::mxf4nvf4 block-scaled (two K = 64 steps per block).
+template <bool PAGED, bool EW, int PVK = 0>
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const PrefillParams p, const PagedSrc pg) {
-  static_assert(!(PVB && (PAGED || EW)), "the BF16 variant exists for contiguous operands with the seed MMA only");
-  using L = Lay<PVB>;
+  constexpr bool PVB = PVK == 1, PV4 = PVK == 2;
+  static_assert(!(PVK != 0 && (PAGED || EW)), "the precision variants exist for contiguous operands with the seed MMA only");
+  using L = Lay<PVK>;
   constexpr int KST = L::KST, VST = L::VST;
   constexpr uint32_t OFF_Q = L::OFF_Q, OFF_K = L::OFF_K, OFF_V = L::OFF_V, OFF_DELTA = L::OFF_DELTA, OFF_ONES = L::OFF_ONES,
                      OFF_SFQ = L::OFF_SFQ, OFF_SFK = L::OFF_SFK, OFF_M = L::OFF_M, OFF_L = L::OFF_L, OFF_BAR = L::OFF_BAR,
                      OFF_MISC = L::OFF_MISC, OFF_RAW = L::OFF_RAW, RAW_STAGE = L::RAW_STAGE, OFF_PS = L::OFF_PS,
-                     V_BYTES = L::V_BYTES;
-  (void)OFF_PS; (void)OFF_RAW; (void)RAW_STAGE;
+                     V_BYTES = L::V_BYTES, PS_BYTES = L::PS_BYTES, OFF_SFP = L::OFF_SFP, OFF_SFV = L::OFF_SFV;
+  (void)OFF_PS; (void)OFF_RAW; (void)RAW_STAGE; (void)PS_BYTES; (void)OFF_SFP; (void)OFF_SFV;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -342,8 +356,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             bulk_load(sbase + OFF_V + vs * 16384 + 8192, pg.v_fp8 + ((size_t)page_hi * p.H_kv + tl.hk) * 8192, 8192, bar);
           }
         } else if (elect_one()) {
-          mbar_expect_tx(cx.bar(BAR_V_FULL + vs), V_BYTES);
+          mbar_expect_tx(cx.bar(BAR_V_FULL + vs), V_BYTES + (PV4 ? 1024u : 0u));
           tma_load_2d(sbase + OFF_V + vs * V_BYTES, &tm_v, 0, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
+          if (PV4)   // channel-major FP4 tile (same row arithmetic as K: 128 channel rows per key tile) + its block scales
+            bulk_load(sbase + OFF_SFV + vs * 1024, p.v_sf + (((size_t)tl.b * p.H_kv + tl.hk) * p.nk_tiles + jb) * 1024, 1024,
+                      cx.bar(BAR_V_FULL + vs));
           if (PVB)   // BF16 rows are 256 bytes: the second 64-channel half is a box of its own
             tma_load_2d(sbase + OFF_V + vs * V_BYTES + 16384, &tm_v, 128, (int)(k_row + (size_t)jb * TILE), cx.bar(BAR_V_FULL + vs));
         }
@@ -459,9 +476,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // =========================== P V issuer ===========================
     const uint32_t id_fp8 = idesc_e4m3(128, 128, 0, 1);
     const uint32_t id_bf16_pv = idesc_bf16(128, 128, 0, 1);
-    const uint64_t d_v0 = smem_desc(sbase + OFF_V, PVB ? 16384 : 16, 1024, SWZ_128B);
-    const uint64_t d_p0 = smem_desc(sbase + OFF_PS, 16, 1024, SWZ_128B);
-    (void)id_fp8; (void)id_bf16_pv; (void)d_p0;
+    const uint32_t id_fp4_pv = idesc_nvfp4(128, 128);
+    const uint64_t d_v0 = PV4 ? smem_desc(sbase + OFF_V, 16, 512, SWZ_64B) : smem_desc(sbase + OFF_V, PVB ? 16384 : 16, 1024, SWZ_128B);
+    const uint64_t d_p0 = PV4 ? smem_desc(sbase + OFF_PS, 16, 512, SWZ_64B) : smem_desc(sbase + OFF_PS, 16, 1024, SWZ_128B);
+    const uint64_t d_sfp0 = smem_desc(sbase + OFF_SFP, 0, 128, SWZ_NONE);
+    const uint64_t d_sfv0 = smem_desc(sbase + OFF_SFV, 0, 128, SWZ_NONE);
+    (void)id_fp8; (void)id_bf16_pv; (void)d_p0; (void)id_fp4_pv; (void)d_sfp0; (void)d_sfv0;
     bool ok = true;
     uint32_t n_used = 0;   // items so far that used the accumulators (T > 0)
     for (; ok && walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
@@ -493,6 +513,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             for (int k16 = 0; k16 < 8; ++k16)
               mma_bf16_ss(tOacc, d_p + (uint64_t)(((k16 >> 2) * 16384 + (k16 & 3) * 32) >> 4), d_v + (uint64_t)((2048 * k16) >> 4),
                           id_bf16_pv, (t >= 2 || k16 > 0) ? 1u : 0u);
+          } else if constexpr (PV4) {
+            // block-scaled FP4: A = P-hat codes of this group (K-major, 64-byte rows), B = V codes (channel-major);
+            // both operands' block scales go to tensor memory first (their columns were last read by block c-2)
+            const uint64_t d_p = d_p0 + (uint64_t)((sb * PS_BYTES) >> 4);
+            const uint64_t d_sfp = d_sfp0 + (uint64_t)((sb * 1024) >> 4), d_sfv = d_sfv0 + (uint64_t)((vs * 1024) >> 4);
+            const uint32_t tSFP = tm + (sb ? TM_SFP1 : TM_SFP0), tSFV = tm + (sb ? TM_SFV1 : TM_SFV0);
+            tmem_cp_32x128b_warpx4(tSFP, d_sfp);
+            tmem_cp_32x128b_warpx4(tSFP + 4, d_sfp + (512 >> 4));
+            tmem_cp_32x128b_warpx4(tSFV, d_sfv);
+            tmem_cp_32x128b_warpx4(tSFV + 4, d_sfv + (512 >> 4));
+            mma_nvfp4_ss(tOacc, d_p, d_v, id_fp4_pv, tSFP, tSFV, t >= 2 ? 1u : 0u);
+            mma_nvfp4_ss(tOacc, d_p + (32 >> 4), d_v + (32 >> 4), id_fp4_pv, tSFP + 4, tSFV + 4, 1u);
           } else {
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
@@ -519,7 +551,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t tS = tm + TM_S + lane_off;
     const uint32_t tP = tm + (grp ? TM_P1 : TM_P0) + lane_off;
     uint8_t *const ps_row = smem + OFF_PS + grp * 32768 + row * 128;   // PVB: this thread's row of the group's P operand
-    (void)tP; (void)ps_row;
+    // PV4: this thread's 64-byte row of the group's FP4 operand (64B swizzle: 16-byte chunk ^ ((row >> 1) & 3)) and its
+    // word in each of the group's two scale-factor atoms
+    uint8_t *const p4_row = smem + OFF_PS + grp * 8192 + row * 64;
+    uint8_t *const sfp_row = smem + OFF_SFP + grp * 1024 + (row & 31) * 16 + (row >> 5) * 4;
+    (void)tP; (void)ps_row; (void)p4_row; (void)sfp_row;
     bool ok = true;
     uint32_t n_used = 0;   // items so far with T > 0: only those go through the row-sum ring
     for (; ok && walk.template next<PAGED>(p, pg, tl); gb += tl.T, ++ti) {
@@ -667,11 +703,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #endif
           // q = 448 P is the E4M3 operand (Section 4.1); the row sum is taken over q and the factor
           // 448 is divided out once in the epilogue.
+          uint32_t sfw = 0u;   // PV4: the E4M3 block scales of 64 keys
+          (void)sfw;
 #pragma unroll
           for (int c0 = 0; c0 < 128; c0 += 32) {
             uint32_t packed[8];
             uint32_t pbf[4];
-            (void)packed; (void)pbf;
+            float qv[32];
+            (void)packed; (void)pbf; (void)qv;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               float x0, x1, x2, x3;
@@ -680,7 +719,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
               const float q0 = EX2_(x0), q1 = EX2_(x1), q2 = EX2_(x2), q3 = EX2_(x3);
               acc2(sum0, sum1, q0, q1);
               acc2(sum2, sum3, q2, q3);
-              if constexpr (PVB) {
+              if constexpr (PV4) {
+                qv[4 * i] = q0, qv[4 * i + 1] = q1, qv[4 * i + 2] = q2, qv[4 * i + 3] = q3;
+              } else if constexpr (PVB) {
                 // BF16 pairs (first operand of the conversion goes to the upper half)
                 asm("cvt.rn.bf16x2.f32 %0, %2, %1;" : "=r"(pbf[2 * (i & 1)]) : "f"(q0), "f"(q1));
                 asm("cvt.rn.bf16x2.f32 %0, %2, %1;" : "=r"(pbf[2 * (i & 1) + 1]) : "f"(q2), "f"(q3));
@@ -700,7 +741,35 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                   : "f"(q0), "f"(q1), "f"(q2), "f"(q3));
               }
             }
-            if constexpr (!PVB) {
+            if constexpr (PV4) {
+              // two blocks of 16 keys: scale = E4M3(max q), codes = E2M1(q * (6 / scale)) (Eq. 1 with the tensor scale
+              // of P fixed at 1 / (6 * 448))
+              uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+              for (int hb = 0; hb < 2; ++hb) {
+                const float *qb = qv + 16 * hb;
+                float a0 = max3(qb[0], qb[1], qb[2]), a1 = max3(qb[3], qb[4], qb[5]), a2 = max3(qb[6], qb[7], qb[8]),
+                      a3 = max3(qb[9], qb[10], qb[11]);
+                a0 = max3(a0, qb[12], qb[13]);
+                a1 = max3(a1, qb[14], qb[15]);
+                const float amax = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
+                const uint32_t sc = (uint32_t)__nv_cvt_float_to_fp8(amax, __NV_SATFINITE, __NV_E4M3);
+                const float sdec = __half2float(__half(__nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)sc, __NV_E4M3)));
+                const float inv = sdec > 0.0f ? __fdiv_rn(6.0f, sdec) : 0.0f;
+                sfw |= sc << (8 * (((c0 >> 4) + hb) & 3));
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const uint32_t byte = (uint32_t)__nv_cvt_float2_to_fp4x2(
+                      make_float2(__fmul_rn(qb[2 * j], inv), __fmul_rn(qb[2 * j + 1], inv)), __NV_E2M1, cudaRoundNearest);
+                  w[2 * hb + (j >> 2)] |= (byte & 0xFFu) << (8 * (j & 3));
+                }
+              }
+              *reinterpret_cast<uint4 *>(p4_row + ((((c0 >> 5)) ^ ((row >> 1) & 3)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+              if (c0 & 32) {   // 64 keys done: one word of the row in this half's scale-factor atom
+                *reinterpret_cast<uint32_t *>(sfp_row + (c0 >> 6) * 512) = sfw;
+                sfw = 0u;
+              }
+            } else if constexpr (!PVB) {
 #ifndef MPFA_ABLATE_NO_PST
             tmem_st8(tP + (c0 >> 2), packed);
 #else
@@ -712,7 +781,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         l_own = __fadd_rn(__fmul_rn(a_own, l_own), (sum0 + sum1) + (sum2 + sum3));
         m_own = m_t;
         TR(2 + grp, c, 5);
-        if constexpr (PVB) {
+        if constexpr (PVB || PV4) {
           fence_proxy_async_smem();   // the P rows were written through the generic proxy, the MMA reads them through the async one
         } else {
           tmem_st_wait();
@@ -896,9 +965,11 @@ extern "C" mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *q, const mpfa
                                             const void *delta_s_bf16, const mpfa_stats *st, float v_scale, int causal,
                                             float softmax_scale, int variant, void *out_bf16, float *out_f32,
                                             int32_t *device_status, void *stream) {
-  if (variant != 0 && variant != MPFA_VARIANT_COMP_ELEMENTWISE && variant != MPFA_VARIANT_PV_BF16) return MPFA_ERR_INVALID_ARG;
+  if (variant != 0 && variant != MPFA_VARIANT_COMP_ELEMENTWISE && variant != MPFA_VARIANT_PV_BF16 && variant != MPFA_VARIANT_PV_FP4)
+    return MPFA_ERR_INVALID_ARG;
   const bool ew = variant == MPFA_VARIANT_COMP_ELEMENTWISE && delta_s_bf16 != nullptr;
   const bool pvb = variant == MPFA_VARIANT_PV_BF16;   // v_fp8 then points at the BF16 tile tensor of mpfa_pack_v_bf16
+  const bool pv4 = variant == MPFA_VARIANT_PV_FP4;    // ... at the FP4 operand of mpfa_quantize_v_fp4, v_scale = its v_gscale
   if (!q || !k || !v_fp8 || !st || !out_bf16 || !device_status) return MPFA_ERR_INVALID_ARG;
   if (!q->codes || !q->sf || !k->codes || !k->sf || !st->q_gscale || !st->k_gscale) return MPFA_ERR_INVALID_ARG;
   if (q->B <= 0 || q->B != k->B || q->H <= 0 || k->H <= 0 || q->N <= 0 || k->N <= 0) return MPFA_ERR_INVALID_ARG;
@@ -934,27 +1005,36 @@ extern "C" mpfa_status mpfa_prefill_variant(const mpfa_fp4_tensor *q, const mpfa
   p.softmax_scale = softmax_scale;
   p.v_scale = v_scale;
   p.n_items = (int)n_cta;
-  if (g_arrangement == 1 && !pvb) return launch_prefill_pair(q, k, v_fp8, p, ew, static_cast<cudaStream_t>(stream));
+  if (pv4) {
+    // codes of all tiles first, then the block scales; the MMA result is in units of 6 * 448 P x V / v_gscale and the
+    // row sum carries the 448
+    p.v_sf = v_fp8 + (size_t)k->B * k->H * nk_tiles * 8192;
+    p.v_scale = v_scale * (1.0f / 6.0f);
+  }
+  if (g_arrangement == 1 && !pvb && !pv4) return launch_prefill_pair(q, k, v_fp8, p, ew, static_cast<cudaStream_t>(stream));
   EncodeTiledFn enc;
   rc = get_encoder(&enc);
   if (rc != MPFA_OK) return rc;
   CUtensorMap tq, tk, tv;
   if ((rc = make_map(enc, &tq, q->codes, q_rows, 64)) != MPFA_OK) return rc;
   if ((rc = make_map(enc, &tk, k->codes, k_rows, 64)) != MPFA_OK) return rc;
-  if ((rc = pvb ? make_map(enc, &tv, v_fp8, k_rows, 256, 128) : make_map(enc, &tv, v_fp8, k_rows, 128)) != MPFA_OK) return rc;
+  if ((rc = pvb ? make_map(enc, &tv, v_fp8, k_rows, 256, 128) : make_map(enc, &tv, v_fp8, k_rows, pv4 ? 64 : 128)) != MPFA_OK) return rc;
   int dev = 0, n_sm = 0;
   MPFA_CUDA_OK(cudaGetDevice(&dev));
   MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
   const unsigned grid = (unsigned)(n_cta < (uint64_t)n_sm ? n_cta : (uint64_t)n_sm);   // one persistent CTA per SM
   if (pvb) {
-    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<true>::SMEM_BYTES));
-    prefill_kernel<false, false, true><<<grid, NTHREADS, Lay<true>::SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<1>::SMEM_BYTES));
+    prefill_kernel<false, false, 1><<<grid, NTHREADS, Lay<1>::SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+  } else if (pv4) {
+    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<2>::SMEM_BYTES));
+    prefill_kernel<false, false, 2><<<grid, NTHREADS, Lay<2>::SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
   } else if (ew) {
-    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::SMEM_BYTES));
-    prefill_kernel<false, true><<<grid, NTHREADS, Lay<false>::SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<0>::SMEM_BYTES));
+    prefill_kernel<false, true><<<grid, NTHREADS, Lay<0>::SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
   } else {
-    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::SMEM_BYTES));
-    prefill_kernel<false, false><<<grid, NTHREADS, Lay<false>::SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
+    MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<0>::SMEM_BYTES));
+    prefill_kernel<false, false><<<grid, NTHREADS, Lay<0>::SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, p, PagedSrc{});
   }
   MPFA_LAUNCH_OK();
   return MPFA_OK;
@@ -1021,8 +1101,8 @@ extern "C" mpfa_status mpfa_prefill_paged(const mpfa_fp4_tensor *q, const mpfa_p
   MPFA_CUDA_OK(cudaGetDevice(&dev));
   MPFA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
   const unsigned grid = (unsigned)(n_cta < (uint64_t)n_sm ? n_cta : (uint64_t)n_sm);
-  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::SMEM_BYTES_PAGED));
-  prefill_kernel<true, false><<<grid, NTHREADS, Lay<false>::SMEM_BYTES_PAGED, static_cast<cudaStream_t>(stream)>>>(tq, tq, tq, p, pg);
+  MPFA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<0>::SMEM_BYTES_PAGED));
+  prefill_kernel<true, false><<<grid, NTHREADS, Lay<0>::SMEM_BYTES_PAGED, static_cast<cudaStream_t>(stream)>>>(tq, tq, tq, p, pg);
   MPFA_LAUNCH_OK();
   return MPFA_OK;
 }

@@ -12,6 +12,7 @@ namespace mpfa {
 struct PrefillParams {
   const uint8_t *q_sf;
   const uint8_t *k_sf;
+  const uint8_t *v_sf = nullptr;   // NVFP4 + NVFP4 variant only: block scales of the FP4 V operand
   const __nv_bfloat16 *delta;  // may be null
   const float *q_gscale;
   const float *k_gscale;

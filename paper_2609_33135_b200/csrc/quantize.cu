@@ -556,6 +556,48 @@ __global__ void __launch_bounds__(256) pack_v_bf16_kernel(const __nv_bfloat16 *_
   }
 }
 
+// grid (N_pad/128, H, B): V tile for the NVFP4 + NVFP4 precision assignment of Section 3.1.  The second MMA contracts
+// over the keys, so the 16-element blocks of Eq. 1 lie along the token axis and the operand is stored channel-major
+// (K-major B operand): codes [B, H, N_pad/128, 128 channels, 64 bytes] (two keys per byte, the even key in the low
+// nibble), block scales as two 512-byte tcgen05.cp atoms per tile (atom = 64 keys: byte (c mod 32) 16 + (c / 32) 4 +
+// block mod 4).  Recipe of the Q/K quantizer with the caller's tensor scale d and no centering; keys past N are zero.
+__global__ void __launch_bounds__(256) quantize_v_fp4_tile_kernel(const __nv_bfloat16 *__restrict__ v, int N, int H, float d,
+                                                                  uint8_t *__restrict__ codes, uint8_t *__restrict__ sf) {
+  __shared__ __align__(16) __nv_bfloat16 tile[TILE][HEAD_DIM + 8];   // padded rows: the column reads below stay conflict-free
+  __shared__ __align__(16) uint8_t ctile[HEAD_DIM][64];
+  __shared__ __align__(16) uint8_t stile[1024];
+  const int t0 = blockIdx.x * TILE, h = blockIdx.y, b = blockIdx.z;
+  const int n_tiles = gridDim.x;
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int id = it * 256 + threadIdx.x;
+    const int r = id >> 4, seg = id & 15;
+    uint4 u = make_uint4(0u, 0u, 0u, 0u);
+    if (t0 + r < N) u = __ldcs(reinterpret_cast<const uint4 *>(v + (((size_t)b * N + t0 + r) * H + h) * HEAD_DIM + seg * 8));
+    *reinterpret_cast<uint4 *>(&tile[r][seg * 8]) = u;
+  }
+  __syncthreads();
+#pragma unroll 1
+  for (int it = 0; it < 4; ++it) {
+    const int id = it * 256 + threadIdx.x;
+    const int c = id & 127, kb = id >> 7;   // channel, 16-key block of the tile
+    float x[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x[i] = __bfloat162float(tile[kb * 16 + i][c]);
+    uint8_t sc;
+    uint2 cw;
+    quantize_block16(x, d, sc, cw);
+    *reinterpret_cast<uint2 *>(&ctile[c][kb * 8]) = cw;
+    stile[(kb >> 2) * 512 + (c & 31) * 16 + (c >> 5) * 4 + (kb & 3)] = sc;
+  }
+  __syncthreads();
+  const size_t tile_id = ((size_t)b * H + h) * n_tiles + blockIdx.x;
+  uint4 *cdst = reinterpret_cast<uint4 *>(codes + tile_id * 8192);
+#pragma unroll
+  for (int it = 0; it < 2; ++it) cdst[it * 256 + threadIdx.x] = reinterpret_cast<const uint4 *>(&ctile[0][0])[it * 256 + threadIdx.x];
+  if (threadIdx.x < 64) reinterpret_cast<uint4 *>(sf + tile_id * 1024)[threadIdx.x] = reinterpret_cast<const uint4 *>(stile)[threadIdx.x];
+}
+
 // Paged cache write for one request: grid (pages, H_kv).  K and V of one (page, head) are
 // quantized into shared memory in the byte order of the decode kernel's shared-memory operand
 // tiles (so that decode fills a tile with one bulk copy) and copied out with 16-byte stores.
@@ -876,6 +918,24 @@ extern "C" mpfa_status mpfa_pack_v_bf16(const void *v_bf16, int B, int N_kv, int
   if (rc != MPFA_OK) return rc;
   pack_v_bf16_kernel<<<dim3(pad128(N_kv) / TILE, H_kv, B), 256, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16 *>(v_bf16), N_kv, H_kv, static_cast<__nv_bfloat16 *>(v_tiles_bf16));
+  MPFA_LAUNCH_OK();
+  return MPFA_OK;
+}
+
+extern "C" size_t mpfa_v_fp4_bytes(int B, int H_kv, int N_kv) {
+  if (B <= 0 || H_kv <= 0 || N_kv <= 0) return 0;
+  return (size_t)B * H_kv * (pad128(N_kv) / TILE) * (8192 + 1024);
+}
+
+extern "C" mpfa_status mpfa_quantize_v_fp4(const void *v_bf16, int B, int N_kv, int H_kv, float v_gscale, uint8_t *v_fp4,
+                                           void *stream) {
+  if (!v_bf16 || !v_fp4 || B <= 0 || N_kv <= 0 || H_kv <= 0 || !(v_gscale > 0.0f)) return MPFA_ERR_INVALID_ARG;
+  if (!aligned(v_bf16, 16) || !aligned(v_fp4, 1024)) return MPFA_ERR_ALIGNMENT;
+  mpfa_status rc = check_arch();
+  if (rc != MPFA_OK) return rc;
+  const size_t n_tiles = (size_t)B * H_kv * (pad128(N_kv) / TILE);
+  quantize_v_fp4_tile_kernel<<<dim3(pad128(N_kv) / TILE, H_kv, B), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16 *>(v_bf16), N_kv, H_kv, v_gscale, v_fp4, v_fp4 + n_tiles * 8192);
   MPFA_LAUNCH_OK();
   return MPFA_OK;
 }

@@ -53,3 +53,19 @@ def paged_delta_to_logical(page: np.ndarray, G: int) -> np.ndarray:
     h = np.arange(page.shape[0])[:, None]
     t = np.arange(64)[None, :]
     return np.take_along_axis(page, (((t // 8) ^ (h % G)) * 8 + t % 8), axis=1)
+
+
+def v_fp4_to_logical(buf: np.ndarray, B, H, N):
+    """FP4 V operand (codes of all tiles, then block scales; flat uint8) -> (codes [B,H,128,NB,8], sf [B,H,128,NB],
+    pad codes, pad scales) with NB = ceil(N/16); the pads (blocks past NB) are returned for a zero check."""
+    tiles = pad128(N) // 128
+    nb = (N + 15) // 16
+    n_codes = B * H * tiles * 8192
+    c = buf[:n_codes].reshape(B, H, tiles, 128, 8, 8).transpose(0, 1, 3, 2, 4, 5).reshape(B, H, 128, tiles * 8, 8)
+    a = buf[n_codes:n_codes + B * H * tiles * 1024].reshape(B, H, tiles, 2, 512)
+    ch = np.arange(128)
+    kb = np.arange(8)
+    off = (ch[:, None] % 32) * 16 + (ch[:, None] // 32) * 4 + (kb[None, :] % 4)      # [128, 8]
+    atom = np.broadcast_to(kb[None, :] // 4, (128, 8))
+    s = a[:, :, :, atom, off].transpose(0, 1, 3, 2, 4).reshape(B, H, 128, tiles * 8)
+    return c[:, :, :, :nb], s[:, :, :, :nb], c[:, :, :, nb:], s[:, :, :, nb:]

@@ -175,7 +175,7 @@ def test_fp4_pv_loop_against_the_numpy_statement():
     for scale in (0.02, 0.006, 0.002):
         lam = np.float32(np.float32(scale) * LOG2E)
         want_c, want_s, want_o = _loop_by_hand(s, _unpack(vc[0, 0]), vs[0, 0], d_v, lam)
-        o32, _, pc, ps = orc.prefill_rows_pv_fp4(z, vc, vs, d_v, rows, scale, False, want_codes=True)
+        o32, _, pc, ps, _, _ = orc.prefill_rows_pv_fp4(z, vc, vs, d_v, rows, scale, False, want_codes=True)
         assert np.array_equal(pc[0], want_c), scale
         assert np.array_equal(ps[0], want_s), scale
         assert np.abs(o32[0] - want_o).max() <= 2e-6 * max(1.0, np.abs(want_o).max()), scale
@@ -204,3 +204,29 @@ def test_fp4_pv_is_attention_and_coarser_than_the_method():
     for hq in range(4):
         r = hq * 384
         assert np.abs(o4[r] - deq0[hq // 2]).max() <= 1e-6 * max(1.0, np.abs(deq0).max())
+
+
+def test_inspection_switches_change_nothing_unless_asked():
+    """The hooks a GPU test uses to show that a row differs by one rounding decision: asking for the codes leaves the
+    output as it is; moving one key's code or one block's scale by a step changes that row, and only in the way
+    the decoded values say."""
+    z, s, vb = _case()
+    d_v = float(np.float32(np.abs(orc.bits_to_f32(vb)).max() / (6.0 * 448.0)))
+    vc, vs = orc.quantize_v_fp4(vb, d_v)
+    rows = np.array([[0, 0, 0]], np.int32)
+    scale = 0.004
+    plain, _ = orc.prefill_rows_pv_fp4(z, vc, vs, d_v, rows, scale, False)
+    o, _, pc, ps, y, am = orc.prefill_rows_pv_fp4(z, vc, vs, d_v, rows, scale, False, want_codes=True)
+    assert np.array_equal(o, plain)
+    # the recorded pre-rounding values are the ones the codes were made from
+    assert np.array_equal(_e2m1_codes_rne(y[0]), pc[0])
+    assert np.array_equal(_e4m3_codes_rne(am[0]), ps[0])
+    key = int(np.nonzero((pc[0] > 1) & (pc[0] < 7))[0][0])
+    f1, _, pc1, _, _, _ = orc.prefill_rows_pv_fp4(z, vc, vs, d_v, rows, scale, False, want_codes=True, flip_key=key, flip_dir=1)
+    assert pc1[0, key] == pc[0, key] + 1 and (np.delete(pc1[0], key) == np.delete(pc[0], key)).all()
+    assert np.abs(f1 - plain).max() > 0
+    blk = key // 16
+    f2, _, pc2, ps2, _, _ = orc.prefill_rows_pv_fp4(z, vc, vs, d_v, rows, scale, False, want_codes=True, flip_blk=blk, flip_blk_dir=-1)
+    assert ps2[0, blk] == ps[0, blk] - 1 and (np.delete(ps2[0], blk) == np.delete(ps[0], blk)).all()
+    assert np.array_equal(pc2[0, :16 * blk], pc[0, :16 * blk]) and np.array_equal(pc2[0, 16 * blk + 16:], pc[0, 16 * blk + 16:])
+    assert np.abs(f2 - plain).max() > 0
