@@ -180,6 +180,48 @@ def cpu_baseline_record(flops, times, sample, cores):
             "attention_seconds": att, "seconds_per_query_key_pair": att / (flops / 512.0), "stage1_seconds_full_tensors": s1}
 
 
+def cpu_oracle_config1_full():
+    """Config 1 (256 tokens, one head, non-causal) through the oracle in full: stage 1 + attention of all rows."""
+    from oracle import mpfa_oracle as orc
+    from paper_2609_33135_b200 import workloads as wl
+    w = wl.config1_tiny()
+    q, k, v = orc.bf16_bits(w.q), orc.bf16_bits(w.k), orc.bf16_bits(w.v)
+    rows = orc.all_rows(w.B, w.H_q, w.N_q)
+    orc.prefill_rows(orc.stage1(q, k, v), rows, w.softmax_scale, w.causal)   # first call loads the library
+    reps = 20
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        z = orc.stage1(q, k, v)
+        orc.prefill_rows(z, rows, w.softmax_scale, w.causal)
+    sec = (time.perf_counter() - t0) / reps
+    return {"workload": w.name, "seconds_stage1_plus_attention": sec, "tflops": w.flops / sec / 1e12,
+            "sample": "the whole config: all 256 rows against all 256 keys, stage 1 included"}
+
+
+def cpu_oracle_decode_sample(n_requests: int = 2):
+    """Config 5 through the oracle on a bounded sample: the first `n_requests` requests, all 32 heads each; the cache
+    (stage 1 of each request's K/V with frozen statistics) is built outside the timed part, as on the GPU."""
+    from oracle import mpfa_oracle as orc
+    from paper_2609_33135_b200 import workloads as wl
+    import numpy as np
+    w = wl.config5_decode()
+    tokens, sec = 0, 0.0
+    for b in range(n_requests):
+        k, v = w.kv_for_request(b, "cpu")
+        kb, vb = orc.bf16_bits(k), orc.bf16_bits(v)
+        z = orc.stage1(orc.bf16_bits(w.q_sample[b:b + 1].contiguous()), kb, vb)
+        zq = orc.stage1(orc.bf16_bits(w.q_new[b:b + 1].contiguous()), kb, vb, frozen=z)
+        L = int(w.seq_lens[b])
+        t0 = time.perf_counter()
+        orc.decode(zq.q_codes[:, :, 0], zq.q_sf[:, :, 0], z.k_codes, z.k_sf, z.v_codes, z.delta, z.dq, z.dk, 1.0, w.softmax_scale,
+                   np.array([L], np.int32))
+        sec += time.perf_counter() - t0
+        tokens += L
+    bytes_ = float(tokens) * w.H_kv * KV_BYTES_PER_TOKEN_HEAD
+    return {"workload": w.name, "value": bytes_ / sec / 1e9, "unit": "GB/s", "seconds": sec, "tokens": tokens,
+            "sample": f"requests 0..{n_requests - 1} of 32 (all 32 heads each), decode attention only; the cache is built before the timed part"}
+
+
 def run_reference(args, rank):
     """Reference arm: the CPU oracle on the host cores (rank 0 only)."""
     if rank != 0:
@@ -633,6 +675,12 @@ def run_ours(args, rank, world, local):
             cores = os.cpu_count() or 1
             fl, times, sample = cpu_oracle_sample(w, 1, rows_per_head=args.cpu_rows_per_head)
             result["cpu_baseline"] = cpu_baseline_record(fl, times, sample, cores)
+            if not args.no_configs:
+                try:
+                    result["cpu_baseline"]["config1_full"] = cpu_oracle_config1_full()
+                    result["cpu_baseline"]["config5_decode"] = cpu_oracle_decode_sample()
+                except Exception as e:
+                    result["cpu_baseline"]["other_configs_error"] = repr(e)
         print(json.dumps(result))
 
 
