@@ -687,7 +687,7 @@ def run_ours(args, rank, world, local):
 # DRAM bytes per prefill launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum), keyed by
 # (q heads, sequence length); lengths without a capture report no traffic figure.
 NCU_TRAFFIC_BYTES = {
-    (32, 16384): {"bytes": 145981696, "source": "profiles/prefill_kernel_llama_shape.md section 2 (65,293,056 read + 80,688,640 written)"},
+    (32, 16384): {"bytes": 143500000, "source": "profiles/prefill_kernel_llama_shape.md section 1 (65.4 MB read + 78.1 MB written per launch)"},
     (32, 131072): {"bytes": 44430000000, "source": "profiles/prefill_kernel_128k_and_paged_source.md section 1 (43.4 GB read + 1.03 GB written)"},
 }
 
