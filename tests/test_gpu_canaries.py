@@ -3,6 +3,8 @@ paged pools are carved out of one arena filled with a pattern, with guard bands 
 stage 1, prefill (both arrangements, all variants), the cache writes and decode, every guard byte must still hold
 the pattern.  Ragged lengths, so that tile tails and pad rows are exercised; the results are also checked against
 runs on ordinary allocations, so the carving itself is known to be harmless."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -13,6 +15,7 @@ pytestmark = pytest.mark.gpu
 
 GUARD = 4096
 PATTERN = 0xA5
+SUITE_ARRANGEMENT = int(os.environ.get("MPFA_TEST_ARRANGEMENT", "0"))   # what the rest of the suite runs on
 
 
 class Arena:
@@ -60,7 +63,11 @@ def test_stage1_and_prefill_stay_inside_their_buffers(arrangement):
     w = wl.prefill_workload("canary", 91, 2, 333, 4, 2, True, N_q=301, q_bias=True)   # ragged in both lengths
     q, k, v = w.q.cuda(), w.k.cuda(), w.v.cuda()
     ref = B_.stage1(q, k, v)
-    ref_out, ref32, st0 = B_.prefill(ref, True, w.softmax_scale, want_f32=True)
+    B_.mpfa_set_prefill_arrangement(0)
+    try:
+        ref_out, ref32, st0 = B_.prefill(ref, True, w.softmax_scale, want_f32=True)
+    finally:
+        B_.mpfa_set_prefill_arrangement(SUITE_ARRANGEMENT)
     arena = Arena(64 << 20)
     s1, ws = _stage1_in(arena, B_, w)
     out = arena.take(w.B * w.N_q * w.H_q * 128 * 2).view(torch.bfloat16).view(w.B, w.N_q, w.H_q, 128)
@@ -81,7 +88,7 @@ def test_stage1_and_prefill_stay_inside_their_buffers(arrangement):
         B_.mpfa_prefill(s1.q, s1.k, s1.v_fp8, s1.delta, s1.stats, 1.0, True, w.softmax_scale, out, o32, status)
         arena.check("prefill")
     finally:
-        B_.mpfa_set_prefill_arrangement(0)
+        B_.mpfa_set_prefill_arrangement(SUITE_ARRANGEMENT)
     if arrangement == 0:
         assert torch.equal(out.view(torch.uint16), ref_out.view(torch.uint16)) and torch.equal(o32, ref32)
     # the precision variants' operands and outputs
@@ -164,5 +171,5 @@ def test_cache_writes_paged_prefill_and_decode_stay_inside_their_buffers():
             B_.mpfa_prefill_paged(qc4, kv, table, seq, stats, 1.0, 128 ** -0.5, pout, None, status, q_lens=q_lens)
             arena.check(f"paged prefill, arrangement {arrangement}")
         finally:
-            B_.mpfa_set_prefill_arrangement(0)
+            B_.mpfa_set_prefill_arrangement(SUITE_ARRANGEMENT)
     assert int(status.item()) == 0
