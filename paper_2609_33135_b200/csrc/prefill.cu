@@ -623,10 +623,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const uint4 d = __ldg(dp + i);
             const uint32_t w[4] = {d.x, d.y, d.z, d.w};
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              s[8 * i + 2 * j] = __float_as_uint(__fadd_rn(__uint_as_float(s[8 * i + 2 * j]), __uint_as_float(w[j] << 16)));
-              s[8 * i + 2 * j + 1] =
-                  __float_as_uint(__fadd_rn(__uint_as_float(s[8 * i + 2 * j + 1]), __uint_as_float(w[j] & 0xFFFF0000u)));
+            for (int j = 0; j < 4; ++j) {   // packed pair: both halves round like the scalar add
+              float x0 = __uint_as_float(s[8 * i + 2 * j]), x1 = __uint_as_float(s[8 * i + 2 * j + 1]);
+              acc2(x0, x1, __uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u));
+              s[8 * i + 2 * j] = __float_as_uint(x0), s[8 * i + 2 * j + 1] = __float_as_uint(x1);
             }
           }
         }
@@ -657,10 +657,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const uint32_t w[4] = {d.x, d.y, d.z, d.w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              s[64 + 8 * i + 2 * j] =
-                  __float_as_uint(__fadd_rn(__uint_as_float(s[64 + 8 * i + 2 * j]), __uint_as_float(w[j] << 16)));
-              s[64 + 8 * i + 2 * j + 1] =
-                  __float_as_uint(__fadd_rn(__uint_as_float(s[64 + 8 * i + 2 * j + 1]), __uint_as_float(w[j] & 0xFFFF0000u)));
+              float x0 = __uint_as_float(s[64 + 8 * i + 2 * j]), x1 = __uint_as_float(s[64 + 8 * i + 2 * j + 1]);
+              acc2(x0, x1, __uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u));
+              s[64 + 8 * i + 2 * j] = __float_as_uint(x0), s[64 + 8 * i + 2 * j + 1] = __float_as_uint(x1);
             }
           }
         }
@@ -794,6 +793,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         TR(2 + grp, c, 5);
         if constexpr (PVB || PV4) {
           fence_proxy_async_smem();   // the P rows were written through the generic proxy, the MMA reads them through the async one
+          tc_fence_before();
+          warp_arrive(cx.bar(BAR_P_FULL + grp), lane);
+        } else if constexpr (EW) {   // measured: this variant is faster with the hand-over where the stores are
+          tmem_st_wait();
           tc_fence_before();
           warp_arrive(cx.bar(BAR_P_FULL + grp), lane);
         } else {
