@@ -32,6 +32,7 @@ def test_host_only_helpers(built):
     assert L.mpfa_fp4_sf_bytes(1, 2, 130) == 2 * 2 * 1024
     assert L.mpfa_delta_s_bytes(1, 4, 130) == 4 * 256 * 2
     assert L.mpfa_v_fp8_bytes(2, 2, 128) == 2 * 2 * 128 * 128
+    assert L.mpfa_v_fp4_bytes(2, 3, 130) == 2 * 3 * 2 * (8192 + 1024) and L.mpfa_v_fp4_bytes(1, 0, 5) == 0
     assert L.mpfa_fp4_codes_bytes(0, 1, 1) == 0
     assert L.mpfa_status_string(0) == b"ok" and L.mpfa_status_string(-3) == b"misaligned buffer"
     # layout maps agree with the documented formulas and are bijections
@@ -60,6 +61,8 @@ def test_argument_errors_without_gpu(built):
     st = binding._Stats(0, 0, 0, 0)
     assert L.mpfa_quantize_qk(None, None, 1, 1, 1, 1, 1, 0, ctypes.byref(st), None, None, None, None, 0, None) == -1
     assert L.mpfa_quantize_v(None, 1, 1, 1, 1.0, None, None) == -1
+    assert L.mpfa_quantize_v_fp4(None, 1, 1, 1, 1.0, None, None) == -1
+    assert L.mpfa_pack_v_bf16(None, 1, 1, 1, None, None) == -1
     assert L.mpfa_prefill(None, None, None, None, None, 1.0, 0, 1.0, None, None, None, None) == -1
     assert L.mpfa_prefill_variant(None, None, None, None, None, 1.0, 0, 1.0, 0, None, None, None, None) == -1
     assert L.mpfa_prefill_variant(None, None, None, None, None, 1.0, 0, 1.0, 5, None, None, None, None) == -1
