@@ -94,7 +94,7 @@ def test_v_quantizer_reproduces_values_built_from_codes():
     c4 = rng.integers(0, 16, (B, H, 128, 4, 16), dtype=np.uint8)
     c4[..., 0] = 7                                                        # +6 in every block
     c4[(c4 & 7) == 0] = 0                                                 # no negative zeros
-    sc = rng.integers(0x28, 0x48, (B, H, 128, 4), dtype=np.uint8)          # normal scales around 1
+    sc = rng.integers(0x28, 0x48, (B, H, 128, 4), dtype=np.uint8)          # normal scales close to 1.0
     x = _signed_vals(c4) * (_e4m3_vals(sc)[..., None] * d)                # exact in BF16: <= 2+4 significant bits
     x = x.reshape(B, H, 128, N).transpose(0, 3, 1, 2).astype(np.float32)
     bits = (np.ascontiguousarray(x).view(np.uint32) >> 16).astype(np.uint16)
