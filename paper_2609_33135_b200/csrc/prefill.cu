@@ -57,12 +57,13 @@ constexpr int NTHREADS = 512;
 // setmaxnreg only moves registers inside the pool the CTA got at launch (512 threads x the 128 registers of the
 // launch bound); a request beyond the pool would block forever, so the split is checked here.
 #ifndef MPFA_REGS_UTIL_PAGED
-#define MPFA_REGS_UTIL_PAGED 88
-#define MPFA_REGS_CORR_PAGED 88
+#define MPFA_REGS_UTIL_PAGED 64
+#define MPFA_REGS_CORR_PAGED 112
 #endif
 constexpr int REGS_SOFTMAX = 168;
 // measured: the contiguous kernel gains 4 % when the correction warps' epilogue (two accumulator chunks in
-// registers) does not spill; the paged variant's producer and re-tiling warps want the registers instead
+// registers) does not spill; the paged variant's producer and re-tiling warps need a few more (measured on the
+// config-2 shape from pages: 56/120 1217, 64/112 1223, 72/104 1211, 80/96 1172, 88/88 1173 TFLOPS)
 template <bool PAGED> constexpr int REGS_UTIL = PAGED ? MPFA_REGS_UTIL_PAGED : 56;
 template <bool PAGED> constexpr int REGS_CORR = PAGED ? MPFA_REGS_CORR_PAGED : 120;
 static_assert(4 * REGS_UTIL<false> + 8 * REGS_SOFTMAX + 4 * REGS_CORR<false> <= 16 * 128, "register pool");
