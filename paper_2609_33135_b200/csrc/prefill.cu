@@ -31,8 +31,8 @@
 //                (the older one times the last alpha) and writes O / (448 l) * v_scale as BF16.
 // Tensor memory (512 columns): S [0,128) O0 [128,256) O1 [256,384), P_hat0 [384,416)
 // P_hat1 [416,448), scale factors of two query tiles [448,464) and of two K blocks [464,472) [472,480).
-// Register budget is moved between the roles with setmaxnreg (56 for warps 0-3, 168 for the softmax warps,
-// 120 for the correction warps, whose epilogue holds two accumulator chunks at once).
+// Register budget is moved between the roles with setmaxnreg (72 for warps 0-3, 168 for the softmax warps,
+// 104 for the correction warps, whose epilogue holds two accumulator chunks at once).
 // Template parameter EW: the compensation-placement ablation (mpfa_prefill_variant): no seed MMA, Delta_S added
 // element by element by the softmax threads.
 //
@@ -60,12 +60,18 @@ constexpr int NTHREADS = 512;
 #define MPFA_REGS_UTIL_PAGED 64
 #define MPFA_REGS_CORR_PAGED 112
 #endif
-constexpr int REGS_SOFTMAX = 168;
-// measured: the contiguous kernel gains 4 % when the correction warps' epilogue (two accumulator chunks in
-// registers) does not spill; the paged variant's producer and re-tiling warps need a few more (measured on the
+#ifndef MPFA_REGS_SOFTMAX
+#define MPFA_REGS_SOFTMAX 168
+#define MPFA_REGS_UTIL 72
+#define MPFA_REGS_CORR 104
+#endif
+constexpr int REGS_SOFTMAX = MPFA_REGS_SOFTMAX;
+// measured (16K / 64K TFLOPS, utility / softmax / correction): 56/168/120 1325 / 1418, 72/168/104 1339 / 1447,
+// 72/160/112 1335 / 1447, 64/168/112 1307 / 1423, 80/160/104 1310 / 1435, 96/160/88 1302 / 1427, 152 for the softmax
+// warps 1243 / 1318 (their row spills); the paged variant's producer and re-tiling warps need a few more (measured on the
 // config-2 shape from pages: 56/120 1217, 64/112 1223, 72/104 1211, 80/96 1172, 88/88 1173 TFLOPS)
-template <bool PAGED> constexpr int REGS_UTIL = PAGED ? MPFA_REGS_UTIL_PAGED : 56;
-template <bool PAGED> constexpr int REGS_CORR = PAGED ? MPFA_REGS_CORR_PAGED : 120;
+template <bool PAGED> constexpr int REGS_UTIL = PAGED ? MPFA_REGS_UTIL_PAGED : MPFA_REGS_UTIL;
+template <bool PAGED> constexpr int REGS_CORR = PAGED ? MPFA_REGS_CORR_PAGED : MPFA_REGS_CORR;
 static_assert(4 * REGS_UTIL<false> + 8 * REGS_SOFTMAX + 4 * REGS_CORR<false> <= 16 * 128, "register pool");
 static_assert(4 * REGS_UTIL<true> + 8 * REGS_SOFTMAX + 4 * REGS_CORR<true> <= 16 * 128, "register pool");
 // the utility and correction warps give registers back (setmaxnreg.dec: the target must not exceed the 128 of the
