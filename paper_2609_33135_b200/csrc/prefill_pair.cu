@@ -25,12 +25,13 @@
 //                (Eq. 6), and at the end of an item O_r / (448 l) * v_scale -> BF16 (Algorithm 1 line 17).
 // Tensor memory (496 of 512 columns): S [0,128), O_0 [128,256), O_1 [256,384), P_hat_0 [384,416), P_hat_1 [416,448),
 // scale factors of 2 x 2 query tiles [448,480) and of two K blocks [480,496).
-// Measured on B200 against the one-query-tile kernel of prefill.cu (same arithmetic row by row): 1046 against 1273
-// TFLOPS at 16K, 1142 against 1397 at 64K, although this kernel executes 12 % fewer instructions per block.  With the
-// rescaling of O compiled out both take the same time; with it, one accumulator per tile puts the rescale between two
+// Measured on B200 against the one-query-tile kernel of prefill.cu (same arithmetic row by row): 1251 against 1338
+// TFLOPS at 16K, 1317 against 1445 at 64K (0.94x / 0.91x), although this kernel executes 12 % fewer instructions per
+// block.  Before P-hat was handed to the P V issuer late (at the top of the stage's next block instead of after its
+// tensor-memory stores) it stood at 1105 / 1188: with one accumulator per tile the rescale of O sits between two
 // dependent P V MMAs of that tile (the other kernel alternates two accumulators), and at these lengths some row of a
-// warp moves its maximum in most blocks.  This arrangement is therefore not the default
-// (mpfa_set_prefill_arrangement).
+// warp moves its maximum in most blocks; with the rescaling compiled out both kernels take the same time.  This
+// arrangement is therefore not the default (mpfa_set_prefill_arrangement).
 // Template parameter EW: the compensation-placement ablation (no seed MMA, Delta_S added element by element by the
 // softmax threads).  Every mbarrier wait is bounded; on expiry the CTA raises MPFA_DEV_TIMEOUT in *device_status,
 // all roles leave their loops, outstanding TMA copies are drained and tensor memory is released.
@@ -66,8 +67,15 @@ constexpr int KSTAGES = 4;
 constexpr int VSTAGES = 3;
 constexpr int NTHREADS = 512;
 constexpr int REGS_SOFTMAX = 168;
-template <bool PAGED> constexpr int REGS_UTIL = PAGED ? 88 : 56;
-template <bool PAGED> constexpr int REGS_CORR = PAGED ? 88 : 120;
+#ifndef MPFA_PAIR_LATE
+#define MPFA_PAIR_LATE 1
+#endif
+#ifndef MPFA_PAIR_REGS_UTIL
+#define MPFA_PAIR_REGS_UTIL 72
+#define MPFA_PAIR_REGS_CORR 104
+#endif
+template <bool PAGED> constexpr int REGS_UTIL = PAGED ? 64 : MPFA_PAIR_REGS_UTIL;
+template <bool PAGED> constexpr int REGS_CORR = PAGED ? 112 : MPFA_PAIR_REGS_CORR;
 // setmaxnreg only moves registers inside the pool the CTA got at launch (512 threads x 128 registers); a request
 // beyond the pool would block forever, and a "dec" to more than 128 or an "inc" to less is an illegal instruction.
 static_assert(4 * REGS_UTIL<false> + 8 * REGS_SOFTMAX + 4 * REGS_CORR<false> <= 16 * 128, "register pool");
@@ -501,11 +509,22 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int limit = (r_abs >= it.nq) ? -1   // a row past the request's own query count sees nothing
                         : p.causal ? min(it.nkv - 1, r_abs + (it.nkv - it.nq)) : it.nkv - 1;   // last visible key
       const float lam = __fmul_rn(__fmul_rn(__fmul_rn(p.softmax_scale, 1.4426950408889634f), p.q_gscale[it.b]), p.k_gscale[it.b]);
+#if MPFA_PAIR_LATE
+      bool p_pending = false;
+#endif
       float m_run = -INFINITY;   // running maximum (Eq. 3)
       float l_run = 0.0f;        // running sum of 448 P (Eq. 5)
       for (int jb = T - 1; jb >= 0; --jb, ++n) {
         const int key0 = jb * TILE;
         TR(r, n, 0);
+#if MPFA_PAIR_LATE == 2
+        if (p_pending) {
+          tmem_st_wait();
+          tc_fence_before();
+          warp_arrive(cx.bar(BAR_P_FULL + r), lane);
+          p_pending = false;
+        }
+#endif
         if (!__all_sync(0xffffffffu, cx.wait(BAR_S_FULL + r, n & 1u))) { ok = false; break; }
         TR(r, n, 1);
         tc_fence_after();
@@ -516,6 +535,14 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tmem_ld32(tS, s0);
           tmem_ld32(tS + 32, s1);
         }
+#if MPFA_PAIR_LATE == 1
+        if (p_pending) {
+          tmem_st_wait();
+          tc_fence_before();
+          warp_arrive(cx.bar(BAR_P_FULL + r), lane);
+          p_pending = false;
+        }
+#endif
         // P V of the stage's previous block has consumed the P_hat columns (tested early, used before the stores)
         const bool pe_early = (n < 1) || cx.probe(BAR_P_EMPTY + r, (n - 1) & 1u);
         const bool ragged = key0 + TILE - 1 > limit;   // diagonal / ragged block only
@@ -527,6 +554,14 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tmem_ld32(tS + 64, s2);
           tmem_ld32(tS + 96, s3);
         }
+#if MPFA_PAIR_LATE == 3
+        if (p_pending) {
+          tmem_st_wait();
+          tc_fence_before();
+          warp_arrive(cx.bar(BAR_P_FULL + r), lane);
+          p_pending = false;
+        }
+#endif
         if constexpr (EW) {
           const uint4 *dp = reinterpret_cast<const uint4 *>(
               p.delta + ((size_t)it.b * p.H_q + it.hq) * (size_t)(p.nk_tiles * TILE) + key0);
@@ -634,12 +669,24 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tmem_st8(tP + (c0 >> 2), packed);
         }
         l_run = __fadd_rn(__fmul_rn(alpha, l_run), (sum0 + sum1) + (sum2 + sum3));
+#if MPFA_PAIR_LATE
+        p_pending = true;
+#else
         tmem_st_wait();
         TR(r, n, 5);
         tc_fence_before();
         warp_arrive(cx.bar(BAR_P_FULL + r), lane);
+#endif
         TR(r, n, 6);
       }
+#if MPFA_PAIR_LATE
+      if (p_pending) {
+        tmem_st_wait();
+        tc_fence_before();
+        warp_arrive(cx.bar(BAR_P_FULL + r), lane);
+        p_pending = false;
+      }
+#endif
       if (!ok) break;
       s_l[(u & 3) * 128 + row] = l_run;
       warp_arrive(cx.bar(BAR_L_FULL + r * 4 + (u & 3)), lane);
@@ -684,7 +731,11 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tmem_ld32(tO + c0, v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__fmul_rn(__uint_as_float(v[i]), alpha));
+                for (int i = 0; i < 32; i += 2) {   // packed pairs: half the issue slots, same roundings
+                  float y0, y1;
+                  mul2(y0, y1, __uint_as_float(v[i]), __uint_as_float(v[i + 1]), alpha);
+                  v[i] = __float_as_uint(y0), v[i + 1] = __float_as_uint(y1);
+                }
                 tmem_st32(tO + c0, v);
               }
               tmem_st_wait();
