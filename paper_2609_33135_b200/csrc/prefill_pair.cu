@@ -25,8 +25,8 @@
 //                (Eq. 6), and at the end of an item O_r / (448 l) * v_scale -> BF16 (Algorithm 1 line 17).
 // Tensor memory (496 of 512 columns): S [0,128), O_0 [128,256), O_1 [256,384), P_hat_0 [384,416), P_hat_1 [416,448),
 // scale factors of 2 x 2 query tiles [448,480) and of two K blocks [480,496).
-// Measured on B200 against the one-query-tile kernel of prefill.cu (same arithmetic row by row): 1251 against 1338
-// TFLOPS at 16K, 1317 against 1445 at 64K (0.94x / 0.91x), although this kernel executes 12 % fewer instructions per
+// Measured on B200 against the one-query-tile kernel of prefill.cu (same arithmetic row by row): 1264 against 1338
+// TFLOPS at 16K, 1354 against 1445 at 64K (0.94x), although this kernel executes 12 % fewer instructions per
 // block.  Before P-hat was handed to the P V issuer late (at the top of the stage's next block instead of after its
 // tensor-memory stores) it stood at 1105 / 1188: with one accumulator per tile the rescale of O sits between two
 // dependent P V MMAs of that tile (the other kernel alternates two accumulators), and at these lengths some row of a
@@ -71,8 +71,8 @@ constexpr int REGS_SOFTMAX = 168;
 #define MPFA_PAIR_LATE 1
 #endif
 #ifndef MPFA_PAIR_REGS_UTIL
-#define MPFA_PAIR_REGS_UTIL 72
-#define MPFA_PAIR_REGS_CORR 104
+#define MPFA_PAIR_REGS_UTIL 56   // measured for this kernel: 56/120 1264 / 1354, 72/104 1245 / 1318, 80/96 1228 / 1288
+#define MPFA_PAIR_REGS_CORR 120
 #endif
 template <bool PAGED> constexpr int REGS_UTIL = PAGED ? 64 : MPFA_PAIR_REGS_UTIL;
 template <bool PAGED> constexpr int REGS_CORR = PAGED ? 112 : MPFA_PAIR_REGS_CORR;
