@@ -109,15 +109,19 @@ enum {
 };
 static_assert(NUM_BARS <= 64, "barrier table");
 // Shared-memory layout.  PVK selects the operands of the second MMA (mpfa_prefill_variant): 0 = the method (FP8);
-// 1 = the NVFP4 + BF16 precision assignment: V tiles are BF16 (32 KB, two stages), P is handed to the second MMA
-// through shared memory as a K-major BF16 A operand (2 x 32 KB), and the K ring has three stages to make room;
+// 1 = the NVFP4 + BF16 precision assignment: V tiles are BF16 (32 KB, three stages), P is handed to the second MMA
+// through shared memory as a K-major BF16 A operand (2 x 32 KB), and the K ring has two stages to make room;
 // 2 = the NVFP4 + NVFP4 assignment: V tiles are channel-major FP4 (8 KB + 1 KB of block scales), P goes through
 // shared memory as a K-major FP4 A operand (2 x 8 KB) with its block scales (2 x 1 KB).
 template <int PVK>
 struct Lay {
   static constexpr bool PVB = PVK == 1, PV4 = PVK == 2;
-  static constexpr int KST = PVB ? 3 : KSTAGES;
-  static constexpr int VST = PVB ? 2 : VSTAGES;
+  // ring depths measured on the product kernel (16K / 64K TFLOPS, K / V stages): 4/3 1340 / 1446, 6/3 1342 / 1452, 4/4
+  // 1325 / 1464, 3/3 1329 / 1450, 2/3 within 1 % of 4/3, but 4/2 and 3/2 894 / 822: a V stage is held from its load until
+  // the P V MMA of its block, which the late hand-over of P-hat issues a block later.  The BF16 variant therefore gives
+  // up K stages, not V stages, to make room for its 32 KB tiles.
+  static constexpr int KST = PVB ? 2 : KSTAGES;
+  static constexpr int VST = VSTAGES;
   static constexpr uint32_t V_BYTES = PVB ? 32768u : (PV4 ? 8192u : 16384u);
   static constexpr uint32_t OFF_Q = 0;                               // 2 tiles (the next tile's queries are prefetched)
   static constexpr uint32_t OFF_K = OFF_Q + 2 * 8192;
